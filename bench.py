@@ -1,0 +1,270 @@
+#!/usr/bin/env python
+"""Throughput of the fused DHQ forward (coordinates per second) on N GPUs of one node.
+
+    python bench.py --gpus 1 --steps 200 --warmup 5
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference ...      # the CPU oracle on the host cores, same metric
+
+A step is one dhq_forward call over the workload's whole coordinate grid (one launch of the
+fused kernel).  Inputs are seeded and synthetic (SIREN-initialised network, pixel grid).  With
+N > 1 every rank runs the same grid on its own GPU (independent replicas, no collective on the
+data path), so the aggregate is N times the work: weak scaling.
+
+Timing: CUDA events on the launching stream around each step, an L2 flush (a write of a buffer
+larger than L2) between steps and outside the events, the per-step times summed; the maximum
+over ranks is reported.  SM clocks and throttle reasons are sampled through NVML while the timed
+steps run.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import dhq_inputs  # noqa: E402
+
+METRIC = "coords/sec, fused W8A8 DHQ INR forward"
+UNIT = "coords/s"
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+
+
+def alu_laneops_per_coord(dims) -> float:
+    """Plain-ALU lane operations the method needs per coordinate: per element of every hidden
+    activation vector log2(w) butterfly adds plus 7 (int->float, scale+bias fma, 2 for the sine's
+    range handling, quantizer multiply, rounding, packing/abs-max)."""
+    w = dims[1]
+    hidden_vectors = len(dims) - 2
+    return float(hidden_vectors * w * (7 + int(np.log2(w))))
+
+
+class ClockSampler:
+    """Polls NVML for the SM clock and the clock-event reasons of one GPU while running."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _poll(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def time_oracle(workload, steps, warmup, sample_tokens):
+    """The CPU oracle, as it stands, on `sample_tokens` coordinates of the workload."""
+    from oracle import dhq_oracle as orc
+    weights, biases = workload.network()
+    net = orc.prepare(weights, biases, workload.dims, workload.omega0, workload.w_bits, workload.a_bits,
+                      workload.w_gran, workload.a_gran)
+    coords = workload.coords()[:sample_tokens]
+    if workload.a_gran == 0:
+        orc.calibrate(net, coords)
+    for _ in range(warmup):
+        orc.forward(net, coords[: max(1, sample_tokens // 8)])
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        orc.forward(net, coords)
+    dt = (time.perf_counter() - t0) / steps
+    return coords.shape[0] / dt, dt, orc.threads()
+
+
+def run_reference(args, workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = min(workload.n, 16384)
+    steps = max(1, min(args.steps, 5))
+    warmup = min(args.warmup, 1)
+    value, dt, cores = time_oracle(workload, steps, warmup, sample)
+    desc = f"first {sample} coordinates of the {workload.grid[0]}x{workload.grid[1]} grid per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 codes, int32 accumulate, fp64 epilogue", "data": "synthetic",
+        "config": {"workload": workload.name, "dims": list(workload.dims), "bits": [workload.w_bits, workload.a_bits]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, workload):
+    import torch
+    import torch.distributed as dist
+    import paper_2508_13478_b200 as dhq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dhq.load_library()
+
+    weights, biases = workload.network()
+    coords_np = workload.coords()
+    n, d_L = coords_np.shape[0], workload.dims[-1]
+    W = [torch.from_numpy(w).cuda() for w in weights]
+    B = [torch.from_numpy(b).cuda() for b in biases]
+    h = dhq.dhq_prepare(workload.dims, W, B, workload.omega0, workload.w_bits, workload.a_bits,
+                        workload.w_gran, workload.a_gran)
+    coords = torch.from_numpy(coords_np).cuda()
+    out = torch.empty((n, d_L), dtype=torch.float32, device="cuda")
+    coords_host = torch.from_numpy(coords_np).pin_memory()
+    out_host = torch.empty((n, d_L), dtype=torch.float32).pin_memory()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # > 126 MB of L2
+    stream = torch.cuda.current_stream()
+
+    dhq.dhq_calibrate(h, coords)          # per-tensor scales frozen on the workload's grid; no-op per token
+    for _ in range(max(args.warmup, 3)):
+        dhq.dhq_forward(h, coords, out)
+        dhq.dhq_forward_host(h, coords_host, out_host)
+    torch.cuda.synchronize()
+    if dhq.dhq_last_status(h) != 0:
+        raise SystemExit("device-side wait timed out during warm-up")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        barrier()
+        for a, b in evs:
+            flush.fill_(1)
+            a.record(stream)
+            fn()
+            b.record(stream)
+        barrier()
+        return sum(a.elapsed_time(b) for a, b in evs)   # ms
+
+    launches0 = dhq.dhq_launch_count(h)
+    with ClockSampler(physical_gpu_index(local_rank)) as clocks:
+        total_ms = timed(lambda: dhq.dhq_forward(h, coords, out), args.steps)
+    launches = dhq.dhq_launch_count(h) - launches0
+    e2e_ms = timed(lambda: dhq.dhq_forward_host(h, coords_host, out_host), args.steps)
+    status = dhq.dhq_last_status(h)
+
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+    value = n * world / (ms_per_step * 1e-3)
+    e2e_value = n * world / (e2e_ms / args.steps * 1e-3)
+
+    if rank == 0:
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except Exception:
+            pass
+        sm_max = float(peaks.get("sm_max_mhz", 1965.0))
+        alu_peak = SM_COUNT * FP32_LANES_PER_SM * sm_max * 1e6 / 1e12            # T lane-ops/s
+        achieved = alu_laneops_per_coord(workload.dims) * n / (ms_per_step * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8 codes, int32 accumulate, fp32 epilogue",
+            "data": "synthetic",
+            "config": {"workload": workload.name, "dims": list(workload.dims), "coords_per_step": n,
+                       "bits": [workload.w_bits, workload.a_bits], "w_gran": workload.w_gran,
+                       "a_gran": workload.a_gran, "l2": "flushed between steps (256 MB write)",
+                       "parallelism": f"{world} independent replica(s)"},
+            "clocks": clocks.summary(),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * 8, "d2h_bytes_per_step": n * d_L * 4},
+            "gpu_launches": launches,
+            "roofline": {"bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "Tlaneop/s",
+                         "frac": achieved / alu_peak, "traffic": None,
+                         "peak_source": "148 SMs x 128 fp32 lanes x max SM clock (derived, not measured)"},
+            "device_status": status,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            sample = min(n, 65536)
+            v, dt, cores = time_oracle(workload, 1, 1, sample)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"first {sample} coordinates of the grid, one pass ({dt:.1f} s)"}
+        print(json.dumps(line), flush=True)
+    dhq.dhq_destroy(h)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C2", choices=sorted(dhq_inputs.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    workload = dhq_inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, workload)
+    else:
+        run_ours(args, workload)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,192 @@
+/*
+ * dhq.h - C ABI of the B200 library for the fully quantized forward pass of a sinusoidal INR
+ * (DHQ, arXiv 2508.13478).
+ *
+ * The network is f_theta : coordinate -> signal value (Section II-A of the paper), an MLP with L
+ * linear layers of sizes dims[0] = 2, dims[1..L-1] = w, dims[L] in 1..4.  Every layer l computes
+ * (Section III-B and III-C):
+ *
+ *     x~   = H_K x_l                      online Walsh-Hadamard rotation of the layer input (Eq. 3)
+ *     q_x  = Q_a(x~)                      activation quantizer ("dynamic quantization module")
+ *     acc  = q_x * q_W^T                  integer matmul, int32 accumulation, on the tensor cores
+ *     z    = s_W s_x acc + b              dequantize and add the bias
+ *     x_{l+1} = sin(omega0 z)             hidden layers; the last layer returns z (no activation)
+ *
+ * with q_W = Q_w(W H_K / K) prepared once (Eq. 4-5, the factor acting on the input dimension;
+ * H is symmetric, so (W H/K)(H x) = W x).  The 2 inputs are zero-padded to K = 4 and the outputs
+ * of the last layer to 4, so every Hadamard size is a power of two.
+ *
+ * Quantizer Q (one quantizer for all layers, Section III-B), as implemented: symmetric,
+ * qmax = 2^(bits-1) - 1, a = max |v| over the tensor / output channel / token,
+ * s = a / qmax and inv = qmax / a in IEEE fp32, q = clamp(round_half_even(fl32(v * inv)), +-qmax),
+ * a = 0 gives s = inv = 0 and all-zero codes.  Codes of every bit-width live in int8 lanes.
+ * The fp32 rotation adds in the order of the in-place butterfly with strides 1, 2, 4, ..., K/2,
+ * where the pair (i, i+h) becomes (a+b, a-b); outputs are in natural (Sylvester) order.
+ *
+ * Conventions for every call:
+ *   - Pointers named "device" are CUDA device pointers owned by the caller; the library never
+ *     frees them and does not keep them after the call's stream work has run.  "host" pointers are
+ *     ordinary host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is enqueued
+ *     on it and the call returns without waiting, unless stated otherwise.
+ *   - Argument errors are reported by the return value and enqueue nothing.  Conditions found on
+ *     the device (a bounded wait that ran out) are recorded in a status word read by
+ *     dhq_last_status.  Nothing traps, aborts or throws.
+ *   - One forward may be in flight per handle at a time.  Handles belong to the device that was
+ *     current in dhq_prepare; that device must be current in later calls.
+ */
+#ifndef DHQ_H_
+#define DHQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define DHQ_API
+#else
+#define DHQ_API __attribute__((visibility("default")))
+#endif
+
+typedef struct dhq_handle_s *dhq_handle_t; /* opaque, owned by the library */
+
+typedef enum {
+    DHQ_OK = 0,
+    DHQ_ERR_INVALID_ARG = 1,    /* NULL pointer, negative size, malformed config           */
+    DHQ_ERR_UNSUPPORTED = 2,    /* shape or option outside what the kernels implement      */
+    DHQ_ERR_ALLOC = 3,          /* device or host allocation failed                        */
+    DHQ_ERR_CUDA = 4,           /* a CUDA runtime call failed                              */
+    DHQ_ERR_NOT_CALIBRATED = 5, /* per-tensor activation scales requested but not frozen   */
+    DHQ_ERR_TIMEOUT = 6         /* a bounded wait inside a kernel ran out                  */
+} dhq_status_t;
+
+/* Quantizer granularity: weights per tensor or per output channel; activations per tensor
+ * (static: frozen by calibration) or per token (dynamic: from each coordinate's own values). */
+typedef enum { DHQ_GRAN_TENSOR = 0, DHQ_GRAN_CHANNEL_OR_TOKEN = 1 } dhq_gran_t;
+
+/* Which side of Eq. 4 is applied.  DHQ_ROT_INPUT is the implemented path. */
+typedef enum { DHQ_ROT_INPUT = 0, DHQ_ROT_BOTH = 1, DHQ_ROT_NONE = 2 } dhq_rot_t;
+
+typedef struct {
+    int n_layers;       /* L linear layers, 2..16                                          */
+    const int *dims;    /* host, L+1 ints: 2, w, ..., w, d_L; w a power of two in 64..512, */
+                        /* the same for all hidden layers; d_L in 1..4                     */
+    int w_bits, a_bits; /* 2..8                                                            */
+    float omega0;       /* sine frequency of layers 1..L-1                                 */
+    dhq_gran_t w_gran;
+    dhq_gran_t a_gran;
+    dhq_rot_t rotation; /* only DHQ_ROT_INPUT is accepted                                  */
+} dhq_config_t;
+
+/*
+ * Per-layer dump targets for dhq_forward_debug.  Each member is a host array of L device
+ * pointers (entry l-1 for layer l); a NULL member or NULL entry is skipped.  K and M are the
+ * padded sizes of the layer as the definition pads them: K = 4 for layer 1, else w; M = 4 for
+ * layer L, else w.
+ */
+typedef struct {
+    float **X;      /* [n][K] fp32   layer input (layer 1: [x, y, 0, 0])                   */
+    int8_t **codes; /* [n][K] int8   quantized rotated input                               */
+    float **s_x;    /* [n]    fp32   activation scale of each token                        */
+    int32_t **acc;  /* [n][M] int32  integer accumulators                                  */
+    float **Y;      /* [n][M] fp32   layer output (after the sine for hidden layers)       */
+} dhq_debug_bufs_t;
+
+/*
+ * Weight side, once per network (Eq. 4-5 and the quantizer of Section III-B), run on the
+ * device: pad, rotate every row by H_K in fp32, scale by the exact 1/K, quantize, and pack the
+ * codes into the shared-memory image the tensor-core kernel loads.
+ *   cfg    host.
+ *   W      host array of L device pointers; W[l-1] is row-major [dims[l]][dims[l-1]] fp32
+ *          (the layout of a PyTorch nn.Linear weight).
+ *   b      host array of L device pointers; b[l-1] is [dims[l]] fp32.
+ *   out    receives the handle.  The caller releases it with dhq_destroy.
+ * Allocates device memory; enqueues the preparation kernels on `stream` and returns.  W and b
+ * may be released once that stream work has completed.
+ * Errors: INVALID_ARG (NULL, n_layers out of range), UNSUPPORTED (dims[0] != 2, width not a
+ * power of two in 64..512 or not uniform, d_L outside 1..4, bits outside 2..8, rotation other
+ * than DHQ_ROT_INPUT), ALLOC, CUDA.
+ */
+DHQ_API dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W,
+                                 const float *const *b, void *stream, dhq_handle_t *out);
+
+/*
+ * Freeze the per-tensor activation scales (a_gran = DHQ_GRAN_TENSOR) on a set of coordinates:
+ * for l = 1..L, a_l = max over the n tokens and the K features of |H_K x_l|, taken with layers
+ * < l already quantized with their frozen scales (the run-time statistic of the "dynamic
+ * quantization module", Section III-C, taken once and kept, so that a coordinate's output does
+ * not depend on the batch it arrives in).
+ *   coords device [n][2] fp32, n >= 1.
+ * Enqueues L passes on `stream`.  With a_gran = per token the call is a no-op returning DHQ_OK.
+ * Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+DHQ_API dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void *stream);
+
+/*
+ * The forward pass f_theta over n coordinates: one launch of the fused kernel, activations
+ * never leave the SM between layers.
+ *   coords device [n][2] fp32 (x, y per token), 8-byte aligned.
+ *   out    device [n][d_L] fp32, dense.
+ * n = 0 is a no-op; n need not be a multiple of any tile size.  If the handle uses per-tensor
+ * activation scales and none are frozen yet, this call first calibrates on its own coordinates
+ * (as dhq_calibrate) and freezes them; later calls reuse them.
+ * Non-finite coordinates give unspecified values but do not hang.
+ * Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+DHQ_API dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *out,
+                                 void *stream);
+
+/*
+ * As dhq_forward but with HOST buffers: copies coords to the device, runs the forward and
+ * copies the result back, all enqueued on `stream` (pass pinned memory for the copies to be
+ * asynchronous).  Uses staging buffers owned by the handle, grown on demand (this may allocate
+ * and synchronize the first time a larger n is seen).
+ */
+DHQ_API dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t n,
+                                      float *out_host, void *stream);
+
+/*
+ * Layer-by-layer forward that writes every intermediate to the caller's buffers (see
+ * dhq_debug_bufs_t), for checking each stage against a reference.  Same arithmetic as
+ * dhq_forward, operation for operation, so `out` and Y[L-1] equal dhq_forward's output bit for
+ * bit; activations go through device memory between layers, in chunks, using scratch memory
+ * owned by the handle.  `out` and `bufs` may each be NULL.  Requires frozen scales when
+ * a_gran = per tensor (NOT_CALIBRATED otherwise).
+ */
+DHQ_API dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int64_t n, float *out,
+                                       const dhq_debug_bufs_t *bufs, void *stream);
+
+/*
+ * Read back one prepared layer (1-based).  Synchronizes the handle's preparation work.
+ *   codes       host [M][K] int8, row-major, unswizzled (M, K as in dhq_debug_bufs_t), or NULL.
+ *   w_scales    host [M] fp32 (per-tensor: the same value M times), or NULL.
+ *   act_absmax  host, one fp32: the frozen per-tensor a_l, or NaN if not frozen / per token;
+ *               or NULL.
+ * Errors: INVALID_ARG (layer out of range), CUDA.
+ */
+DHQ_API dhq_status_t dhq_get_layer(dhq_handle_t h, int layer, int8_t *codes, float *w_scales,
+                                   float *act_absmax);
+
+/* Layer sizes as the library pads them: K, M of layer `layer` (1-based).  Either may be NULL. */
+DHQ_API dhq_status_t dhq_layer_dims(dhq_handle_t h, int layer, int *K, int *M);
+
+/*
+ * Device-side status of the handle: DHQ_OK, or DHQ_ERR_TIMEOUT if a bounded wait inside a
+ * kernel ran out since the last call.  Synchronizes the device and clears the word.
+ */
+DHQ_API dhq_status_t dhq_last_status(dhq_handle_t h);
+
+/* Number of kernels the library has launched for this handle since it was created. */
+DHQ_API int64_t dhq_launch_count(dhq_handle_t h);
+
+/* Waits for the handle's outstanding work, then frees everything it owns.  NULL is ignored. */
+DHQ_API void dhq_destroy(dhq_handle_t h);
+
+DHQ_API const char *dhq_status_string(dhq_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DHQ_H_ */

@@ -1,0 +1,48 @@
+/*
+ * dhq_peaks.h - micro-benchmarks of the execution pipes that bound the DHQ forward kernel.
+ *
+ * The paper (arXiv 2508.13478) has no counterpart: its cost model is FPGA resources (Table 2).
+ * On a GPU the same datapath (Section III-C: MAC array, activation, dynamic quantization) is
+ * bounded by the int8 tensor pipe, the special-function unit (sine) and the plain fp32/integer
+ * pipes, whose peaks these loops measure so that roofline fractions have measured denominators.
+ */
+#ifndef DHQ_PEAKS_H_
+#define DHQ_PEAKS_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define DHQ_PEAKS_API
+#else
+#define DHQ_PEAKS_API __attribute__((visibility("default")))
+#endif
+
+typedef enum {
+    DHQ_PIPE_FFMA = 0,     /* fp32 fused multiply-add, independent chains          */
+    DHQ_PIPE_FADD = 1,     /* fp32 add                                             */
+    DHQ_PIPE_MUFU_SIN = 2, /* sin.approx.f32 (multiply by 1/2pi + special function) */
+    DHQ_PIPE_I2F = 3,      /* cvt.rn.f32.s32                                       */
+    DHQ_PIPE_F2I = 4,      /* cvt.rni.s32.f32                                      */
+    DHQ_PIPE_PRMT = 5,     /* byte permute                                         */
+    DHQ_PIPE_FMNMX = 6,    /* fp32 min/max                                         */
+    DHQ_PIPE_TENSOR_I8 = 7 /* tcgen05.mma kind::i8, 128x256x32, operands resident in shared memory */
+} dhq_pipe_t;
+
+/*
+ * Runs one micro-benchmark on the current device (all SMs busy), timed with CUDA events on
+ * `stream` after one warm-up launch; synchronizes.
+ *   ops_per_s  host, receives operations per second: instructions x 32 lanes for the scalar
+ *              pipes (an FMA counts as one), 2*M*N*K integer operations per MMA for the tensor
+ *              pipe.
+ *   ms         host, receives the duration of the timed launch, or NULL.
+ * Returns 0 on success, a negative value on a CUDA error or unknown pipe, 1 if the tensor-pipe
+ * loop hit its bounded wait.
+ */
+DHQ_PEAKS_API int dhq_measure_pipe(int pipe, int iters, void *stream, double *ops_per_s, double *ms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DHQ_PEAKS_H_ */

@@ -1,0 +1,13 @@
+"""B200 (sm_100a) library for the fully quantized forward pass of a sinusoidal INR (DHQ).
+
+The work is done by hand-written CUDA kernels behind the C ABI of `include/dhq.h`; this package
+is the thin Python binding over that shared library.  There is no CPU or PyTorch fallback: if the
+library has not been built (`python -m paper_2508_13478_b200.build`), importing the binding's
+functions raises.
+"""
+from .binding import (  # noqa: F401
+    DHQ_GRAN_TENSOR, DHQ_GRAN_CHANNEL_OR_TOKEN, DHQ_ROT_INPUT, DhqError, PIPES,
+    dhq_prepare, dhq_calibrate, dhq_forward, dhq_forward_host, dhq_forward_debug, dhq_get_layer,
+    dhq_layer_dims, dhq_last_status, dhq_launch_count, dhq_destroy, dhq_status_string,
+    dhq_measure_pipe, library_path, load_library,
+)

@@ -1,0 +1,318 @@
+// C ABI of the library (see include/dhq.h): argument checks, the handle, and the sequencing of
+// kernels on the caller's stream.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include "dhq_internal.cuh"
+
+using namespace dhq;
+
+#define CK(call)                                         \
+    do {                                                 \
+        cudaError_t e_ = (call);                         \
+        if (e_ != cudaSuccess) return DHQ_ERR_CUDA;      \
+    } while (0)
+
+namespace {
+
+template <typename T> bool dev_alloc(T **p, size_t count)
+{
+    return cudaMalloc((void **)p, count * sizeof(T) < 16 ? 16 : count * sizeof(T)) == cudaSuccess;
+}
+
+void free_layer(LayerDev &d)
+{
+    cudaFree(d.w_rot); cudaFree(d.row_absmax); cudaFree(d.qw); cudaFree(d.qw_k4m); cudaFree(d.qw_umma);
+    cudaFree(d.s_w); cudaFree(d.inv_w); cudaFree(d.bias); cudaFree(d.cA); cudaFree(d.cA_lo); cudaFree(d.cB);
+    cudaFree(d.act);
+    d = LayerDev();
+}
+
+bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+dhq_status_t ensure_scratch(dhq_handle_s *h, int64_t tokens)
+{
+    if (tokens <= h->scratch_tokens) return DHQ_OK;
+    CK(cudaDeviceSynchronize());
+    cudaFree(h->scratch[0]); cudaFree(h->scratch[1]);
+    h->scratch[0] = h->scratch[1] = nullptr;
+    h->scratch_tokens = 0;
+    for (int i = 0; i < 2; ++i)
+        if (!dev_alloc(&h->scratch[i], (size_t)tokens * h->w)) return DHQ_ERR_ALLOC;
+    h->scratch_tokens = tokens;
+    return DHQ_OK;
+}
+
+// Arguments of layer l (1-based) over tokens [t0, t0+cnt) with the given input/output buffers.
+LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X, int64_t cnt)
+{
+    const LayerDev &d = h->layer[l - 1];
+    LayerArgs a;
+    memset(&a, 0, sizeof(a));
+    a.X = X; a.coords = coords; a.n = cnt;
+    a.K = d.K; a.M = d.M; a.d_L = h->d_L;
+    a.a_bits = h->cfg.a_bits;
+    a.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
+    a.epi_mode = d.epi_mode;
+    a.qw_k4m = d.qw_k4m; a.cA = d.cA; a.cA_lo = d.cA_lo; a.cB = d.cB; a.act = d.act;
+    return a;
+}
+
+dhq_status_t calibrate_impl(dhq_handle_s *h, const float *coords, int64_t n, cudaStream_t st)
+{
+    const int64_t chunk = n < kDebugChunk ? n : kDebugChunk;
+    dhq_status_t s = ensure_scratch(h, chunk);
+    if (s != DHQ_OK) return s;
+    for (int l = 1; l <= h->L; ++l) {
+        LayerDev &d = h->layer[l - 1];
+        CK(cudaMemsetAsync(d.act, 0, 4 * sizeof(float), st));
+        for (int64_t t0 = 0; t0 < n; t0 += chunk) {
+            int64_t cnt = n - t0 < chunk ? n - t0 : chunk;
+            const float *X = nullptr;
+            for (int j = 1; j <= l; ++j) {
+                LayerArgs a = layer_args(h, j, coords + t0 * 2, X, cnt);
+                if (j == l) a.calib_only = 1;
+                else a.Y = h->scratch[(j - 1) & 1];
+                CK(launch_layer(a, st));
+                h->launches++;
+                X = a.Y;
+            }
+        }
+        CK(launch_finalize(d, h->cfg.a_bits, 0, l < h->L, (double)h->cfg.omega0, st, &h->launches));
+    }
+    h->calibrated = true;
+    return DHQ_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+const char *dhq_status_string(dhq_status_t s)
+{
+    switch (s) {
+    case DHQ_OK: return "ok";
+    case DHQ_ERR_INVALID_ARG: return "invalid argument";
+    case DHQ_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case DHQ_ERR_ALLOC: return "allocation failed";
+    case DHQ_ERR_CUDA: return "CUDA runtime error";
+    case DHQ_ERR_NOT_CALIBRATED: return "per-tensor activation scales are not calibrated";
+    case DHQ_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    }
+    return "unknown status";
+}
+
+void dhq_destroy(dhq_handle_t h)
+{
+    if (!h) return;
+    cudaDeviceSynchronize();
+    fused_destroy(h);
+    for (int l = 0; l < kMaxLayers; ++l) free_layer(h->layer[l]);
+    cudaFree(h->d_status);
+    cudaFree(h->scratch[0]); cudaFree(h->scratch[1]);
+    cudaFree(h->stage_in); cudaFree(h->stage_out);
+    delete h;
+}
+
+dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const float *const *b,
+                         void *stream, dhq_handle_t *out)
+{
+    if (!cfg || !W || !b || !out || !cfg->dims) return DHQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    const int L = cfg->n_layers;
+    if (L < 2 || L > kMaxLayers) return DHQ_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l)
+        if (!W[l] || !b[l]) return DHQ_ERR_INVALID_ARG;
+    const int w = cfg->dims[1], d_L = cfg->dims[L];
+    if (cfg->dims[0] != 2 || !is_pow2(w) || w < 64 || w > 512 || d_L < 1 || d_L > 4) return DHQ_ERR_UNSUPPORTED;
+    for (int l = 1; l < L; ++l)
+        if (cfg->dims[l] != w) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits < 2 || cfg->a_bits > 8) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->rotation != DHQ_ROT_INPUT) return DHQ_ERR_UNSUPPORTED;
+    if ((cfg->w_gran != DHQ_GRAN_TENSOR && cfg->w_gran != DHQ_GRAN_CHANNEL_OR_TOKEN) ||
+        (cfg->a_gran != DHQ_GRAN_TENSOR && cfg->a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN))
+        return DHQ_ERR_INVALID_ARG;
+    if (!(cfg->omega0 == cfg->omega0) || std::isinf(cfg->omega0)) return DHQ_ERR_INVALID_ARG;
+
+    dhq_handle_s *h = new (std::nothrow) dhq_handle_s();
+    if (!h) return DHQ_ERR_ALLOC;
+    h->cfg = *cfg;
+    for (int i = 0; i <= L; ++i) h->dims[i] = cfg->dims[i];
+    h->cfg.dims = h->dims;
+    h->L = L; h->w = w; h->d_L = d_L;
+    cudaStream_t st = (cudaStream_t)stream;
+    dhq_status_t rc = DHQ_OK;
+    float *d_bounds = nullptr;
+    const bool per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
+    do {
+        if (cudaGetDevice(&h->device) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+        if (!dev_alloc(&h->d_status, 4) || !dev_alloc(&d_bounds, kMaxLayers)) { rc = DHQ_ERR_ALLOC; break; }
+        if (cudaMemsetAsync(h->d_status, 0, 16, st) != cudaSuccess ||
+            cudaMemsetAsync(d_bounds, 0, kMaxLayers * sizeof(float), st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+        for (int l = 1; l <= L && rc == DHQ_OK; ++l) {
+            LayerDev &d = h->layer[l - 1];
+            d.K = (l == 1) ? 4 : w;
+            d.M = (l == L) ? 4 : w;
+            d.Mt = d.M < 16 ? 16 : d.M;
+            d.slab_rows = fused_slab_rows(d.K, d.Mt);
+            d.d_in = cfg->dims[l - 1];
+            d.d_out = cfg->dims[l];
+            const size_t MK = (size_t)d.M * d.K;
+            bool ok = dev_alloc(&d.w_rot, MK) && dev_alloc(&d.row_absmax, d.M) && dev_alloc(&d.qw, MK) &&
+                      dev_alloc(&d.qw_k4m, MK / 4) && dev_alloc(&d.qw_umma, (size_t)d.Mt * (d.K < 16 ? 16 : d.K)) &&
+                      dev_alloc(&d.s_w, d.M) && dev_alloc(&d.inv_w, d.M) && dev_alloc(&d.bias, d.M) &&
+                      dev_alloc(&d.cA, d.M) && dev_alloc(&d.cA_lo, d.M) && dev_alloc(&d.cB, d.M) &&
+                      dev_alloc(&d.act, 4);
+            if (!ok) { rc = DHQ_ERR_ALLOC; break; }
+            if (cudaMemsetAsync(d.act, 0, 16, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+            PrepArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = W[l - 1]; a.b = b[l - 1];
+            a.d_out = d.d_out; a.d_in = d.d_in; a.K = d.K; a.M = d.M; a.Mt = d.Mt;
+            a.bits = cfg->w_bits;
+            a.per_channel = cfg->w_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
+            a.sine = l < L; a.first = l == 1;
+            a.omega0 = (double)cfg->omega0;
+            a.dev = d;
+            a.phase_bound = d_bounds + (l - 1);
+            if (launch_prepare(a, st, &h->launches) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+            if (per_token &&
+                launch_finalize(d, cfg->a_bits, 1, l < L, (double)cfg->omega0, st, &h->launches) != cudaSuccess) {
+                rc = DHQ_ERR_CUDA; break;
+            }
+        }
+        if (rc != DHQ_OK) break;
+        float bounds[kMaxLayers];
+        if (cudaMemcpyAsync(bounds, d_bounds, sizeof(bounds), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+        for (int l = 1; l <= L; ++l) {
+            LayerDev &d = h->layer[l - 1];
+            d.phase_bound = bounds[l - 1];
+            if (l == L) d.epi_mode = EPI_LINEAR;
+            else if (l == 1) d.epi_mode = EPI_SINE_WIDE;   // coordinates are not bounded by the weights
+            else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit) ? EPI_SINE_FAST : EPI_SINE_WIDE;
+        }
+        h->calibrated = per_token;
+        rc = fused_create(h);
+    } while (0);
+    cudaFree(d_bounds);
+    if (rc != DHQ_OK) {
+        dhq_destroy(h);
+        return rc;
+    }
+    *out = h;
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void *stream)
+{
+    if (!h || !coords || n < 1) return DHQ_ERR_INVALID_ARG;
+    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
+    return calibrate_impl(h, coords, n, (cudaStream_t)stream);
+}
+
+dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int64_t n, float *out,
+                               const dhq_debug_bufs_t *bufs, void *stream)
+{
+    if (!h || n < 0 || (n > 0 && !coords)) return DHQ_ERR_INVALID_ARG;
+    if (n == 0) return DHQ_OK;
+    if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t chunk = n < kDebugChunk ? n : kDebugChunk;
+    dhq_status_t s = ensure_scratch(h, chunk);
+    if (s != DHQ_OK) return s;
+    for (int64_t t0 = 0; t0 < n; t0 += chunk) {
+        int64_t cnt = n - t0 < chunk ? n - t0 : chunk;
+        const float *X = nullptr;
+        for (int l = 1; l <= h->L; ++l) {
+            const LayerDev &d = h->layer[l - 1];
+            LayerArgs a = layer_args(h, l, coords + t0 * 2, X, cnt);
+            a.Y = h->scratch[(l - 1) & 1];
+            if (l == h->L) a.out = out ? out + t0 * h->d_L : nullptr;
+            if (bufs) {
+                if (bufs->X && bufs->X[l - 1]) a.dX = bufs->X[l - 1] + t0 * d.K;
+                if (bufs->codes && bufs->codes[l - 1]) a.dcodes = bufs->codes[l - 1] + t0 * d.K;
+                if (bufs->s_x && bufs->s_x[l - 1]) a.ds_x = bufs->s_x[l - 1] + t0;
+                if (bufs->acc && bufs->acc[l - 1]) a.dacc = bufs->acc[l - 1] + t0 * d.M;
+                if (bufs->Y && bufs->Y[l - 1]) a.Y = bufs->Y[l - 1] + t0 * d.M;
+            }
+            CK(launch_layer(a, st));
+            h->launches++;
+            X = a.Y;
+        }
+    }
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *out, void *stream)
+{
+    if (!h || n < 0 || (n > 0 && (!coords || !out))) return DHQ_ERR_INVALID_ARG;
+    if (n == 0) return DHQ_OK;
+    if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!h->calibrated) {
+        dhq_status_t s = calibrate_impl(h, coords, n, st);
+        if (s != DHQ_OK) return s;
+    }
+    return fused_forward(h, coords, n, out, st);
+}
+
+dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t n, float *out_host,
+                              void *stream)
+{
+    if (!h || n < 0 || (n > 0 && (!coords_host || !out_host))) return DHQ_ERR_INVALID_ARG;
+    if (n == 0) return DHQ_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n > h->stage_tokens) {
+        CK(cudaDeviceSynchronize());
+        cudaFree(h->stage_in); cudaFree(h->stage_out);
+        h->stage_in = h->stage_out = nullptr;
+        h->stage_tokens = 0;
+        if (!dev_alloc(&h->stage_in, (size_t)n * 2) || !dev_alloc(&h->stage_out, (size_t)n * h->d_L))
+            return DHQ_ERR_ALLOC;
+        h->stage_tokens = n;
+    }
+    CK(cudaMemcpyAsync(h->stage_in, coords_host, (size_t)n * 2 * sizeof(float), cudaMemcpyHostToDevice, st));
+    dhq_status_t s = dhq_forward(h, h->stage_in, n, h->stage_out, stream);
+    if (s != DHQ_OK) return s;
+    CK(cudaMemcpyAsync(out_host, h->stage_out, (size_t)n * h->d_L * sizeof(float), cudaMemcpyDeviceToHost, st));
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_layer_dims(dhq_handle_t h, int layer, int *K, int *M)
+{
+    if (!h || layer < 1 || layer > h->L) return DHQ_ERR_INVALID_ARG;
+    if (K) *K = h->layer[layer - 1].K;
+    if (M) *M = h->layer[layer - 1].M;
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_get_layer(dhq_handle_t h, int layer, int8_t *codes, float *w_scales, float *act_absmax)
+{
+    if (!h || layer < 1 || layer > h->L) return DHQ_ERR_INVALID_ARG;
+    const LayerDev &d = h->layer[layer - 1];
+    CK(cudaDeviceSynchronize());
+    if (codes) CK(cudaMemcpy(codes, d.qw, (size_t)d.M * d.K, cudaMemcpyDeviceToHost));
+    if (w_scales) CK(cudaMemcpy(w_scales, d.s_w, (size_t)d.M * sizeof(float), cudaMemcpyDeviceToHost));
+    if (act_absmax) {
+        *act_absmax = NAN;
+        if (h->cfg.a_gran == DHQ_GRAN_TENSOR && h->calibrated)
+            CK(cudaMemcpy(act_absmax, d.act, sizeof(float), cudaMemcpyDeviceToHost));
+    }
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_last_status(dhq_handle_t h)
+{
+    if (!h) return DHQ_ERR_INVALID_ARG;
+    int v = 0;
+    CK(cudaDeviceSynchronize());
+    CK(cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+    CK(cudaMemset(h->d_status, 0, sizeof(int)));
+    return v == 0 ? DHQ_OK : DHQ_ERR_TIMEOUT;
+}
+
+int64_t dhq_launch_count(dhq_handle_t h) { return h ? h->launches : 0; }
+
+} // extern "C"

@@ -1,0 +1,110 @@
+// Host-side handle and the argument blocks passed to kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "../../include/dhq.h"
+#include "dhq_math.cuh"
+
+namespace dhq {
+
+constexpr int kMaxLayers = 16;
+constexpr int kDebugChunk = 65536; // tokens per pass of the layer-by-layer path
+
+// Device arrays of one prepared layer.
+struct LayerDev {
+    int K = 0, M = 0;          // padded sizes as the definition pads them (K = 4 | w, M = w | 4)
+    int Mt = 0;                // rows of the tensor-core weight tile (M rounded up to 16)
+    int slab_rows = 0;         // rows per contiguous slab of the tensor-core image
+    int d_in = 0, d_out = 0;
+    int epi_mode = EPI_LINEAR;
+    float phase_bound = 0.f;   // omega0 * max_m (sum_k |W_mk| + |b_m|), hidden layers
+    float *w_rot = nullptr;    // [M][K] fp32 rotated weights (kept for inspection)
+    float *row_absmax = nullptr; // [M]
+    int8_t *qw = nullptr;      // [M][K] codes, row-major
+    uint32_t *qw_k4m = nullptr; // [K/4][M] four consecutive-k codes per word (layer-by-layer path)
+    uint8_t *qw_umma = nullptr; // [Mt][K] codes in the tensor-core shared-memory image
+    float *s_w = nullptr;      // [M]
+    float *inv_w = nullptr;    // [M]
+    float *bias = nullptr;     // [M] zero padded
+    float *cA = nullptr, *cA_lo = nullptr, *cB = nullptr; // [M] epilogue constants
+    float *act = nullptr;      // [4]: frozen absmax (max taken on the bit pattern), s_x, inv, unused
+};
+
+} // namespace dhq
+
+struct dhq_handle_s {
+    dhq_config_t cfg;
+    int dims[dhq::kMaxLayers + 1];
+    int L = 0, w = 0, d_L = 0;
+    int device = 0;
+    bool calibrated = false;
+    dhq::LayerDev layer[dhq::kMaxLayers];
+    int *d_status = nullptr;        // device status word
+    float *scratch[2] = {nullptr, nullptr}; // ping-pong activations of the layer-by-layer path
+    int64_t scratch_tokens = 0;
+    float *stage_in = nullptr, *stage_out = nullptr; // dhq_forward_host staging
+    int64_t stage_tokens = 0;
+    int64_t launches = 0;
+    void *fused = nullptr;          // state of the fused path (device parameter block)
+};
+
+namespace dhq {
+
+// Arguments of one pass of the layer-by-layer kernel.
+struct LayerArgs {
+    const float *X;        // [n][K] layer input, or NULL for layer 1 (built from coords)
+    const float *coords;   // [n][2], layer 1 only
+    int64_t n;
+    int K, M, d_L;
+    int a_bits;
+    int per_token;
+    int epi_mode;
+    int calib_only;        // 1: only take max |rotated input| into act[0] (bit pattern max)
+    const uint32_t *qw_k4m;
+    const float *cA, *cA_lo, *cB;
+    float *act;            // frozen absmax / s_x / inv (per-tensor mode)
+    float *Y;              // [n][M] or NULL
+    float *out;            // [n][d_L] or NULL (last layer)
+    float *dX; int8_t *dcodes; float *ds_x; int32_t *dacc; // dumps, may be NULL
+};
+
+cudaError_t launch_layer(const LayerArgs &a, cudaStream_t st);
+
+struct PrepArgs {
+    const float *W, *b;
+    int d_out, d_in, K, M, Mt;
+    int bits, per_channel;
+    int sine;              // hidden or first layer
+    int first;             // layer 1: no phase bound from the weights (coordinates are unbounded)
+    double omega0;
+    LayerDev dev;
+    float *phase_bound;    // device scalar
+};
+cudaError_t launch_prepare(const PrepArgs &a, cudaStream_t st, int64_t *launches);
+// Epilogue constants from s_w and (per-tensor) the frozen activation scale.
+cudaError_t launch_finalize(const LayerDev &dev, int a_bits, int per_token, int sine, double omega0,
+                            cudaStream_t st, int64_t *launches);
+
+// Byte offset of code (n, k) in the tensor-core shared-memory image of a weight matrix with K
+// codes per row: contiguous slabs of `slab_rows` rows; inside a slab the 16-byte k-groups are
+// the outer index and rows the inner one, i.e. 8-row x 16-byte core matrices stacked along rows
+// (128 bytes apart) and along k (slab_rows * 16 bytes apart) - the K-major, unswizzled operand
+// layout of tcgen05.mma.
+__host__ __device__ inline size_t umma_offset(int n, int k, int K, int slab_rows)
+{
+    return (size_t)(n / slab_rows) * slab_rows * K + (size_t)(k >> 4) * slab_rows * 16 +
+           (size_t)(n % slab_rows) * 16 + (k & 15);
+}
+// Rows per slab for a layer with K inputs and Mt (padded) outputs: slabs hold at most 64 KB.
+inline int fused_slab_rows(int K, int Mt)
+{
+    int rows = 65536 / (K < 16 ? 16 : K);
+    return rows < Mt ? rows : Mt;
+}
+
+// Fused tensor-core forward.
+dhq_status_t fused_create(dhq_handle_s *h);
+void fused_destroy(dhq_handle_s *h);
+dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st);
+
+} // namespace dhq

@@ -1,0 +1,86 @@
+// Per-element arithmetic shared by every kernel of the library, so that the layer-by-layer
+// path and the fused path execute the same fp32 operations in the same order and agree bit
+// for bit.  Every fp32 step uses an explicit round-to-nearest intrinsic: nothing here may be
+// contracted, reassociated or replaced by a fast-math variant.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dhq {
+
+// Epilogue variants, chosen per layer when the network is prepared.
+enum EpiMode : int {
+    EPI_LINEAR = 0,    // last layer: z = c * acc + b
+    EPI_SINE_FAST = 1, // hidden layer whose phase is provably small: sin.approx(fma(acc, c, B))
+    EPI_SINE_WIDE = 2  // first layer / large phases: compensated phase and explicit 2*pi reduction
+};
+
+// Largest |omega0 z| for which EPI_SINE_FAST keeps the result within 1e-5 of an exact sine:
+// fma rounding (ulp(32)/2 = 1.9e-6) + constant rounding (32 * 2^-24 = 1.9e-6) + the multiply by
+// 1/(2 pi) inside sin.approx (1.5e-6) + the approximation itself (about 7e-7).
+constexpr float kFastPhaseLimit = 32.0f;
+
+__device__ __forceinline__ float qmax_of(int bits) { return (float)((1 << (bits - 1)) - 1); }
+
+// Symmetric absmax scales: s = a / qmax, inv = qmax / a, both IEEE divisions; a = 0 -> 0, 0.
+__device__ __forceinline__ void scales_of(float a, float qmaxf, float &s, float &inv)
+{
+    if (a > 0.0f) {
+        s = __fdiv_rn(a, qmaxf);
+        inv = __fdiv_rn(qmaxf, a);
+    } else {
+        s = 0.0f;
+        inv = 0.0f;
+    }
+}
+
+// q = clamp(round_half_even(fl32(v * inv)), -qmax, +qmax).  Clamping before rounding gives the
+// same integer because qmax is one.  NaN inputs come out as +-qmax (fminf/fmaxf drop the NaN).
+__device__ __forceinline__ int quantize(float v, float inv, float qmaxf)
+{
+    float t = __fmul_rn(v, inv);
+    t = fmaxf(fminf(t, qmaxf), -qmaxf);
+    return __float2int_rn(t);
+}
+
+__device__ __forceinline__ float sin_approx(float x)
+{
+    float y;
+    asm("sin.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// sin(x) for |x| up to a few thousand: k = nearest integer to x / (2 pi), r = x - k * 2 pi with
+// 2 pi split into fl32(2 pi) and the remainder (two fused multiply-adds, each exact before its
+// single rounding), then the hardware approximation on |r| <= pi.
+__device__ __forceinline__ float sin_wide(float x)
+{
+    const float inv_two_pi = 0.15915494309189535f;
+    const float two_pi_hi = 6.2831854820251465f;   // fl32(2 pi)
+    const float two_pi_lo = -1.7484555e-07f;       // 2 pi - fl32(2 pi)
+    float k = rintf(__fmul_rn(x, inv_two_pi));
+    float r = __fmaf_rn(k, -two_pi_hi, x);
+    r = __fmaf_rn(k, -two_pi_lo, r);
+    return sin_approx(r);
+}
+
+// Per-(token, channel) epilogue.  accf = (float)acc is exact (|acc| < 2^24).
+//   c_hi, c_lo : the dequantization constant omega0 * s_w * s_x (or s_w * s_x for the last
+//                layer) as an fp32 value and its remainder; c_lo is only read by EPI_SINE_WIDE.
+//   cb         : omega0 * b (or b for the last layer).
+__device__ __forceinline__ float epilogue(int mode, float accf, float c_hi, float c_lo, float cb)
+{
+    if (mode == EPI_SINE_FAST) return sin_approx(__fmaf_rn(accf, c_hi, cb));
+    if (mode == EPI_SINE_WIDE) return sin_wide(__fmaf_rn(accf, c_lo, __fmaf_rn(accf, c_hi, cb)));
+    return __fmaf_rn(accf, c_hi, cb);
+}
+
+// Per-token activation scales: the per-channel constant cA (+ remainder cA_lo) times the
+// token's s_x.  c_lo collects the rounding error of that product and the remainder term.
+__device__ __forceinline__ void token_const(float cA, float cA_lo, float s_x, float &c_hi, float &c_lo)
+{
+    c_hi = __fmul_rn(cA, s_x);
+    c_lo = __fmaf_rn(cA_lo, s_x, __fmaf_rn(cA, s_x, -c_hi));
+}
+
+} // namespace dhq

@@ -1,0 +1,143 @@
+// Weight side of DHQ (Eq. 4-5 of the paper, the factor acting on the input dimension, and the
+// quantizer of Section III-B), run once per network on the device:
+//   pad -> rotate each row by H_K (fp32 butterfly, strides 1, 2, ..., K/2) -> scale by 1/K
+//   -> absmax per tensor or per row -> quantize -> write the codes in three layouts.
+#include "dhq_internal.cuh"
+
+namespace dhq {
+
+// One block per padded output row; K/2 threads, one butterfly pair each per stage.
+__global__ void prep_rotate_kernel(PrepArgs a)
+{
+    extern __shared__ float row[];
+    const int m = blockIdx.x, K = a.K;
+    for (int k = threadIdx.x; k < K; k += blockDim.x)
+        row[k] = (m < a.d_out && k < a.d_in) ? a.W[(size_t)m * a.d_in + k] : 0.0f;
+    // phase bound of this row: sum_k |W_mk| + |b_m| (inputs of hidden layers lie in [-1, 1])
+    __shared__ float red[32];
+    float part = 0.f;
+    __syncthreads();
+    for (int k = threadIdx.x; k < K; k += blockDim.x) part += fabsf(row[k]);
+    for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = part;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int i = 0; i < (blockDim.x + 31) / 32; ++i) s += red[i];
+        float bm = (m < a.d_out) ? fabsf(a.b[m]) : 0.f;
+        float bound = (float)a.omega0 * (s + bm) * 1.0001f;
+        atomicMax((unsigned int *)a.phase_bound, __float_as_uint(bound));
+        a.dev.bias[m] = (m < a.d_out) ? a.b[m] : 0.0f;
+    }
+    for (int h = 1; h < K; h <<= 1) {
+        __syncthreads();
+        for (int p = threadIdx.x; p < K / 2; p += blockDim.x) {
+            int i = ((p & ~(h - 1)) << 1) | (p & (h - 1));
+            float x = row[i], y = row[i + h];
+            row[i] = __fadd_rn(x, y);
+            row[i + h] = __fsub_rn(x, y);
+        }
+    }
+    __syncthreads();
+    const float invK = 1.0f / (float)K; // power of two: exact
+    float amax = 0.f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        float v = __fmul_rn(row[k], invK);
+        a.dev.w_rot[(size_t)m * K + k] = v;
+        amax = fmaxf(amax, fabsf(v));
+    }
+    for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float r = 0.f;
+        for (int i = 0; i < (blockDim.x + 31) / 32; ++i) r = fmaxf(r, red[i]);
+        a.dev.row_absmax[m] = r;
+    }
+}
+
+// One block: per-tensor or per-row scales.
+__global__ void prep_scales_kernel(PrepArgs a)
+{
+    __shared__ float tensor_max;
+    if (threadIdx.x == 0) {
+        float r = 0.f;
+        for (int m = 0; m < a.M; ++m) r = fmaxf(r, a.dev.row_absmax[m]);
+        tensor_max = r;
+    }
+    __syncthreads();
+    const float qmaxf = qmax_of(a.bits);
+    for (int m = threadIdx.x; m < a.M; m += blockDim.x) {
+        float s, inv;
+        scales_of(a.per_channel ? a.dev.row_absmax[m] : tensor_max, qmaxf, s, inv);
+        a.dev.s_w[m] = s;
+        a.dev.inv_w[m] = inv;
+    }
+}
+
+__global__ void prep_quant_kernel(PrepArgs a)
+{
+    const int K = a.K, M = a.M, Mt = a.Mt;
+    const float qmaxf = qmax_of(a.bits);
+    const int total = Mt * K;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        int m = idx / K, k = idx % K;
+        int q = 0;
+        if (m < M) q = quantize(a.dev.w_rot[(size_t)m * K + k], a.dev.inv_w[m], qmaxf);
+        if (m < M) {
+            a.dev.qw[(size_t)m * K + k] = (int8_t)q;
+            ((int8_t *)a.dev.qw_k4m)[((size_t)(k >> 2) * M + m) * 4 + (k & 3)] = (int8_t)q;
+        }
+        a.dev.qw_umma[umma_offset(m, k, K, a.dev.slab_rows)] = (uint8_t)(int8_t)q;
+    }
+}
+
+// Epilogue constants in fp64, rounded once: cA = fl32(A), cA_lo = fl32(A - cA) with
+// A = f * s_w[m] (* s_x when the activation scale is per tensor), cB = fl32(f * b[m]),
+// f = omega0 for sine layers and 1 for the last layer.  Also derives s_x and inv from the frozen
+// absmax in per-tensor mode.
+__global__ void finalize_kernel(LayerDev dev, int a_bits, int per_token, int sine, double omega0)
+{
+    __shared__ float s_x_sh;
+    if (threadIdx.x == 0) {
+        float s = 1.0f;
+        if (!per_token) {
+            float inv;
+            scales_of(dev.act[0], qmax_of(a_bits), s, inv);
+            dev.act[1] = s;
+            dev.act[2] = inv;
+        }
+        s_x_sh = s;
+    }
+    __syncthreads();
+    const double f = sine ? omega0 : 1.0;
+    for (int m = threadIdx.x; m < dev.M; m += blockDim.x) {
+        double A = f * (double)dev.s_w[m] * (per_token ? 1.0 : (double)s_x_sh);
+        float hi = (float)A;
+        dev.cA[m] = hi;
+        dev.cA_lo[m] = (float)(A - (double)hi);
+        dev.cB[m] = (float)(f * (double)dev.bias[m]);
+    }
+}
+
+cudaError_t launch_prepare(const PrepArgs &a, cudaStream_t st, int64_t *launches)
+{
+    int threads = a.K / 2 < 32 ? 32 : a.K / 2;
+    prep_rotate_kernel<<<a.M, threads, a.K * sizeof(float), st>>>(a);
+    prep_scales_kernel<<<1, 256, 0, st>>>(a);
+    int total = a.Mt * a.K;
+    prep_quant_kernel<<<(total + 255) / 256, 256, 0, st>>>(a);
+    *launches += 3;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finalize(const LayerDev &dev, int a_bits, int per_token, int sine, double omega0,
+                            cudaStream_t st, int64_t *launches)
+{
+    finalize_kernel<<<1, 256, 0, st>>>(dev, a_bits, per_token, sine, omega0);
+    *launches += 1;
+    return cudaGetLastError();
+}
+
+} // namespace dhq

@@ -1,0 +1,216 @@
+"""GPU parity: the CUDA library through its C ABI against the CPU oracle.
+
+Integer stages (weight codes, activation codes, int32 accumulators) and scales must match bit
+for bit; fp32 layer outputs within 1e-5 absolute of the oracle's fp64 epilogue.  Parity is taken
+layer by layer on the library's own layer inputs (teacher forcing), because a sine evaluated in
+fp32 cannot be bit-identical to an fp64 one and one flipped code downstream would otherwise
+hide everything after it; the dump chain is checked to close, and the fused kernel's output
+must equal the layer-by-layer path bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+import dhq_inputs
+from tests.gpu_util import TOL_Y, check_layers_against_oracle, check_weights, prepare_pair, run_debug, to_dev
+
+pytestmark = pytest.mark.gpu
+
+dhq = pytest.importorskip("paper_2508_13478_b200")
+from oracle import dhq_oracle as orc  # noqa: E402
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2508_13478_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _p1(workload, coords_np, fused=True):
+    weights, biases = workload.network()
+    h, net = prepare_pair(workload.dims, weights, biases, workload.omega0, workload.w_bits,
+                          workload.a_bits, workload.w_gran, workload.a_gran)
+    try:
+        check_weights(h, net)
+        cd = to_dev(coords_np)
+        if workload.a_gran == 0:
+            dhq.dhq_calibrate(h, cd)
+        out_dbg, bufs = run_debug(h, net, cd)
+        worst = check_layers_against_oracle(h, net, coords_np, out_dbg, bufs)
+        if fused:
+            out = torch.full((coords_np.shape[0], workload.dims[-1]), float("nan"), device="cuda")
+            dhq.dhq_forward(h, cd, out)
+            torch.cuda.synchronize()
+            assert dhq.dhq_last_status(h) == 0
+            assert torch.equal(out.view(torch.int32), out_dbg.view(torch.int32)), "fused != layer-by-layer"
+        return worst
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_layer_by_layer_path_alone_c1_and_per_token():
+    w = dhq_inputs.WORKLOADS["C1"]
+    _p1(w, w.coords(), fused=False)
+    w3 = dhq_inputs.WORKLOADS["C3"]
+    _p1(w3, w3.coords()[:3000], fused=False)
+
+
+def test_c1_full_grid():
+    w = dhq_inputs.WORKLOADS["C1"]
+    _p1(w, w.coords())
+
+
+def test_c2_full_grid():
+    w = dhq_inputs.WORKLOADS["C2"]
+    _p1(w, w.coords())
+
+
+@pytest.mark.parametrize("name,count", [("C3", 20000 + 77), ("C4-W4A4", 12000 + 1), ("C4-W6A6", 12000 + 1)])
+def test_c3_c4_sampled_tokens(name, count):
+    w = dhq_inputs.WORKLOADS[name]
+    coords = w.coords()
+    idx = np.linspace(0, coords.shape[0] - 1, count).astype(np.int64)
+    _p1(w, np.ascontiguousarray(coords[idx]))
+
+
+@pytest.mark.parametrize("n", [1, 127, 128, 129, 255, 257, 1000])
+def test_ragged_tails_small_width(n):
+    w = dhq_inputs.WORKLOADS["C1"]
+    _p1(w, w.coords()[:n])
+
+
+@pytest.mark.parametrize("w_gran,a_gran", [(0, 0), (0, 1), (1, 0), (1, 1)])
+@pytest.mark.parametrize("bits", [4, 8])
+def test_granularity_and_bit_width_combinations(w_gran, a_gran, bits):
+    wl = dhq_inputs.Workload("combo", (2, 128, 128, 128, 3), 30.0, 40 + bits, bits, bits, w_gran, a_gran, (40, 41))
+    _p1(wl, wl.coords())
+
+
+def test_trained_like_weights_and_wide_phases():
+    # bell-shaped hidden weights, two-peaked last layer (Section III-A), and a first layer scaled up
+    # so that phases reach hundreds of radians
+    dims = (2, 256, 256, 256, 3)
+    weights, biases = dhq_inputs.trained_like_init(dims, 30.0, 12)
+    weights[0] = (weights[0] * 4).astype(np.float32)
+    weights[1] = (weights[1] * 6).astype(np.float32)
+    coords = dhq_inputs.grid_coords(50, 50)
+    h, net = prepare_pair(dims, weights, biases, 30.0, 8, 8, 1, 1)
+    try:
+        check_weights(h, net)
+        out_dbg, bufs = run_debug(h, net, to_dev(coords))
+        check_layers_against_oracle(h, net, coords, out_dbg, bufs)
+        out = torch.empty_like(out_dbg)
+        dhq.dhq_forward(h, to_dev(coords), out)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int32), out_dbg.view(torch.int32))
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_zero_token_and_empty_batch():
+    w = dhq_inputs.WORKLOADS["C3"]
+    coords = np.zeros((130, 2), np.float32)
+    coords[1:] = w.coords()[:129]
+    _p1(w, coords)
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 1, 1)
+    try:
+        out = torch.zeros((0, 3), device="cuda")
+        dhq.dhq_forward(h, torch.zeros((0, 2), device="cuda"), out)   # n = 0: no-op
+        assert dhq.dhq_last_status(h) == 0
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_unsupported_and_invalid_arguments():
+    w = dhq_inputs.WORKLOADS["C1"]
+    weights, biases = w.network()
+    W = [to_dev(x) for x in weights]
+    B = [to_dev(x) for x in biases]
+    with pytest.raises(dhq.DhqError) as e:
+        dhq.dhq_prepare((2, 64, 64, 64, 1), W, B, w_bits=9)
+    assert e.value.code == 2
+    with pytest.raises(dhq.DhqError) as e:
+        dhq.dhq_prepare((3, 64, 64, 64, 1), W, B)
+    assert e.value.code == 2
+    with pytest.raises(dhq.DhqError) as e:
+        dhq.dhq_prepare((2, 64, 64, 64, 1), W, B, rotation=1)
+    assert e.value.code == 2
+    h = dhq.dhq_prepare(w.dims, W, B)
+    try:
+        with pytest.raises(dhq.DhqError) as e:     # per-tensor scales not frozen yet
+            dhq.dhq_forward_debug(h, to_dev(w.coords()[:8]))
+        assert e.value.code == 5
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_forward_auto_calibrates_and_is_deterministic_and_batch_independent():
+    w = dhq_inputs.WORKLOADS["C1"]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 0, 0)
+    try:
+        cd = to_dev(w.coords())
+        out1 = torch.empty((w.n, 1), device="cuda")
+        dhq.dhq_forward(h, cd, out1)                      # freezes the scales on this grid
+        out2 = torch.empty_like(out1)
+        dhq.dhq_forward(h, cd, out2)
+        sub = torch.empty((300, 1), device="cuda")
+        dhq.dhq_forward(h, cd[1000:1300].contiguous(), sub)
+        torch.cuda.synchronize()
+        assert torch.equal(out1.view(torch.int32), out2.view(torch.int32))
+        assert torch.equal(sub.view(torch.int32), out1[1000:1300].view(torch.int32))
+        # the frozen values are the oracle's own calibration on its own free-running chain, up to
+        # the fp32-vs-fp64 sine: equal to a few ulps
+        frozen = orc.calibrate(net, w.coords())
+        for l in range(1, 5):
+            a = dhq.dhq_get_layer(h, l)[2]
+            assert abs(a - frozen[l - 1]) <= 2e-5 * max(1.0, abs(frozen[l - 1]))
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_free_running_end_to_end_report():
+    # Reported, loosely gated: oracle on its own chain and calibration.  A code flipped at a
+    # near-tie moves one accumulator by one weight code, so a small fraction of coordinates may
+    # differ by more than 1e-5; all stay far below one quantization step of the output.
+    w = dhq_inputs.WORKLOADS["C2"]
+    weights, biases = w.network()
+    coords = w.coords()[:: 16]
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 0, 0)
+    try:
+        out = torch.empty((coords.shape[0], 3), device="cuda")
+        dhq.dhq_forward(h, to_dev(coords), out)
+        torch.cuda.synchronize()
+        orc.calibrate(net, coords)
+        ref = orc.forward(net, coords)
+        d = np.abs(out.cpu().numpy().astype(np.float64) - ref)
+        frac = float((d.max(axis=1) > TOL_Y).mean())
+        print(f"free-running: max |d| = {d.max():.3e}, fraction of coordinates beyond 1e-5 = {frac:.4f}")
+        assert frac < 0.25 and d.max() < 5e-2
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_forward_host_buffers():
+    w = dhq_inputs.WORKLOADS["C1"]
+    weights, biases = w.network()
+    h, _ = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 0, 1)
+    try:
+        ch = torch.from_numpy(w.coords()).pin_memory()
+        oh = torch.empty((w.n, 1)).pin_memory()
+        dhq.dhq_forward_host(h, ch, oh)
+        out = torch.empty((w.n, 1), device="cuda")
+        dhq.dhq_forward(h, ch.cuda(), out)
+        torch.cuda.synchronize()
+        assert torch.equal(oh.view(torch.int32), out.cpu().view(torch.int32))
+        assert dhq.dhq_launch_count(h) > 0
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_pipe_micro_benchmarks_run():
+    for pipe in ("ffma", "mufu_sin", "tensor_i8"):
+        ops, ms = dhq.dhq_measure_pipe(pipe, 200)
+        assert ops > 1e11 and ms > 0
