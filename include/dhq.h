@@ -59,7 +59,8 @@ typedef enum {
     DHQ_ERR_ALLOC = 3,          /* device or host allocation failed                        */
     DHQ_ERR_CUDA = 4,           /* a CUDA runtime call failed                              */
     DHQ_ERR_NOT_CALIBRATED = 5, /* per-tensor activation scales requested but not frozen   */
-    DHQ_ERR_TIMEOUT = 6         /* a bounded wait inside a kernel ran out                  */
+    DHQ_ERR_TIMEOUT = 6,        /* a bounded wait inside a kernel ran out                  */
+    DHQ_ERR_TOO_LARGE = 7       /* more tokens than a fixed-size scratch area can hold     */
 } dhq_status_t;
 
 /* Quantizer granularity: weights per tensor or per output channel; activations per tensor
@@ -168,6 +169,38 @@ DHQ_API dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int6
  */
 DHQ_API dhq_status_t dhq_get_layer(dhq_handle_t h, int layer, int8_t *codes, float *w_scales,
                                    float *act_absmax);
+
+/*
+ * Forward pass for callers that must not allocate device memory.  (The paper has no
+ * counterpart; this is a deployment variant of dhq_forward_debug without the dumps.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a framework that owns
+ * the whole device heap through its own caching allocator, in a process whose memory budget is
+ * fixed at start-up, or in a latency-critical loop where an allocation's implicit device
+ * synchronisation is not acceptable.  The other layer-by-layer entry points grow scratch
+ * buffers with cudaMalloc on demand; this one never does.  It runs the same per-layer kernel,
+ * but the activations that travel between layers live in a fixed array that is part of the
+ * library image itself: 2 x DHQ_STATIC_MAX_TOKENS x 512 floats = 16 MiB, which every GPU that
+ * loads the library carries until the process exits, whether or not this call is ever used.
+ *
+ *   coords  device [n][2] fp32, out device [n][d_L] fp32, as for dhq_forward.
+ *   n       0 .. DHQ_STATIC_MAX_TOKENS; a larger n returns DHQ_ERR_TOO_LARGE and enqueues
+ *           nothing (split the batch and call again once the previous call has finished).
+ * Results equal dhq_forward's bit for bit.  Per-tensor activation scales must already be frozen
+ * (dhq_calibrate, which does allocate, or an earlier dhq_forward): otherwise NOT_CALIBRATED.
+ * The call makes no cudaMalloc/cudaFree and calls no allocating library routine.
+ *
+ * Set-up: the first call on each device looks up the device address of the scratch array
+ * (once per device, with that device current) and keeps it; make that first call before any
+ * stream capture begins.
+ * Sharing: all handles and all calls on a device use the same array, and it keeps whatever the
+ * last call left there.  Nothing in it needs clearing, because each layer pass writes every
+ * value that the next pass reads; but two calls whose kernels overlap on the GPU (different
+ * streams, no ordering between them) race on it and both give wrong results.  Order them.
+ */
+#define DHQ_STATIC_MAX_TOKENS 4096
+DHQ_API dhq_status_t dhq_forward_static_scratch(dhq_handle_t h, const float *coords, int64_t n,
+                                                float *out, void *stream);
 
 /* Layer sizes as the library pads them: K, M of layer `layer` (1-based).  Either may be NULL. */
 DHQ_API dhq_status_t dhq_layer_dims(dhq_handle_t h, int layer, int *K, int *M);

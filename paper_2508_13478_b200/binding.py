@@ -21,6 +21,7 @@ DHQ_GRAN_CHANNEL_OR_TOKEN = 1
 DHQ_ROT_INPUT = 0
 DHQ_ROT_BOTH = 1
 DHQ_ROT_NONE = 2
+DHQ_STATIC_MAX_TOKENS = 4096
 
 PIPES = {"ffma": 0, "fadd": 1, "mufu_sin": 2, "i2f": 3, "f2i": 4, "prmt": 5, "fmnmx": 6, "tensor_i8": 7}
 
@@ -61,6 +62,8 @@ def load_library():
     L.dhq_calibrate.argtypes = [vp, vp, c_i64, vp]
     L.dhq_forward.argtypes = [vp, vp, c_i64, vp, vp]
     L.dhq_forward_host.argtypes = [vp, vp, c_i64, vp, vp]
+    L.dhq_forward_static_scratch.argtypes = [vp, vp, c_i64, vp, vp]
+    L.dhq_forward_static_scratch.restype = c_i
     L.dhq_forward_debug.argtypes = [vp, vp, c_i64, vp, ctypes.POINTER(_DebugBufs), vp]
     L.dhq_get_layer.argtypes = [vp, c_i, vp, vp, vp]
     L.dhq_layer_dims.argtypes = [vp, c_i, ctypes.POINTER(c_i), ctypes.POINTER(c_i)]
@@ -127,6 +130,16 @@ def dhq_forward(handle, coords, out, stream=None):
     n = coords.shape[0]
     _check(load_library().dhq_forward(handle, _dev_ptr(coords, torch.float32, "coords"), n,
                                       _dev_ptr(out, torch.float32, "out"), _stream_ptr(stream)), "dhq_forward")
+
+
+def dhq_forward_static_scratch(handle, coords, out, stream=None):
+    """The forward pass for callers that must not allocate device memory: same arguments as
+    dhq_forward, at most DHQ_STATIC_MAX_TOKENS coordinates per call, scratch in a fixed array
+    inside the library.  This wrapper allocates nothing either."""
+    n = coords.shape[0]
+    _check(load_library().dhq_forward_static_scratch(handle, _dev_ptr(coords, torch.float32, "coords"), n,
+                                                     _dev_ptr(out, torch.float32, "out"), _stream_ptr(stream)),
+           "dhq_forward_static_scratch")
 
 
 def dhq_forward_host(handle, coords_host, out_host, stream=None):

@@ -8,7 +8,8 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libdhq_b200.so")
-SOURCES = ["dhq_api.cu", "dhq_prepare.cu", "dhq_layerwise.cu", "dhq_fused.cu", "dhq_peaks.cu"]
+SOURCES = ["dhq_api.cu", "dhq_prepare.cu", "dhq_layerwise.cu", "dhq_fused.cu", "dhq_peaks.cu",
+           "dhq_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--fmad=false", "-Xcompiler", "-fPIC,-fvisibility=hidden", "-shared", "-cudart", "shared"]
 

@@ -99,6 +99,7 @@ const char *dhq_status_string(dhq_status_t s)
     case DHQ_ERR_CUDA: return "CUDA runtime error";
     case DHQ_ERR_NOT_CALIBRATED: return "per-tensor activation scales are not calibrated";
     case DHQ_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case DHQ_ERR_TOO_LARGE: return "more tokens than the fixed-size scratch area holds";
     }
     return "unknown status";
 }
