@@ -25,6 +25,7 @@ void free_layer(LayerDev &d)
 {
     cudaFree(d.w_rot); cudaFree(d.row_absmax); cudaFree(d.qw); cudaFree(d.qw_k4m); cudaFree(d.qw_umma);
     cudaFree(d.s_w); cudaFree(d.inv_w); cudaFree(d.bias); cudaFree(d.cA); cudaFree(d.cA_lo); cudaFree(d.cB);
+    cudaFree(d.fxP); cudaFree(d.fxQ); cudaFree(d.fxB);
     cudaFree(d.act);
     d = LayerDev();
 }
@@ -56,6 +57,7 @@ LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X
     a.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
     a.epi_mode = d.epi_mode;
     a.qw_k4m = d.qw_k4m; a.cA = d.cA; a.cA_lo = d.cA_lo; a.cB = d.cB; a.act = d.act;
+    a.fxP = d.fxP; a.fxQ = d.fxQ; a.fxB = d.fxB;
     return a;
 }
 
@@ -159,11 +161,13 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             d.slab_rows = fused_slab_rows(d.K, d.Mt);
             d.d_in = cfg->dims[l - 1];
             d.d_out = cfg->dims[l];
+            if (l == 1) d.epi_mode = per_token ? EPI_SINE_WIDE : EPI_SINE_FIXED; // coordinates are not bounded by the weights
             const size_t MK = (size_t)d.M * d.K;
             bool ok = dev_alloc(&d.w_rot, MK) && dev_alloc(&d.row_absmax, d.M) && dev_alloc(&d.qw, MK) &&
                       dev_alloc(&d.qw_k4m, MK / 4) && dev_alloc(&d.qw_umma, (size_t)d.Mt * (d.K < 16 ? 16 : d.K)) &&
                       dev_alloc(&d.s_w, d.M) && dev_alloc(&d.inv_w, d.M) && dev_alloc(&d.bias, d.M) &&
                       dev_alloc(&d.cA, d.M) && dev_alloc(&d.cA_lo, d.M) && dev_alloc(&d.cB, d.M) &&
+                      dev_alloc(&d.fxP, d.M) && dev_alloc(&d.fxQ, d.M) && dev_alloc(&d.fxB, d.M) &&
                       dev_alloc(&d.act, 4);
             if (!ok) { rc = DHQ_ERR_ALLOC; break; }
             if (cudaMemsetAsync(d.act, 0, 16, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
@@ -191,7 +195,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             LayerDev &d = h->layer[l - 1];
             d.phase_bound = bounds[l - 1];
             if (l == L) d.epi_mode = EPI_LINEAR;
-            else if (l == 1) d.epi_mode = EPI_SINE_WIDE;   // coordinates are not bounded by the weights
+            else if (l == 1) {}
             else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit) ? EPI_SINE_FAST : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;

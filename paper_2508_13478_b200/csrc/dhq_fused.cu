@@ -1,24 +1,30 @@
-// Fused forward kernel: the whole quantized INR (Sections III-B and III-C of the paper) for a
-// tile of 128 coordinates without activations leaving the SM between layers.
+// Fused forward kernel: the whole quantized INR (Sections III-B and III-C of the paper) for
+// tiles of 128 coordinates without activations leaving the SM between layers.
 //
-// One persistent CTA per SM, 10 warps:
-//   warps 0-3, 4-7  two epilogue groups; each owns a "slot": one tile of 128 tokens in flight,
-//                   thread = one token (TMEM lane), so rotation, absmax and quantizer are
-//                   thread-local and need no exchange between threads.
-//   warp 8          issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in tensor memory).
-//   warp 9          brings the packed weight codes into shared memory with bulk async copies:
-//                   once, if every hidden layer fits (they then stay resident), else through a
-//                   ring that is refilled layer by layer from L2.
-// While one slot's threads run their epilogue on the CUDA cores, the tensor core works on the
-// other slot's tile.
+// One persistent CTA per SM, 18 warps:
+//   warps 0-15  epilogue warps.  Width <= 256: two "slots" of 8 warps, each slot has one tile of
+//               128 tokens in flight (its own A operand tile and 256 tensor-memory columns), so
+//               that one slot's CUDA-core work overlaps the other slot's MMA.  Width 512: one slot
+//               of 16 warps, the layer's MMA split in four N = 128 pieces so that the epilogue of
+//               piece j overlaps the MMA of piece j+1.
+//               A token (row) is a tensor-memory lane; R = 2 (or 4) threads from different warps
+//               share a row and split its columns.
+//   warp 16     issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in tensor memory).
+//   warp 17     brings the packed weight codes into shared memory with bulk async copies: once,
+//               if every hidden layer fits (they then stay resident), else through a ring that
+//               is refilled slab by slab from L2.
 //
-// Per layer and tile:  acc (TMEM, int32) -> dequantize, bias, sine (dhq_math.cuh) -> fp32
-//   -> butterfly stages with stride < 64 inside a 64-column register chunk -> the chunk goes back
-//   to the same TMEM columns as fp32 -> the remaining stages (stride 64, 128) combine one value
-//   from each chunk -> (per token: absmax, second trip through TMEM) -> quantize, pack 16 codes
-//   -> st.shared into the next layer's A operand tile -> mbarrier -> next MMA.
-// Layer 1 (K = 4) runs on the CUDA cores (one dp4a per output); the last layer is an MMA with
-// N = 16 whose first d_L columns are the result.
+// Per layer and tile:
+//   pass 1  each thread takes its chunks of 64 columns: acc (TMEM, int32) -> dequantize, bias,
+//           sine (dhq_math.cuh) -> butterfly stages with stride < 64 in registers -> fp32 back to
+//           the same TMEM columns.                                   [slot-wide mbarrier]
+//   pass 2  each thread takes its groups: one value from every chunk at G consecutive positions
+//           -> the remaining butterfly stages (stride 64, 128, ...) -> quantize, pack, st.shared
+//           into the next layer's A operand tile -> mbarrier -> next MMA.
+//           Per-token scales: the rotated values go back to TMEM once more while the row's
+//           absmax is combined through shared memory, then pass 3 quantizes.
+// Layer 1 (K = 4) runs on the CUDA cores; the last layer is an MMA with N = 16 whose first d_L
+// columns are the result.
 //
 // Every wait on an mbarrier is bounded: when it runs out the kernel records an error in the
 // handle's status word, all roles leave their loops, tensor memory is released and the kernel
@@ -31,19 +37,36 @@
 namespace dhq {
 
 constexpr int kTile = 128;
-constexpr int kThreads = 320;
-constexpr int kMmaWarp = 8, kLoadWarp = 9;
+constexpr int kEpiWarps = 16;
+constexpr int kMmaWarp = 16, kLoadWarp = 17;
+constexpr int kThreads = 18 * 32;
 constexpr int kMaxStages = 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull; // 2 s per wait
 constexpr int kMinSmem = 120 * 1024; // more than half an SM's shared memory: one CTA per SM
+
+// Work split for a hidden width W.
+template <int W> struct Cfg {
+    static constexpr int SLOTS = (W == 512) ? 1 : 2;
+    static constexpr int R = kEpiWarps / (4 * SLOTS);          // threads per row: 2 or 4
+    static constexpr int CH = (W / R < 64) ? W / R : 64;       // columns per register chunk
+    static constexpr int NCH = W / CH;                         // chunks per row
+    static constexpr int CPT = NCH / R;                        // chunks per thread
+    static constexpr int G = (64 / NCH < CH / R) ? 64 / NCH : CH / R; // positions per pass-2 group
+    static constexpr int GPT = CH / (G * R);                   // groups per thread
+    static constexpr int PIECES = (W == 512) ? 4 : 1;          // MMAs per layer along N
+    static constexpr int PW = W / PIECES;                      // N of one MMA = rows of one weight slab
+    static constexpr int SLOT_THREADS = R * kTile;
+    static constexpr int TMEM_COLS_PER_SLOT = 512 / SLOTS;
+};
 
 struct FusedLayer {
     const uint8_t *qw_umma;
     const uint32_t *qw_k4m;
     const float *cA, *cA_lo, *cB;
+    const uint32_t *fxP, *fxQ, *fxB;
     const float *act;
     int epi_mode;
-    int pad_;
+    int c_off; // word offset of this layer's constants in the shared-memory constant area
 };
 
 struct FusedParams {
@@ -53,6 +76,7 @@ struct FusedParams {
     int L, W, d_L, per_token;
     float qmaxf;
     int n_stages, resident;
+    int const_words;
     int *status;
     FusedLayer layer[kMaxLayers];
 };
@@ -63,29 +87,36 @@ struct FusedState {
     int sm_count;
 };
 
-// Shared-memory map (offsets from a 1024-byte aligned base).
+// Shared-memory map (byte offsets from a 1024-byte aligned base).
 struct SmemMap {
     uint32_t a_tile[2];
-    uint32_t ring;
-    uint32_t last_w;
-    uint32_t acc_full[2], codes_full[2], last_full, drain;
-    uint32_t w_full, w_empty; // arrays of kMaxStages barriers
+    uint32_t ring, last_w, consts, amax;
+    uint32_t acc_full;   // [2 slots][4 pieces]
+    uint32_t acc_last;   // [2]
+    uint32_t codes_full; // [2]
+    uint32_t slot_sync;  // [2]
+    uint32_t last_full, drain;
+    uint32_t w_full, w_empty; // [kMaxStages] each
     uint32_t tmem_holder, abort_flag;
     uint32_t total;
 };
 
-__host__ __device__ inline SmemMap smem_map(int W, int n_stages)
+__host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words)
 {
+    const int slots = (W == 512) ? 1 : 2;
+    const int pw = (W == 512) ? 128 : W;
     SmemMap m;
     uint32_t off = 0;
     m.a_tile[0] = off; off += kTile * W;
-    m.a_tile[1] = off; off += kTile * W;
-    m.ring = off; off += (uint32_t)n_stages * W * W;
+    m.a_tile[1] = off; if (slots == 2) off += kTile * W;
+    m.ring = off; off += (uint32_t)n_stages * pw * W;
     m.last_w = off; off += 16 * W;
-    m.acc_full[0] = off; off += 8;
-    m.acc_full[1] = off; off += 8;
-    m.codes_full[0] = off; off += 8;
-    m.codes_full[1] = off; off += 8;
+    m.consts = off; off += (uint32_t)const_words * 4;
+    m.amax = off; off += 2 * 4 * kTile * 4;
+    m.acc_full = off; off += 8 * 8;
+    m.acc_last = off; off += 8 * 2;
+    m.codes_full = off; off += 8 * 2;
+    m.slot_sync = off; off += 8 * 2;
     m.last_full = off; off += 8;
     m.drain = off; off += 8;
     m.w_full = off; off += 8 * kMaxStages;
@@ -113,6 +144,11 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         }
     }
 }
+// The same for a whole warp: every lane takes the same decision.
+__device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_flag, status));
+}
 
 // In-register butterfly stages with strides 1 .. N/2 on N values: pair (i, i+h) -> (a+b, a-b).
 template <int N> __device__ __forceinline__ void fwht_local(float (&f)[N])
@@ -130,13 +166,14 @@ template <int N> __device__ __forceinline__ void fwht_local(float (&f)[N])
     }
 }
 
-// Round-half-even to an integer code held in the low byte: clamp, then add 1.5 * 2^23 (the sum
-// rounds to the integer grid, ties to even, and its low mantissa bits are the two's complement
-// code).  Same integer as __float2int_rn(clamp(v * inv)).
-__device__ __forceinline__ uint32_t code_bits(float v, float inv, float qmaxf)
+// Round-half-even to an integer code held in the low byte: (clamp,) then add 1.5 * 2^23 (the
+// sum rounds to the integer grid, ties to even, and its low mantissa bits are the two's
+// complement code).  Same integer as __float2int_rn(clamp(v * inv)).  With a per-token scale
+// |v * inv| <= qmax (1 + 2^-23) already, so the clamp is skipped.
+template <bool CLAMP> __device__ __forceinline__ uint32_t code_bits(float v, float inv, float qmaxf)
 {
     float t = __fmul_rn(v, inv);
-    t = fmaxf(fminf(t, qmaxf), -qmaxf);
+    if (CLAMP) t = fmaxf(fminf(t, qmaxf), -qmaxf);
     return __float_as_uint(__fadd_rn(t, 12582912.0f));
 }
 __device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3)
@@ -145,164 +182,261 @@ __device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2,
     uint32_t hi = __byte_perm(b2, b3, 0x0040);
     return __byte_perm(lo, hi, 0x5410);
 }
-// Quantize 16 consecutive-k values of this thread's token and store them as one 16-byte k-group
-// of the A operand tile: byte offset (k/16) * 2048 + row * 16.
-__device__ __forceinline__ void store_codes16(uint32_t a_tile, int row, int kgroup, const float *v, float inv, float qmaxf)
+// Quantize N (8 or 16) consecutive-k values of this thread's token, k0 a multiple of N, and store
+// them into the A operand tile: byte offset (k/16) * 2048 + row * 16 + k % 16.
+template <int N, bool CLAMP>
+__device__ __forceinline__ void store_codes(uint32_t a_tile, int row, int k0, const uint32_t *v, float inv, float qmaxf)
 {
-    uint32_t w[4];
+    uint32_t w[N / 4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-        w[j] = pack4(code_bits(v[4 * j], inv, qmaxf), code_bits(v[4 * j + 1], inv, qmaxf),
-                     code_bits(v[4 * j + 2], inv, qmaxf), code_bits(v[4 * j + 3], inv, qmaxf));
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_tile + kgroup * 2048 + row * 16),
-                 "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+    for (int j = 0; j < N / 4; ++j)
+        w[j] = pack4(code_bits<CLAMP>(__uint_as_float(v[4 * j]), inv, qmaxf),
+                     code_bits<CLAMP>(__uint_as_float(v[4 * j + 1]), inv, qmaxf),
+                     code_bits<CLAMP>(__uint_as_float(v[4 * j + 2]), inv, qmaxf),
+                     code_bits<CLAMP>(__uint_as_float(v[4 * j + 3]), inv, qmaxf));
+    const uint32_t addr = a_tile + (k0 >> 4) * 2048 + row * 16 + (k0 & 15);
+    if constexpr (N == 16)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+    else
+        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(w[0]), "r"(w[1]) : "memory");
 }
 
-// Dequantize + bias + activation of 64 consecutive channels starting at m0.
-template <bool PER_TOKEN, int MODE>
-__device__ __forceinline__ void epilogue64_mode(const FusedLayer &ly, int m0, float s_x, const int (&acc)[64], float (&f)[64])
+template <int N> __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[N])
 {
-    const float4 *cA4 = reinterpret_cast<const float4 *>(ly.cA + m0);
-    const float4 *cL4 = reinterpret_cast<const float4 *>(ly.cA_lo + m0);
-    const float4 *cB4 = reinterpret_cast<const float4 *>(ly.cB + m0);
+    if constexpr (N == 8) ptx::tmem_ld8(taddr, v);
+    else if constexpr (N == 16) ptx::tmem_ld16(taddr, v);
+    else if constexpr (N == 32) ptx::tmem_ld32(taddr, v);
+    else ptx::tmem_ld64(taddr, v);
+}
+template <int N> __device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&v)[N])
+{
+    if constexpr (N == 8) ptx::tmem_st8(taddr, v);
+    else if constexpr (N == 16) ptx::tmem_st16(taddr, v);
+    else if constexpr (N == 32) ptx::tmem_st32(taddr, v);
+    else ptx::tmem_st64(taddr, v);
+}
+
+__device__ __forceinline__ float4 lds128(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
+// Dequantize + bias + sine of CH consecutive channels starting at m0, in place: v holds the
+// int32 accumulators on entry and the fp32 activations (as bits) on exit.  Constants come from
+// shared memory: area A = cA, B = cB, C = cA_lo, each W words.
+template <int W, int CH, bool PER_TOKEN, int MODE>
+__device__ __forceinline__ void epilogue_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH])
+{
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        float4 a = __ldg(cA4 + j), b = __ldg(cB4 + j);
+    for (int j = 0; j < CH / 4; ++j) {
+        const float4 a = lds128(cbase + (m0 + 4 * j) * 4);
+        const float4 b = lds128(cbase + (W + m0 + 4 * j) * 4);
         float4 lo = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (MODE == EPI_SINE_WIDE) lo = __ldg(cL4 + j);
+        if (MODE == EPI_SINE_WIDE) lo = lds128(cbase + (2 * W + m0 + 4 * j) * 4);
         const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w}, lv[4] = {lo.x, lo.y, lo.z, lo.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             float c_hi = av[e], c_lo = lv[e];
             if (PER_TOKEN) token_const(av[e], lv[e], s_x, c_hi, c_lo);
-            f[4 * j + e] = epilogue(MODE, (float)acc[4 * j + e], c_hi, c_lo, bv[e]);
+            v[4 * j + e] = __float_as_uint(epilogue(MODE, (float)(int)v[4 * j + e], c_hi, c_lo, bv[e]));
         }
     }
 }
-template <bool PER_TOKEN>
-__device__ __forceinline__ void epilogue64(const FusedLayer &ly, int m0, float s_x, const int (&acc)[64], float (&f)[64])
+
+// Layer 1 for CH channels starting at m0.  Fixed-point mode: areas A = P, B = B, C = Q.
+// Float mode (per-token scales): A = cA, B = cB, C = cA_lo, D = the weight codes, one word per
+// channel, and acc = dp4a(codes of the token, codes of the channel).
+template <int W, int CH, bool PER_TOKEN>
+__device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int qd, uint32_t qx, float s_x, uint32_t (&v)[CH])
 {
-    if (ly.epi_mode == EPI_SINE_FAST) epilogue64_mode<PER_TOKEN, EPI_SINE_FAST>(ly, m0, s_x, acc, f);
-    else epilogue64_mode<PER_TOKEN, EPI_SINE_WIDE>(ly, m0, s_x, acc, f);
+    if constexpr (!PER_TOKEN) {
+#pragma unroll
+        for (int j = 0; j < CH / 4; ++j) {
+            const float4 P = lds128(cbase + (m0 + 4 * j) * 4);
+            const float4 B = lds128(cbase + (W + m0 + 4 * j) * 4);
+            const float4 Q = lds128(cbase + (2 * W + m0 + 4 * j) * 4);
+            const float Pv[4] = {P.x, P.y, P.z, P.w}, Bv[4] = {B.x, B.y, B.z, B.w}, Qv[4] = {Q.x, Q.y, Q.z, Q.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                v[4 * j + e] = __float_as_uint(sine_fixed(qs, qd, __float_as_uint(Pv[e]), __float_as_uint(Qv[e]), __float_as_uint(Bv[e])));
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < CH / 4; ++j) {
+            const float4 wq = lds128(cbase + (3 * W + m0 + 4 * j) * 4);
+            v[4 * j + 0] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.x), 0);
+            v[4 * j + 1] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.y), 0);
+            v[4 * j + 2] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.z), 0);
+            v[4 * j + 3] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.w), 0);
+        }
+        epilogue_chunk<W, CH, true, EPI_SINE_WIDE>(cbase, m0, s_x, v);
+    }
 }
 
-// After the 64-column chunks have been through the local stages: the remaining stages, the
-// quantizer and the store of the codes.  W = 64: everything is still in registers (f).
-// W > 64: chunk c of the token sits in TMEM columns [c*64, c*64+64) as fp32.
-// Returns the token's activation scale s_x of this layer (needed by the next epilogue).
-template <int W, bool PER_TOKEN>
-__device__ __forceinline__ float cross_and_quantize(uint32_t taddr, uint32_t a_tile, int row, float (&f)[64],
-                                                    float static_s, float static_inv, float qmaxf)
+template <int CH> __device__ __forceinline__ void fwht_chunk(uint32_t (&v)[CH])
 {
-    constexpr int NCH = W / 64;
-    if constexpr (NCH == 1) {
-        float s = static_s, inv = static_inv;
-        if (PER_TOKEN) {
-            float a = 0.f;
+    float f[CH];
 #pragma unroll
-            for (int i = 0; i < 64; ++i) a = fmaxf(a, fabsf(f[i]));
-            scales_of(a, qmaxf, s, inv);
-        }
+    for (int i = 0; i < CH; ++i) f[i] = __uint_as_float(v[i]);
+    fwht_local<CH>(f);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) store_codes16(a_tile, row, g, &f[16 * g], inv, qmaxf);
-        return s;
-    } else {
-        constexpr int G = 64 / NCH; // local indices per group: NCH * G = 64 values in registers
-        constexpr int NG = 64 / G;
-        ptx::tmem_wait_st();
-        float amax = 0.f;
+    for (int i = 0; i < CH; ++i) v[i] = __float_as_uint(f[i]);
+}
+
+// Everything a slot's threads need to finish a layer once their chunks are back in tensor memory.
+struct SlotCtx {
+    uint32_t taddr;      // TMEM address of this thread's lane, column 0 of the slot
+    uint32_t a_tile;     // shared-memory address of the slot's A operand tile
+    uint32_t bar_sync;   // slot-wide mbarrier
+    uint32_t bar_codes;  // "codes ready" mbarrier
+    uint32_t amax_addr;  // shared memory: [R][128] floats for this slot
+    uint32_t sync_parity;
+    int row, sub;
+    float qmaxf;
+    volatile int *abort_flag;
+    int *status;
+};
+
+__device__ __forceinline__ bool slot_barrier(SlotCtx &c)
+{
+    ptx::mbar_arrive(c.bar_sync);
+    bool ok = wait_bar_warp(c.bar_sync, c.sync_parity, c.abort_flag, c.status);
+    c.sync_parity ^= 1;
+    return ok;
+}
+
+// Passes 2 and 3: remaining butterfly stages across chunks, quantizer, store of the codes, and the
+// arrival on the "codes ready" barrier.  Returns false if a wait ran out.  s_out receives the
+// token's activation scale of the next layer.
+template <int W, bool PER_TOKEN>
+__device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float static_inv, float &s_out)
+{
+    using C = Cfg<W>;
+    constexpr int NCH = C::NCH, G = C::G, CH = C::CH;
+    constexpr int SN = (G >= 16) ? 16 : 8; // codes per shared-memory store
+    ptx::tmem_wait_st();
+    ptx::tc_fence_before();
+    if (!slot_barrier(c)) return false;
+    ptx::tc_fence_after();
+    float amax = 0.f;
 #pragma unroll 1
-        for (int g = 0; g < NG; ++g) {
+    for (int gg = 0; gg < C::GPT; ++gg) {
+        const int g = c.sub * C::GPT + gg;
+        uint32_t u[NCH][G];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
+        ptx::tmem_wait_ld();
+        // strides CH, 2 CH, ...: the chunk index is the butterfly index
+#pragma unroll
+        for (int h = 1; h < NCH; h <<= 1) {
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                if ((ch & h) == 0) {
+#pragma unroll
+                    for (int i = 0; i < G; ++i) {
+                        float a = __uint_as_float(u[ch][i]), b = __uint_as_float(u[ch + h][i]);
+                        u[ch][i] = __float_as_uint(__fadd_rn(a, b));
+                        u[ch + h][i] = __float_as_uint(__fsub_rn(a, b));
+                    }
+                }
+            }
+        }
+        if (PER_TOKEN) {
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+#pragma unroll
+                for (int i = 0; i < G; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(u[ch][i])));
+                tmem_st<G>(c.taddr + ch * CH + g * G, u[ch]);
+            }
+        } else {
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+#pragma unroll
+                for (int i = 0; i < G; i += SN)
+                    store_codes<SN, true>(c.a_tile, c.row, ch * CH + g * G + i, &u[ch][i], static_inv, c.qmaxf);
+            }
+        }
+    }
+    if (!PER_TOKEN) {
+        s_out = static_s;
+    } else {
+        // combine the row's absmax over the R threads that share it
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(c.amax_addr + (c.sub * kTile + c.row) * 4), "f"(amax) : "memory");
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before();
+        if (!slot_barrier(c)) return false;
+        ptx::tc_fence_after();
+#pragma unroll
+        for (int r = 0; r < C::R; ++r) {
+            float o;
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(o) : "r"(c.amax_addr + (r * kTile + c.row) * 4));
+            amax = fmaxf(amax, o);
+        }
+        float s, inv;
+        scales_of(amax, c.qmaxf, s, inv);
+        s_out = s;
+#pragma unroll 1
+        for (int gg = 0; gg < C::GPT; ++gg) {
+            const int g = c.sub * C::GPT + gg;
             uint32_t u[NCH][G];
 #pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                if constexpr (G == 16) ptx::tmem_ld16(taddr + c * 64 + g * G, u[c]);
-                else if constexpr (G == 32) ptx::tmem_ld32(taddr + c * 64 + g * G, u[c]);
-                else ptx::tmem_ld8(taddr + c * 64 + g * G, u[c]);
-            }
-            ptx::tmem_wait_ld();
-            // strides 64, 128, ...: chunk index is the butterfly index
-#pragma unroll
-            for (int h = 1; h < NCH; h <<= 1) {
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    if ((c & h) == 0) {
-#pragma unroll
-                        for (int i = 0; i < G; ++i) {
-                            float a = __uint_as_float(u[c][i]), b = __uint_as_float(u[c + h][i]);
-                            u[c][i] = __float_as_uint(__fadd_rn(a, b));
-                            u[c + h][i] = __float_as_uint(__fsub_rn(a, b));
-                        }
-                    }
-                }
-            }
-            if (PER_TOKEN) {
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-#pragma unroll
-                    for (int i = 0; i < G; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(u[c][i])));
-                    if constexpr (G == 16) ptx::tmem_st16(taddr + c * 64 + g * G, u[c]);
-                    else if constexpr (G == 32) ptx::tmem_st32(taddr + c * 64 + g * G, u[c]);
-                    else ptx::tmem_st8(taddr + c * 64 + g * G, u[c]);
-                }
-            } else {
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-#pragma unroll
-                    for (int i = 0; i < G; i += 16) {
-                        float v[16];
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) v[e] = __uint_as_float(u[c][i + e]);
-                        store_codes16(a_tile, row, (c * 64 + g * G + i) / 16, v, static_inv, qmaxf);
-                    }
-                }
-            }
-        }
-        if (!PER_TOKEN) return static_s;
-        float s, inv;
-        scales_of(amax, qmaxf, s, inv);
-        ptx::tmem_wait_st();
-#pragma unroll 1
-        for (int c = 0; c < NCH; ++c) {
-            uint32_t u[64];
-            ptx::tmem_ld64(taddr + c * 64, u);
+            for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
             ptx::tmem_wait_ld();
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                float v[16];
+            for (int ch = 0; ch < NCH; ++ch) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = __uint_as_float(u[16 * g + e]);
-                store_codes16(a_tile, row, c * 4 + g, v, inv, qmaxf);
+                for (int i = 0; i < G; i += SN)
+                    store_codes<SN, false>(c.a_tile, c.row, ch * CH + g * G + i, &u[ch][i], inv, c.qmaxf);
             }
         }
-        return s;
     }
+    ptx::fence_proxy_async();
+    ptx::tc_fence_before();
+    ptx::mbar_arrive(c.bar_codes);
+    return true;
 }
 
 template <int W, bool PER_TOKEN>
-__device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, int slot, int quad, int lane,
+__device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
-    constexpr int NCH = W / 64;
-    const int row = quad * 32 + lane;
-    const uint32_t taddr = tmem_base + (uint32_t)(slot * 256) + ((uint32_t)(quad * 32) << 16);
-    const uint32_t a_tile = smem_base + sm.a_tile[slot];
-    const uint32_t bar_acc = smem_base + sm.acc_full[slot], bar_codes = smem_base + sm.codes_full[slot];
-    const float qmaxf = p.qmaxf;
-    uint32_t acc_parity = 0;
+    using C = Cfg<W>;
+    constexpr int CH = C::CH;
+    const int slot = warp / (4 * C::R);
+    const int quad = warp & 3;
+    const int sub = (warp % (4 * C::R)) >> 2;
+    SlotCtx c;
+    c.row = quad * 32 + lane;
+    c.sub = sub;
+    c.taddr = tmem_base + (uint32_t)(slot * C::TMEM_COLS_PER_SLOT) + ((uint32_t)(quad * 32) << 16);
+    c.a_tile = smem_base + sm.a_tile[slot];
+    c.bar_sync = smem_base + sm.slot_sync + 8 * slot;
+    c.bar_codes = smem_base + sm.codes_full + 8 * slot;
+    c.amax_addr = smem_base + sm.amax + slot * (4 * kTile * 4);
+    c.sync_parity = 0;
+    c.qmaxf = p.qmaxf;
+    c.abort_flag = abort_flag;
+    c.status = p.status;
+    const uint32_t bar_acc = smem_base + sm.acc_full + 8 * (slot * 4 + (sub * C::PIECES) / C::R);
+    const uint32_t bar_last = smem_base + sm.acc_last + 8 * slot;
+    const uint32_t consts = smem_base + sm.consts;
+    uint32_t acc_parity = 0, last_parity = 0;
     const FusedLayer &l1 = p.layer[0];
+    const float qmaxf = p.qmaxf;
 
     for (long long r = 0;; ++r) {
-        const long long tile = ((long long)blockIdx.x + r * gridDim.x) * 2 + slot;
+        const long long tile = ((long long)blockIdx.x + r * gridDim.x) * C::SLOTS + slot;
         if (tile >= p.n_tiles) break;
-        const long long tok = tile * kTile + row;
+        const long long tok = tile * kTile + c.row;
         const bool valid = tok < p.n;
 
         // ---------------- layer 1 on the CUDA cores: x~ = H_4 [x, y, 0, 0]
         float x = 0.f, y = 0.f;
         if (valid) {
-            float2 c = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
-            x = c.x; y = c.y;
+            float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
+            x = xy.x; y = xy.y;
         }
         float r0 = __fadd_rn(x, y), r1 = __fsub_rn(x, y), r2 = __fadd_rn(0.f, 0.f), r3 = __fsub_rn(0.f, 0.f);
         float e0 = __fadd_rn(r0, r2), e2 = __fsub_rn(r0, r2), e1 = __fadd_rn(r1, r3), e3 = __fsub_rn(r1, r3);
@@ -314,79 +448,58 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
             s_x = __ldg(l1.act + 1);
             inv_x = __ldg(l1.act + 2);
         }
-        const uint32_t qx = pack4(code_bits(e0, inv_x, qmaxf), code_bits(e1, inv_x, qmaxf),
-                                  code_bits(e2, inv_x, qmaxf), code_bits(e3, inv_x, qmaxf));
+        const uint32_t b0 = code_bits<true>(e0, inv_x, qmaxf), b1 = code_bits<true>(e1, inv_x, qmaxf);
+        const uint32_t qx = pack4(b0, b1, code_bits<true>(e2, inv_x, qmaxf), code_bits<true>(e3, inv_x, qmaxf));
+        const int qs = (int)b0 - 0x4B400000, qd = (int)b1 - 0x4B400000;
         float next_s = 1.f, next_inv = 0.f;
         if (!PER_TOKEN) {
             next_s = __ldg(p.layer[1].act + 1);
             next_inv = __ldg(p.layer[1].act + 2);
         }
-        {
-            float f[64];
 #pragma unroll 1
-            for (int ch = 0; ch < NCH; ++ch) {
-                int acc[64];
-                const uint4 *w4 = reinterpret_cast<const uint4 *>(l1.qw_k4m + ch * 64);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    uint4 w = __ldg(w4 + j);
-                    acc[4 * j + 0] = __dp4a((int)qx, (int)w.x, 0);
-                    acc[4 * j + 1] = __dp4a((int)qx, (int)w.y, 0);
-                    acc[4 * j + 2] = __dp4a((int)qx, (int)w.z, 0);
-                    acc[4 * j + 3] = __dp4a((int)qx, (int)w.w, 0);
-                }
-                epilogue64_mode<PER_TOKEN, EPI_SINE_WIDE>(l1, ch * 64, s_x, acc, f);
-                fwht_local<64>(f);
-                if constexpr (NCH > 1) {
-                    uint32_t u[64];
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) u[i] = __float_as_uint(f[i]);
-                    ptx::tmem_st64(taddr + ch * 64, u);
-                }
-            }
-            s_x = cross_and_quantize<W, PER_TOKEN>(taddr, a_tile, row, f, next_s, next_inv, qmaxf);
+        for (int cc = 0; cc < C::CPT; ++cc) {
+            const int ch = sub * C::CPT + cc;
+            uint32_t v[CH];
+            layer1_chunk<W, CH, PER_TOKEN>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v);
+            fwht_chunk<CH>(v);
+            tmem_st<CH>(c.taddr + ch * CH, v);
         }
-        ptx::fence_proxy_async();
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(bar_codes);
+        if (!finish_layer<W, PER_TOKEN>(c, next_s, next_inv, s_x)) return;
 
         // ---------------- layers 2 .. L on the tensor core
-        for (int l = 2; l <= p.L; ++l) {
+        for (int l = 2; l < p.L; ++l) {
             const FusedLayer &ly = p.layer[l - 1];
-            if (!__all_sync(0xffffffffu, wait_bar(bar_acc, acc_parity, abort_flag, p.status))) return;
+            if (!wait_bar_warp(bar_acc, acc_parity, abort_flag, p.status)) return;
             acc_parity ^= 1;
             ptx::tc_fence_after();
-            if (l < p.L) {
-                if (!PER_TOKEN) {
-                    next_s = __ldg(p.layer[l].act + 1);
-                    next_inv = __ldg(p.layer[l].act + 2);
-                }
-                float f[64];
+            if (!PER_TOKEN) {
+                next_s = __ldg(p.layer[l].act + 1);
+                next_inv = __ldg(p.layer[l].act + 2);
+            }
+            const uint32_t cbase = consts + ly.c_off * 4;
+            const bool fast = ly.epi_mode == EPI_SINE_FAST;
 #pragma unroll 1
-                for (int ch = 0; ch < NCH; ++ch) {
-                    uint32_t u[64];
-                    ptx::tmem_ld64(taddr + ch * 64, u);
-                    ptx::tmem_wait_ld();
-                    int acc[64];
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) acc[i] = (int)u[i];
-                    epilogue64<PER_TOKEN>(ly, ch * 64, s_x, acc, f);
-                    fwht_local<64>(f);
-                    if constexpr (NCH > 1) {
-#pragma unroll
-                        for (int i = 0; i < 64; ++i) u[i] = __float_as_uint(f[i]);
-                        ptx::tmem_st64(taddr + ch * 64, u);
-                    }
-                }
-                s_x = cross_and_quantize<W, PER_TOKEN>(taddr, a_tile, row, f, next_s, next_inv, qmaxf);
-                ptx::fence_proxy_async();
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(bar_codes);
-            } else {
-                uint32_t u[4];
-                ptx::tmem_ld4(taddr, u);
+            for (int cc = 0; cc < C::CPT; ++cc) {
+                const int ch = sub * C::CPT + cc;
+                uint32_t v[CH];
+                tmem_ld<CH>(c.taddr + ch * CH, v);
                 ptx::tmem_wait_ld();
-                ptx::tc_fence_before();
+                if (fast) epilogue_chunk<W, CH, PER_TOKEN, EPI_SINE_FAST>(cbase, ch * CH, s_x, v);
+                else epilogue_chunk<W, CH, PER_TOKEN, EPI_SINE_WIDE>(cbase, ch * CH, s_x, v);
+                fwht_chunk<CH>(v);
+                tmem_st<CH>(c.taddr + ch * CH, v);
+            }
+            if (!finish_layer<W, PER_TOKEN>(c, next_s, next_inv, s_x)) return;
+        }
+        {
+            const FusedLayer &ly = p.layer[p.L - 1];
+            if (!wait_bar_warp(bar_last, last_parity, abort_flag, p.status)) return;
+            last_parity ^= 1;
+            ptx::tc_fence_after();
+            if (sub == 0) {
+                uint32_t u[4];
+                ptx::tmem_ld4(c.taddr, u);
+                ptx::tmem_wait_ld();
                 if (valid) {
 #pragma unroll
                     for (int m = 0; m < 4; ++m) {
@@ -398,6 +511,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
                     }
                 }
             }
+            ptx::tc_fence_before();
         }
     }
 }
@@ -406,49 +520,56 @@ template <int W>
 __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, uint32_t tmem_base,
                          volatile int *abort_flag)
 {
+    using C = Cfg<W>;
     uint32_t codes_parity[2] = {0, 0};
-    const uint32_t idesc_hidden = ptx::idesc_i8(kTile, W), idesc_last = ptx::idesc_i8(kTile, 16);
+    const uint32_t idesc_hidden = ptx::idesc_i8(kTile, C::PW), idesc_last = ptx::idesc_i8(kTile, 16);
+    const uint32_t slab = C::PW * W;
     long long use = 0; // ring uses so far (streaming mode)
     bool ok = true;
     for (long long r = 0; ok; ++r) {
-        const long long tile0 = ((long long)blockIdx.x + r * gridDim.x) * 2;
+        const long long tile0 = ((long long)blockIdx.x + r * gridDim.x) * C::SLOTS;
         if (tile0 >= p.n_tiles) break;
-        const bool active1 = tile0 + 1 < p.n_tiles;
+        const int active = (C::SLOTS == 2 && tile0 + 1 < p.n_tiles) ? 2 : 1;
         for (int l = 2; l <= p.L && ok; ++l) {
-            uint32_t b_addr, n_rows, idesc;
-            int stage = 0;
-            if (l < p.L) {
-                stage = p.resident ? (l - 2) : (int)(use % p.n_stages);
-                uint32_t par = p.resident ? 0u : (uint32_t)((use / p.n_stages) & 1);
-                if (!wait_bar(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
-                b_addr = smem_base + sm.ring + (uint32_t)stage * W * W;
-                n_rows = W;
-                idesc = idesc_hidden;
-            } else {
-                if (!wait_bar(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
-                b_addr = smem_base + sm.last_w;
-                n_rows = 16;
-                idesc = idesc_last;
-            }
-            for (int s = 0; s < 2; ++s) {
-                if (s == 1 && !active1) break;
-                if (!wait_bar(smem_base + sm.codes_full[s], codes_parity[s], abort_flag, p.status)) { ok = false; break; }
-                codes_parity[s] ^= 1;
-                ptx::tc_fence_after();
-                const uint32_t a_addr = smem_base + sm.a_tile[s];
-                const uint32_t d = tmem_base + (uint32_t)(s * 256);
-#pragma unroll 1
-                for (int ks = 0; ks < W / 32; ++ks) {
-                    uint64_t ad = ptx::smem_desc(a_addr + ks * 2 * (kTile * 16), kTile * 16, 128);
-                    uint64_t bd = ptx::smem_desc(b_addr + ks * 2 * (n_rows * 16), n_rows * 16, 128);
-                    ptx::mma_i8(d, ad, bd, idesc, ks > 0 ? 1u : 0u);
+            const int pieces = (l < p.L) ? C::PIECES : 1;
+            for (int pc = 0; pc < pieces && ok; ++pc) {
+                uint32_t b_addr, n_rows, idesc;
+                int stage = 0;
+                if (l < p.L) {
+                    const int slab_id = (l - 2) * C::PIECES + pc;
+                    stage = p.resident ? slab_id : (int)(use % p.n_stages);
+                    const uint32_t par = p.resident ? 0u : (uint32_t)((use / p.n_stages) & 1);
+                    if (!wait_bar(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
+                    b_addr = smem_base + sm.ring + (uint32_t)stage * slab;
+                    n_rows = C::PW;
+                    idesc = idesc_hidden;
+                } else {
+                    if (!wait_bar(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
+                    b_addr = smem_base + sm.last_w;
+                    n_rows = 16;
+                    idesc = idesc_last;
                 }
-                ptx::mma_commit(smem_base + sm.acc_full[s]);
-            }
-            if (!ok) break;
-            if (l < p.L && !p.resident) {
-                ptx::mma_commit(smem_base + sm.w_empty + 8 * stage);
-                ++use;
+                for (int s = 0; s < active; ++s) {
+                    if (pc == 0) {
+                        if (!wait_bar(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
+                        codes_parity[s] ^= 1;
+                        ptx::tc_fence_after();
+                    }
+                    const uint32_t a_addr = smem_base + sm.a_tile[s];
+                    const uint32_t d = tmem_base + (uint32_t)(s * C::TMEM_COLS_PER_SLOT) + (l < p.L ? pc * C::PW : 0);
+#pragma unroll 1
+                    for (int ks = 0; ks < W / 32; ++ks) {
+                        uint64_t ad = ptx::smem_desc(a_addr + ks * 2 * (kTile * 16), kTile * 16, 128);
+                        uint64_t bd = ptx::smem_desc(b_addr + ks * 2 * (n_rows * 16), n_rows * 16, 128);
+                        ptx::mma_i8(d, ad, bd, idesc, ks > 0 ? 1u : 0u);
+                    }
+                    ptx::mma_commit(l < p.L ? smem_base + sm.acc_full + 8 * (s * 4 + pc) : smem_base + sm.acc_last + 8 * s);
+                }
+                if (!ok) break;
+                if (l < p.L && !p.resident) {
+                    ptx::mma_commit(smem_base + sm.w_empty + 8 * stage);
+                    ++use;
+                }
             }
         }
     }
@@ -462,17 +583,18 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
 template <int W>
 __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
 {
-    const uint32_t slab = W * W;
+    using C = Cfg<W>;
+    const uint32_t slab = C::PW * W;
     ptx::mbar_expect_tx(smem_base + sm.last_full, 16 * W);
     ptx::bulk_g2s(smem_base + sm.last_w, p.layer[p.L - 1].qw_umma, 16 * W, smem_base + sm.last_full);
-    const int hidden = p.L - 2;
-    if (hidden <= 0) return;
+    const int slabs = (p.L - 2) * C::PIECES; // per tile round
+    if (slabs <= 0) return;
     long long rounds = 0;
     for (long long r = 0;; ++r) {
-        if (((long long)blockIdx.x + r * gridDim.x) * 2 >= p.n_tiles) break;
+        if (((long long)blockIdx.x + r * gridDim.x) * C::SLOTS >= p.n_tiles) break;
         ++rounds;
     }
-    const long long total = p.resident ? hidden : rounds * hidden;
+    const long long total = p.resident ? slabs : rounds * slabs;
     long long issued = 0;
     bool ok = true;
     for (long long i = 0; i < total; ++i) {
@@ -481,9 +603,10 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
             uint32_t par = (uint32_t)(((i / p.n_stages) - 1) & 1);
             if (!wait_bar(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
         }
-        const int l = 2 + (int)(i % hidden);
+        const int id = (int)(i % slabs);
+        const int l = 2 + id / C::PIECES, pc = id % C::PIECES;
         ptx::mbar_expect_tx(smem_base + sm.w_full + 8 * stage, slab);
-        ptx::bulk_g2s(smem_base + sm.ring + (uint32_t)stage * slab, p.layer[l - 1].qw_umma, slab,
+        ptx::bulk_g2s(smem_base + sm.ring + (uint32_t)stage * slab, p.layer[l - 1].qw_umma + (size_t)pc * slab, slab,
                       smem_base + sm.w_full + 8 * stage);
         ++issued;
     }
@@ -501,20 +624,23 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
 template <int W, bool PER_TOKEN>
 __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constant__ FusedParams p)
 {
+    using C = Cfg<W>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t smem_base = (raw + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - raw);
-    const SmemMap sm = smem_map(W, p.n_stages);
+    const SmemMap sm = smem_map(W, p.n_stages, p.const_words);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_gen + sm.abort_flag);
     volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(smem_gen + sm.tmem_holder);
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
+        for (int i = 0; i < 8; ++i) ptx::mbar_init(smem_base + sm.acc_full + 8 * i, 1);
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(smem_base + sm.acc_full[s], 1);
-            ptx::mbar_init(smem_base + sm.codes_full[s], kTile);
+            ptx::mbar_init(smem_base + sm.acc_last + 8 * s, 1);
+            ptx::mbar_init(smem_base + sm.codes_full + 8 * s, C::SLOT_THREADS);
+            ptx::mbar_init(smem_base + sm.slot_sync + 8 * s, C::SLOT_THREADS);
         }
         ptx::mbar_init(smem_base + sm.last_full, 1);
         ptx::mbar_init(smem_base + sm.drain, 1);
@@ -528,13 +654,32 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
         ptx::tmem_alloc(smem_base + sm.tmem_holder, 512);
         ptx::tmem_relinquish();
     }
+    // per-layer epilogue constants -> shared memory
+    {
+        uint32_t *dst = reinterpret_cast<uint32_t *>(smem_gen + sm.consts);
+        for (int l = 0; l < p.L - 1; ++l) {
+            const FusedLayer &ly = p.layer[l];
+            uint32_t *d = dst + ly.c_off;
+            const bool fixed = ly.epi_mode == EPI_SINE_FIXED;
+            const uint32_t *srcA = fixed ? ly.fxP : reinterpret_cast<const uint32_t *>(ly.cA);
+            const uint32_t *srcB = fixed ? ly.fxB : reinterpret_cast<const uint32_t *>(ly.cB);
+            const uint32_t *srcC = fixed ? ly.fxQ : reinterpret_cast<const uint32_t *>(ly.cA_lo);
+            const int areas = (l == 0) ? (fixed ? 3 : 4) : (ly.epi_mode == EPI_SINE_WIDE ? 3 : 2);
+            for (int i = threadIdx.x; i < W; i += kThreads) {
+                d[i] = __ldg(srcA + i);
+                d[W + i] = __ldg(srcB + i);
+                if (areas >= 3) d[2 * W + i] = __ldg(srcC + i);
+                if (areas >= 4) d[3 * W + i] = __ldg(ly.qw_k4m + i);
+            }
+        }
+    }
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
-    if (warp < 8) {
-        epilogue_role<W, PER_TOKEN>(p, sm, smem_base, warp >> 2, warp & 3, lane, tmem_base, abort_flag);
+    if (warp < kEpiWarps) {
+        epilogue_role<W, PER_TOKEN>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_role<W>(p, sm, smem_base, tmem_base, abort_flag);
     } else {
@@ -558,6 +703,7 @@ static fused_fn pick_kernel(int W, bool per_token)
     case 64: return per_token ? fused_kernel<64, true> : fused_kernel<64, false>;
     case 128: return per_token ? fused_kernel<128, true> : fused_kernel<128, false>;
     case 256: return per_token ? fused_kernel<256, true> : fused_kernel<256, false>;
+    case 512: return per_token ? fused_kernel<512, true> : fused_kernel<512, false>;
     }
     return nullptr;
 }
@@ -573,14 +719,23 @@ dhq_status_t fused_create(dhq_handle_s *h)
     p.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
     p.qmaxf = (float)((1 << (h->cfg.a_bits - 1)) - 1);
     p.status = h->d_status;
+    int words = 0;
     for (int l = 0; l < h->L; ++l) {
         const LayerDev &d = h->layer[l];
-        p.layer[l].qw_umma = d.qw_umma;
-        p.layer[l].qw_k4m = d.qw_k4m;
-        p.layer[l].cA = d.cA; p.layer[l].cA_lo = d.cA_lo; p.layer[l].cB = d.cB;
-        p.layer[l].act = d.act;
-        p.layer[l].epi_mode = d.epi_mode;
+        FusedLayer &f = p.layer[l];
+        f.qw_umma = d.qw_umma;
+        f.qw_k4m = d.qw_k4m;
+        f.cA = d.cA; f.cA_lo = d.cA_lo; f.cB = d.cB;
+        f.fxP = d.fxP; f.fxQ = d.fxQ; f.fxB = d.fxB;
+        f.act = d.act;
+        f.epi_mode = d.epi_mode;
+        f.c_off = words;
+        if (l < h->L - 1) {
+            int areas = (l == 0) ? (d.epi_mode == EPI_SINE_FIXED ? 3 : 4) : (d.epi_mode == EPI_SINE_WIDE ? 3 : 2);
+            words += areas * h->w;
+        }
     }
+    p.const_words = words;
     fused_fn fn = pick_kernel(h->w, p.per_token);
     if (!fn) return DHQ_ERR_UNSUPPORTED;
     int dev = 0, max_optin = 0;
@@ -588,16 +743,19 @@ dhq_status_t fused_create(dhq_handle_s *h)
         cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&fs->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return DHQ_ERR_CUDA;
-    // weight ring: as many W*W stages as fit beside the two A tiles; all hidden layers resident
-    // if they fit
-    const int hidden = h->L - 2;
-    const size_t fixed = smem_map(h->w, 0).total + 1024;
-    int stages = (int)(((size_t)max_optin - fixed) / ((size_t)h->w * h->w));
+    // weight ring: as many slab stages as fit beside the A tiles and the constants; all hidden
+    // layers resident if they fit
+    const int pieces = (h->w == 512) ? 4 : 1;
+    const int slabs = (h->L - 2) * pieces;
+    const size_t slab_bytes = (size_t)(h->w / pieces) * h->w;
+    const size_t fixed = smem_map(h->w, 0, words).total + 1024;
+    if (fixed > (size_t)max_optin) return DHQ_ERR_UNSUPPORTED;
+    int stages = (int)(((size_t)max_optin - fixed) / slab_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
-    if (hidden > 0 && stages < 1) return DHQ_ERR_UNSUPPORTED;
-    if (stages >= hidden) { p.resident = 1; p.n_stages = hidden > 0 ? hidden : 0; }
+    if (slabs > 0 && stages < 1) return DHQ_ERR_UNSUPPORTED;
+    if (stages >= slabs) { p.resident = 1; p.n_stages = slabs > 0 ? slabs : 0; }
     else { p.resident = 0; p.n_stages = stages; }
-    size_t bytes = smem_map(h->w, p.n_stages).total + 1024;
+    size_t bytes = smem_map(h->w, p.n_stages, words).total + 1024;
     if (bytes < (size_t)kMinSmem) bytes = kMinSmem;
     fs->smem_bytes = bytes;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
@@ -619,8 +777,9 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     p.coords = coords; p.out = out; p.n = n;
     p.n_tiles = (n + kTile - 1) / kTile;
     fused_fn fn = pick_kernel(h->w, p.per_token);
-    long long pairs = (p.n_tiles + 1) / 2;
-    int grid = (int)(pairs < fs->sm_count ? pairs : fs->sm_count);
+    const int slots = (h->w == 512) ? 1 : 2;
+    long long rounds_all = (p.n_tiles + slots - 1) / slots;
+    int grid = (int)(rounds_all < fs->sm_count ? rounds_all : fs->sm_count);
     fn<<<grid, kThreads, fs->smem_bytes, st>>>(p);
     h->launches++;
     return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;

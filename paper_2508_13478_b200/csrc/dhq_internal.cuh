@@ -27,6 +27,7 @@ struct LayerDev {
     float *inv_w = nullptr;    // [M]
     float *bias = nullptr;     // [M] zero padded
     float *cA = nullptr, *cA_lo = nullptr, *cB = nullptr; // [M] epilogue constants
+    uint32_t *fxP = nullptr, *fxQ = nullptr, *fxB = nullptr; // [M] fixed-point phase constants (EPI_SINE_FIXED)
     float *act = nullptr;      // [4]: frozen absmax (max taken on the bit pattern), s_x, inv, unused
 };
 
@@ -62,6 +63,7 @@ struct LayerArgs {
     int calib_only;        // 1: only take max |rotated input| into act[0] (bit pattern max)
     const uint32_t *qw_k4m;
     const float *cA, *cA_lo, *cB;
+    const uint32_t *fxP, *fxQ, *fxB;
     float *act;            // frozen absmax / s_x / inv (per-tensor mode)
     float *Y;              // [n][M] or NULL
     float *out;            // [n][d_L] or NULL (last layer)

@@ -98,7 +98,11 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
             if (tok >= a.n) continue;
             float c_hi = cA, c_lo = cAl;
             if (a.per_token) token_const(cA, cAl, s_tok[t], c_hi, c_lo);
-            float y = epilogue(a.epi_mode, (float)acc[t], c_hi, c_lo, cB);
+            float y;
+            if (a.epi_mode == EPI_SINE_FIXED)
+                y = sine_fixed((int)cs[t * K + 0], (int)cs[t * K + 1], a.fxP[m], a.fxQ[m], a.fxB[m]);
+            else
+                y = epilogue(a.epi_mode, (float)acc[t], c_hi, c_lo, cB);
             if (a.dacc) a.dacc[tok * M + m] = acc[t];
             if (a.Y) a.Y[tok * M + m] = y;
             if (a.out && m < a.d_L) a.out[tok * a.d_L + m] = y;

@@ -12,7 +12,8 @@ namespace dhq {
 enum EpiMode : int {
     EPI_LINEAR = 0,    // last layer: z = c * acc + b
     EPI_SINE_FAST = 1, // hidden layer whose phase is provably small: sin.approx(fma(acc, c, B))
-    EPI_SINE_WIDE = 2  // first layer / large phases: compensated phase and explicit 2*pi reduction
+    EPI_SINE_WIDE = 2, // large phases: compensated phase and explicit 2*pi reduction
+    EPI_SINE_FIXED = 3 // first layer with a per-tensor activation scale: phase in 32-bit fixed point
 };
 
 // Largest |omega0 z| for which EPI_SINE_FAST keeps the result within 1e-5 of an exact sine:
@@ -58,7 +59,8 @@ __device__ __forceinline__ float sin_wide(float x)
     const float inv_two_pi = 0.15915494309189535f;
     const float two_pi_hi = 6.2831854820251465f;   // fl32(2 pi)
     const float two_pi_lo = -1.7484555e-07f;       // 2 pi - fl32(2 pi)
-    float k = rintf(__fmul_rn(x, inv_two_pi));
+    // nearest integer by adding and subtracting 1.5 * 2^23 (ties to even; |x / 2 pi| < 2^22)
+    float k = __fsub_rn(__fadd_rn(__fmul_rn(x, inv_two_pi), 12582912.0f), 12582912.0f);
     float r = __fmaf_rn(k, -two_pi_hi, x);
     r = __fmaf_rn(k, -two_pi_lo, r);
     return sin_approx(r);
@@ -73,6 +75,19 @@ __device__ __forceinline__ float epilogue(int mode, float accf, float c_hi, floa
     if (mode == EPI_SINE_FAST) return sin_approx(__fmaf_rn(accf, c_hi, cb));
     if (mode == EPI_SINE_WIDE) return sin_wide(__fmaf_rn(accf, c_lo, __fmaf_rn(accf, c_hi, cb)));
     return __fmaf_rn(accf, c_hi, cb);
+}
+
+// First layer, per-tensor activation scale.  The rotated padded coordinate [x, y, 0, 0] has the
+// codes [qs, qd, qs, qd], so acc[m] = qs * u_m + qd * v_m with u_m = q_w[m][0] + q_w[m][2],
+// v_m = q_w[m][1] + q_w[m][3].  With P = frac(c u_m / 2 pi), Q = frac(c v_m / 2 pi),
+// B = frac(omega0 b_m / 2 pi) held as 32-bit binary fractions of a turn (c = omega0 s_w s_x), the
+// phase in turns is qs * P + qd * Q + B modulo 1: unsigned 32-bit arithmetic wraps exactly where
+// the sine is periodic, so no range reduction is needed and the error is that of the constants
+// (at most 127 * 2^-33 turns each) plus one int->float rounding (2^-26 turns).
+__device__ __forceinline__ float sine_fixed(int qs, int qd, uint32_t P, uint32_t Q, uint32_t B)
+{
+    uint32_t ph = (uint32_t)qs * P + ((uint32_t)qd * Q + B);
+    return sin_approx(__fmul_rn((float)(int)ph, 1.4629180792671596e-09f)); // 2 pi / 2^32
 }
 
 // Per-token activation scales: the per-channel constant cA (+ remainder cA_lo) times the

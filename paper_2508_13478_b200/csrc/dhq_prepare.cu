@@ -118,6 +118,15 @@ __global__ void finalize_kernel(LayerDev dev, int a_bits, int per_token, int sin
         dev.cA[m] = hi;
         dev.cA_lo[m] = (float)(A - (double)hi);
         dev.cB[m] = (float)(f * (double)dev.bias[m]);
+        if (dev.epi_mode == EPI_SINE_FIXED) {
+            const double inv_two_pi = 0.15915494309189533576888;
+            const int8_t *q = dev.qw + (size_t)m * 4;   // layer 1: K = 4
+            const double u = (double)((int)q[0] + (int)q[2]), v = (double)((int)q[1] + (int)q[3]);
+            auto to_fix = [](double turns) { return (uint32_t)(unsigned long long)llrint(turns * 4294967296.0); };
+            dev.fxP[m] = to_fix(A * u * inv_two_pi);
+            dev.fxQ[m] = to_fix(A * v * inv_two_pi);
+            dev.fxB[m] = to_fix(f * (double)dev.bias[m] * inv_two_pi);
+        }
     }
 }
 

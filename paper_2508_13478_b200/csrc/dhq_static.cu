@@ -60,6 +60,7 @@ extern "C" dhq_status_t dhq_forward_static_scratch(dhq_handle_t h, const float *
         a.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
         a.epi_mode = d.epi_mode;
         a.qw_k4m = d.qw_k4m; a.cA = d.cA; a.cA_lo = d.cA_lo; a.cB = d.cB; a.act = d.act;
+        a.fxP = d.fxP; a.fxQ = d.fxQ; a.fxB = d.fxB;
         a.Y = scratch + (size_t)((l - 1) & 1) * kHalf; // every row < n is written before it is read
         if (l == h->L) a.out = out;
         if (launch_layer(a, st) != cudaSuccess) return DHQ_ERR_CUDA;

@@ -66,8 +66,9 @@ def test_c2_full_grid():
     _p1(w, w.coords())
 
 
-@pytest.mark.parametrize("name,count", [("C3", 20000 + 77), ("C4-W4A4", 12000 + 1), ("C4-W6A6", 12000 + 1)])
-def test_c3_c4_sampled_tokens(name, count):
+@pytest.mark.parametrize("name,count", [("C3", 20000 + 77), ("C4-W4A4", 12000 + 1), ("C4-W6A6", 12000 + 1),
+                                        ("C5", 6000 + 13)])
+def test_c3_c4_c5_sampled_tokens(name, count):
     w = dhq_inputs.WORKLOADS[name]
     coords = w.coords()
     idx = np.linspace(0, coords.shape[0] - 1, count).astype(np.int64)
@@ -85,6 +86,14 @@ def test_ragged_tails_small_width(n):
 def test_granularity_and_bit_width_combinations(w_gran, a_gran, bits):
     wl = dhq_inputs.Workload("combo", (2, 128, 128, 128, 3), 30.0, 40 + bits, bits, bits, w_gran, a_gran, (40, 41))
     _p1(wl, wl.coords())
+
+
+@pytest.mark.parametrize("width,a_gran", [(64, 1), (256, 0), (512, 1), (512, 0)])
+def test_every_width_with_ragged_tail_and_several_rounds(width, a_gran):
+    # more tiles than one round of the persistent grid holds at width 512, plus a ragged tail
+    wl = dhq_inputs.Workload("w", (2, width, width, width, 3), 30.0, width + a_gran, 8, 8, 1 - a_gran, a_gran, (8, 8))
+    coords = dhq_inputs.grid_coords(150, 131)[: 148 * 128 + 300 if width == 512 else 3000]
+    _p1(wl, coords)
 
 
 def test_trained_like_weights_and_wide_phases():
