@@ -127,43 +127,28 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
     return m;
 }
 
-// Bounded wait.  Returns false when the wait ran out or another role already gave up.
+// Bounded wait.  Returns false when the wait ran out or another role already gave up.  Each
+// try may suspend the thread in hardware for up to kSuspendNs, so a waiting warp issues only a
+// handful of instructions per try.
+constexpr uint32_t kSuspendNs = 20000;
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = ptx::globaltimer();
-    for (uint32_t spin = 1;; ++spin) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((spin & 0xff) == 0) {
-            if (*abort_flag) return false;
-            if (ptx::globaltimer() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicExch(status, 1);
-                return false;
-            }
+    while (!ptx::mbar_try_wait_hint(bar, parity, kSuspendNs)) {
+        if (*abort_flag) return false;
+        if (ptx::globaltimer() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicExch(status, 1);
+            return false;
         }
     }
+    return true;
 }
 // The same for a whole warp: every lane takes the same decision.
 __device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
     return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_flag, status));
-}
-
-// In-register butterfly stages with strides 1 .. N/2 on N values: pair (i, i+h) -> (a+b, a-b).
-template <int N> __device__ __forceinline__ void fwht_local(float (&f)[N])
-{
-#pragma unroll
-    for (int h = 1; h < N; h <<= 1) {
-#pragma unroll
-        for (int i = 0; i < N; ++i) {
-            if ((i & h) == 0) {
-                float a = f[i], b = f[i + h];
-                f[i] = __fadd_rn(a, b);
-                f[i + h] = __fsub_rn(a, b);
-            }
-        }
-    }
 }
 
 // Round-half-even to an integer code held in the low byte: (clamp,) then add 1.5 * 2^23 (the
@@ -173,7 +158,7 @@ template <int N> __device__ __forceinline__ void fwht_local(float (&f)[N])
 template <bool CLAMP> __device__ __forceinline__ uint32_t code_bits(float v, float inv, float qmaxf)
 {
     float t = __fmul_rn(v, inv);
-    if (CLAMP) t = fmaxf(fminf(t, qmaxf), -qmaxf);
+    if (CLAMP) asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(t) : "f"(qmaxf)); // sign(t) * min(|t|, qmax)
     return __float_as_uint(__fadd_rn(t, 12582912.0f));
 }
 __device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3)
@@ -223,14 +208,58 @@ __device__ __forceinline__ float4 lds128(uint32_t addr)
     return v;
 }
 
-// Dequantize + bias + sine of CH consecutive channels starting at m0, in place: v holds the
-// int32 accumulators on entry and the fp32 activations (as bits) on exit.  Constants come from
-// shared memory: area A = cA, B = cB, C = cA_lo, each W words.
-template <int W, int CH, bool PER_TOKEN, int MODE>
-__device__ __forceinline__ void epilogue_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH])
+// One butterfly: (a, b) -> (a + b, a - b).
+__device__ __forceinline__ void bfly(float &a, float &b)
 {
+    const float x = a, y = b;
+    a = __fadd_rn(x, y);
+    b = __fsub_rn(x, y);
+}
+
+// Pass 1 of one chunk, in place: v holds CH int32 accumulators (or nothing, for layer 1) on entry
+// and, on exit, the fp32 activations after the butterfly stages with strides 1 .. CH/2.
+// `sine4(j, out)` produces the four activations 4j .. 4j+3.  The work is ordered as a software
+// pipeline - the sines of group j+1 are issued before the stride-1/2 butterflies of group j, the
+// stride-4/8 butterflies follow every fourth group - so that the special-function unit (one sine
+// per 8 issue cycles and scheduler) is fed evenly instead of in one burst per chunk.  Each
+// element still goes through the stages in the order 1, 2, 4, ...: the sums are unchanged.
+template <int CH, class Sine4> __device__ __forceinline__ void chunk_pipeline(uint32_t (&v)[CH], Sine4 sine4)
+{
+    float f[CH];
+    sine4(0, &f[0]);
 #pragma unroll
     for (int j = 0; j < CH / 4; ++j) {
+        if (j + 1 < CH / 4) sine4(j + 1, &f[4 * (j + 1)]);
+        bfly(f[4 * j], f[4 * j + 1]);
+        bfly(f[4 * j + 2], f[4 * j + 3]);
+        bfly(f[4 * j], f[4 * j + 2]);
+        bfly(f[4 * j + 1], f[4 * j + 3]);
+        if ((j & 3) == 3) {
+            const int base = 4 * (j - 3);
+#pragma unroll
+            for (int h = 4; h <= 8; h <<= 1) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if ((i & h) == 0) bfly(f[base + i], f[base + i + h]);
+            }
+        }
+    }
+#pragma unroll
+    for (int h = 16; h < CH; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < CH; ++i)
+            if ((i & h) == 0) bfly(f[i], f[i + h]);
+    }
+#pragma unroll
+    for (int i = 0; i < CH; ++i) v[i] = __float_as_uint(f[i]);
+}
+
+// Hidden layer: dequantize + bias + sine of the CH channels starting at m0.  Constants come
+// from shared memory: area A = cA, B = cB, C = cA_lo, each W words.
+template <int W, int CH, bool PER_TOKEN, int MODE>
+__device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH])
+{
+    chunk_pipeline<CH>(v, [&](int j, float *out) {
         const float4 a = lds128(cbase + (m0 + 4 * j) * 4);
         const float4 b = lds128(cbase + (W + m0 + 4 * j) * 4);
         float4 lo = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -240,9 +269,9 @@ __device__ __forceinline__ void epilogue_chunk(uint32_t cbase, int m0, float s_x
         for (int e = 0; e < 4; ++e) {
             float c_hi = av[e], c_lo = lv[e];
             if (PER_TOKEN) token_const(av[e], lv[e], s_x, c_hi, c_lo);
-            v[4 * j + e] = __float_as_uint(epilogue(MODE, (float)(int)v[4 * j + e], c_hi, c_lo, bv[e]));
+            out[e] = epilogue(MODE, (float)(int)v[4 * j + e], c_hi, c_lo, bv[e]);
         }
-    }
+    });
 }
 
 // Layer 1 for CH channels starting at m0.  Fixed-point mode: areas A = P, B = B, C = Q.
@@ -251,38 +280,27 @@ __device__ __forceinline__ void epilogue_chunk(uint32_t cbase, int m0, float s_x
 template <int W, int CH, bool PER_TOKEN>
 __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int qd, uint32_t qx, float s_x, uint32_t (&v)[CH])
 {
-    if constexpr (!PER_TOKEN) {
-#pragma unroll
-        for (int j = 0; j < CH / 4; ++j) {
-            const float4 P = lds128(cbase + (m0 + 4 * j) * 4);
-            const float4 B = lds128(cbase + (W + m0 + 4 * j) * 4);
-            const float4 Q = lds128(cbase + (2 * W + m0 + 4 * j) * 4);
-            const float Pv[4] = {P.x, P.y, P.z, P.w}, Bv[4] = {B.x, B.y, B.z, B.w}, Qv[4] = {Q.x, Q.y, Q.z, Q.w};
+    chunk_pipeline<CH>(v, [&](int j, float *out) {
+        const float4 A = lds128(cbase + (m0 + 4 * j) * 4);
+        const float4 B = lds128(cbase + (W + m0 + 4 * j) * 4);
+        const float4 Cc = lds128(cbase + (2 * W + m0 + 4 * j) * 4);
+        const float Av[4] = {A.x, A.y, A.z, A.w}, Bv[4] = {B.x, B.y, B.z, B.w}, Cv[4] = {Cc.x, Cc.y, Cc.z, Cc.w};
+        if constexpr (!PER_TOKEN) {
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                v[4 * j + e] = __float_as_uint(sine_fixed(qs, qd, __float_as_uint(Pv[e]), __float_as_uint(Qv[e]), __float_as_uint(Bv[e])));
-        }
-    } else {
-#pragma unroll
-        for (int j = 0; j < CH / 4; ++j) {
+                out[e] = sine_fixed(qs, qd, __float_as_uint(Av[e]), __float_as_uint(Cv[e]), __float_as_uint(Bv[e]));
+        } else {
             const float4 wq = lds128(cbase + (3 * W + m0 + 4 * j) * 4);
-            v[4 * j + 0] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.x), 0);
-            v[4 * j + 1] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.y), 0);
-            v[4 * j + 2] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.z), 0);
-            v[4 * j + 3] = (uint32_t)__dp4a((int)qx, (int)__float_as_uint(wq.w), 0);
+            const float wv[4] = {wq.x, wq.y, wq.z, wq.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float c_hi, c_lo;
+                token_const(Av[e], Cv[e], s_x, c_hi, c_lo);
+                const int acc = __dp4a((int)qx, (int)__float_as_uint(wv[e]), 0);
+                out[e] = epilogue(EPI_SINE_WIDE, (float)acc, c_hi, c_lo, Bv[e]);
+            }
         }
-        epilogue_chunk<W, CH, true, EPI_SINE_WIDE>(cbase, m0, s_x, v);
-    }
-}
-
-template <int CH> __device__ __forceinline__ void fwht_chunk(uint32_t (&v)[CH])
-{
-    float f[CH];
-#pragma unroll
-    for (int i = 0; i < CH; ++i) f[i] = __uint_as_float(v[i]);
-    fwht_local<CH>(f);
-#pragma unroll
-    for (int i = 0; i < CH; ++i) v[i] = __float_as_uint(f[i]);
+    });
 }
 
 // Everything a slot's threads need to finish a layer once their chunks are back in tensor memory.
@@ -461,7 +479,6 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
             const int ch = sub * C::CPT + cc;
             uint32_t v[CH];
             layer1_chunk<W, CH, PER_TOKEN>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v);
-            fwht_chunk<CH>(v);
             tmem_st<CH>(c.taddr + ch * CH, v);
         }
         if (!finish_layer<W, PER_TOKEN>(c, next_s, next_inv, s_x)) return;
@@ -484,9 +501,8 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
                 uint32_t v[CH];
                 tmem_ld<CH>(c.taddr + ch * CH, v);
                 ptx::tmem_wait_ld();
-                if (fast) epilogue_chunk<W, CH, PER_TOKEN, EPI_SINE_FAST>(cbase, ch * CH, s_x, v);
-                else epilogue_chunk<W, CH, PER_TOKEN, EPI_SINE_WIDE>(cbase, ch * CH, s_x, v);
-                fwht_chunk<CH>(v);
+                if (fast) hidden_chunk<W, CH, PER_TOKEN, EPI_SINE_FAST>(cbase, ch * CH, s_x, v);
+                else hidden_chunk<W, CH, PER_TOKEN, EPI_SINE_WIDE>(cbase, ch * CH, s_x, v);
                 tmem_st<CH>(c.taddr + ch * CH, v);
             }
             if (!finish_layer<W, PER_TOKEN>(c, next_s, next_inv, s_x)) return;
