@@ -17,7 +17,7 @@
 // Per layer and tile:
 //   pass 1  each thread takes its chunks of 64 columns: acc (TMEM, int32) -> dequantize, bias,
 //           sine (dhq_math.cuh) -> butterfly stages with stride < 64 in registers -> fp32 back to
-//           the same TMEM columns.                                   [slot-wide mbarrier]
+//           the same TMEM columns.          [mbarrier of the R warps that share the 32 rows]
 //   pass 2  each thread takes its groups: one value from every chunk at G consecutive positions
 //           -> the remaining butterfly stages (stride 64, 128, ...) -> quantize, pack, st.shared
 //           into the next layer's A operand tile -> mbarrier -> next MMA.
@@ -94,7 +94,7 @@ struct SmemMap {
     uint32_t acc_full;   // [2 slots][4 pieces]
     uint32_t acc_last;   // [2]
     uint32_t codes_full; // [2]
-    uint32_t slot_sync;  // [2]
+    uint32_t slot_sync;  // [2 slots][4 lane quadrants]
     uint32_t last_full, drain;
     uint32_t w_full, w_empty; // [kMaxStages] each
     uint32_t tmem_holder, abort_flag;
@@ -116,7 +116,7 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
     m.acc_full = off; off += 8 * 8;
     m.acc_last = off; off += 8 * 2;
     m.codes_full = off; off += 8 * 2;
-    m.slot_sync = off; off += 8 * 2;
+    m.slot_sync = off; off += 8 * 8;
     m.last_full = off; off += 8;
     m.drain = off; off += 8;
     m.w_full = off; off += 8 * kMaxStages;
@@ -127,28 +127,33 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
     return m;
 }
 
-// Bounded wait.  Returns false when the wait ran out or another role already gave up.  Each
-// try may suspend the thread in hardware for up to kSuspendNs, so a waiting warp issues only a
-// handful of instructions per try.
-constexpr uint32_t kSuspendNs = 20000;
+// Bounded wait.  Returns false when the wait ran out or another role already gave up.  Between
+// tries the thread sleeps, so that a waiting warp leaves the issue slots to the working ones;
+// the time limit and the abort flag are looked at every 64 tries.
+template <int SLEEP_NS>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = ptx::globaltimer();
-    while (!ptx::mbar_try_wait_hint(bar, parity, kSuspendNs)) {
-        if (*abort_flag) return false;
-        if (ptx::globaltimer() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
-            atomicExch(status, 1);
-            return false;
+    unsigned long long t0 = 0;
+    for (uint32_t tries = 1;; ++tries) {
+        __nanosleep(SLEEP_NS);
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((tries & 63) == 0) {
+            if (*abort_flag) return false;
+            const unsigned long long now = ptx::globaltimer();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, 1);
+                return false;
+            }
         }
     }
-    return true;
 }
 // The same for a whole warp: every lane takes the same decision.
 __device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
-    return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_flag, status));
+    return __all_sync(0xffffffffu, wait_bar<32>(bar, parity, abort_flag, status));
 }
 
 // Round-half-even to an integer code held in the low byte: (clamp,) then add 1.5 * 2^23 (the
@@ -307,7 +312,7 @@ __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int
 struct SlotCtx {
     uint32_t taddr;      // TMEM address of this thread's lane, column 0 of the slot
     uint32_t a_tile;     // shared-memory address of the slot's A operand tile
-    uint32_t bar_sync;   // slot-wide mbarrier
+    uint32_t bar_sync;   // mbarrier of the R warps that share this thread's 32 rows
     uint32_t bar_codes;  // "codes ready" mbarrier
     uint32_t amax_addr;  // shared memory: [R][128] floats for this slot
     uint32_t sync_parity;
@@ -430,7 +435,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     c.sub = sub;
     c.taddr = tmem_base + (uint32_t)(slot * C::TMEM_COLS_PER_SLOT) + ((uint32_t)(quad * 32) << 16);
     c.a_tile = smem_base + sm.a_tile[slot];
-    c.bar_sync = smem_base + sm.slot_sync + 8 * slot;
+    c.bar_sync = smem_base + sm.slot_sync + 8 * (slot * 4 + quad);
     c.bar_codes = smem_base + sm.codes_full + 8 * slot;
     c.amax_addr = smem_base + sm.amax + slot * (4 * kTile * 4);
     c.sync_parity = 0;
@@ -555,19 +560,19 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
                     const int slab_id = (l - 2) * C::PIECES + pc;
                     stage = p.resident ? slab_id : (int)(use % p.n_stages);
                     const uint32_t par = p.resident ? 0u : (uint32_t)((use / p.n_stages) & 1);
-                    if (!wait_bar(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
+                    if (!wait_bar<100>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
                     b_addr = smem_base + sm.ring + (uint32_t)stage * slab;
                     n_rows = C::PW;
                     idesc = idesc_hidden;
                 } else {
-                    if (!wait_bar(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
+                    if (!wait_bar<100>(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
                     b_addr = smem_base + sm.last_w;
                     n_rows = 16;
                     idesc = idesc_last;
                 }
                 for (int s = 0; s < active; ++s) {
                     if (pc == 0) {
-                        if (!wait_bar(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
+                        if (!wait_bar<100>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
                         codes_parity[s] ^= 1;
                         ptx::tc_fence_after();
                     }
@@ -617,7 +622,7 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
         const int stage = (int)(i % p.n_stages);
         if (i >= p.n_stages) {
             uint32_t par = (uint32_t)(((i / p.n_stages) - 1) & 1);
-            if (!wait_bar(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
+            if (!wait_bar<100>(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
         }
         const int id = (int)(i % slabs);
         const int l = 2 + id / C::PIECES, pc = id % C::PIECES;
@@ -656,7 +661,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(smem_base + sm.acc_last + 8 * s, 1);
             ptx::mbar_init(smem_base + sm.codes_full + 8 * s, C::SLOT_THREADS);
-            ptx::mbar_init(smem_base + sm.slot_sync + 8 * s, C::SLOT_THREADS);
+            for (int q = 0; q < 4; ++q) ptx::mbar_init(smem_base + sm.slot_sync + 8 * (s * 4 + q), C::R * 32);
         }
         ptx::mbar_init(smem_base + sm.last_full, 1);
         ptx::mbar_init(smem_base + sm.drain, 1);
