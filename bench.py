@@ -145,6 +145,21 @@ def run_reference(args, workload):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of per-rank timings (the slowest rank defines the step time)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_throughput(coords_per_rank, world, ms_per_step):
+    """Whole-job coordinates per second: every rank runs its own replica of the grid."""
+    return coords_per_rank * world / (ms_per_step * 1e-3)
+
+
 def run_ours(args, workload):
     import torch
     import torch.distributed as dist
@@ -205,13 +220,10 @@ def run_ours(args, workload):
     e2e_ms = timed(lambda: dhq.dhq_forward_host(h, coords_host, out_host), args.steps)
     status = dhq.dhq_last_status(h)
 
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, "cuda")
     ms_per_step = total_ms / args.steps
-    value = n * world / (ms_per_step * 1e-3)
-    e2e_value = n * world / (e2e_ms / args.steps * 1e-3)
+    value = aggregate_throughput(n, world, ms_per_step)
+    e2e_value = aggregate_throughput(n, world, e2e_ms / args.steps)
 
     if rank == 0:
         peaks = {}
