@@ -27,7 +27,9 @@ typedef enum {
     DHQ_PIPE_F2I = 4,      /* cvt.rni.s32.f32                                      */
     DHQ_PIPE_PRMT = 5,     /* byte permute                                         */
     DHQ_PIPE_FMNMX = 6,    /* fp32 min/max                                         */
-    DHQ_PIPE_TENSOR_I8 = 7 /* tcgen05.mma kind::i8, 128x256x32, operands resident in shared memory */
+    DHQ_PIPE_TENSOR_I8 = 7, /* tcgen05.mma kind::i8, 128x256x32, operands resident in shared memory */
+    DHQ_PIPE_FADD2 = 8,    /* add.rn.f32x2: two fp32 adds per lane and instruction (counted as 2)   */
+    DHQ_PIPE_FFMA2 = 9     /* fma.rn.f32x2 (counted as 2)                                            */
 } dhq_pipe_t;
 
 /*

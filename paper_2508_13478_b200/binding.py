@@ -23,7 +23,7 @@ DHQ_ROT_BOTH = 1
 DHQ_ROT_NONE = 2
 DHQ_STATIC_MAX_TOKENS = 4096
 
-PIPES = {"ffma": 0, "fadd": 1, "mufu_sin": 2, "i2f": 3, "f2i": 4, "prmt": 5, "fmnmx": 6, "tensor_i8": 7}
+PIPES = {"ffma": 0, "fadd": 1, "mufu_sin": 2, "i2f": 3, "f2i": 4, "prmt": 5, "fmnmx": 6, "tensor_i8": 7, "fadd2": 8, "ffma2": 9}
 
 
 class DhqError(RuntimeError):
@@ -167,10 +167,15 @@ def dhq_forward_debug(handle, coords, out=None, bufs=None, stream=None):
     st = _DebugBufs()
     keep = []
     if bufs:
+        n_layers = 0
+        while n_layers < 16 and load_library().dhq_layer_dims(handle, n_layers + 1, None, None) == 0:
+            n_layers += 1
         for key, dt in dtypes.items():
             lst = bufs.get(key)
             if lst is None:
                 continue
+            if len(lst) != n_layers:       # the library indexes these arrays by layer: never pass a short one
+                raise ValueError(f"dhq_forward_debug: bufs[{key!r}] needs {n_layers} entries (one per layer)")
             arr = (ctypes.c_void_p * len(lst))(*[_dev_ptr(t, dt, key) for t in lst])
             keep.append(arr)
             setattr(st, key, arr)

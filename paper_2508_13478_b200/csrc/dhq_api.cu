@@ -178,6 +178,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             a.bits = cfg->w_bits;
             a.per_channel = cfg->w_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
             a.sine = l < L; a.first = l == 1;
+            a.permute_rows = (l > 1 && l < L) ? 1 : 0;
             a.omega0 = (double)cfg->omega0;
             a.dev = d;
             a.phase_bound = d_bounds + (l - 1);

@@ -48,7 +48,7 @@ constexpr int kMinSmem = 120 * 1024; // more than half an SM's shared memory: on
 template <int W> struct Cfg {
     static constexpr int SLOTS = (W == 512) ? 1 : 2;
     static constexpr int R = kEpiWarps / (4 * SLOTS);          // threads per row: 2 or 4
-    static constexpr int CH = (W / R < 64) ? W / R : 64;       // columns per register chunk
+    static constexpr int CH = (W == 64) ? 32 : 64;             // columns per register chunk (= fused_chunk(W))
     static constexpr int NCH = W / CH;                         // chunks per row
     static constexpr int CPT = NCH / R;                        // chunks per thread
     static constexpr int G = (64 / NCH < CH / R) ? 64 / NCH : CH / R; // positions per pass-2 group
@@ -156,14 +156,61 @@ __device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, vol
     return __all_sync(0xffffffffu, wait_bar<32>(bar, parity, abort_flag, status));
 }
 
-// Round-half-even to an integer code held in the low byte: (clamp,) then add 1.5 * 2^23 (the
-// sum rounds to the integer grid, ties to even, and its low mantissa bits are the two's
-// complement code).  Same integer as __float2int_rn(clamp(v * inv)).  With a per-token scale
-// |v * inv| <= qmax (1 + 2^-23) already, so the clamp is skipped.
+// Two fp32 values in one 64-bit register pair, and the packed sm_100 arithmetic on them: one
+// instruction, two IEEE round-to-nearest results (the same bits as two scalar operations).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f32x2 pack2u(uint32_t lo, uint32_t hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ void unpack2u(f32x2 v, uint32_t &lo, uint32_t &hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+// One butterfly on two independent pairs at once: (a, b) -> (a + b, a - b).
+__device__ __forceinline__ void bfly2(f32x2 &a, f32x2 &b)
+{
+    const f32x2 x = a, y = b;
+    a = add2(x, y);
+    b = sub2(x, y);
+}
+
+// Round-half-even of two values to integer codes held in the low bytes: multiply by inv,
+// (clamp,) add 1.5 * 2^23 - the sum rounds to the integer grid, ties to even, and its low
+// mantissa bits are the two's complement code.  Same integers as
+// __float2int_rn(clamp(v * inv, -qmax, qmax)).  With a per-token scale |v * inv| <= qmax
+// (1 + 2^-23) already, so the clamp is skipped.  The clamp is sign(t) * min(|t|, qmax).
+template <bool CLAMP> __device__ __forceinline__ void code_bits2(f32x2 v, f32x2 inv2, float qmaxf, uint32_t &b0, uint32_t &b1)
+{
+    f32x2 t = mul2(v, inv2);
+    float lo, hi;
+    unpack2(t, lo, hi);
+    if (CLAMP) {
+        asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(lo) : "f"(qmaxf));
+        asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(hi) : "f"(qmaxf));
+        unpack2u(add2(pack2(lo, hi), pack2(12582912.0f, 12582912.0f)), b0, b1);
+    } else {
+        // Scalar adds here: a packed multiply directly followed by a packed add was observed to be
+        // merged into one fused multiply-add by the assembler, which rounds v * inv only once and
+        // turns exact ties (x.5) the wrong way.  The product must be rounded to fp32 first.
+        b0 = __float_as_uint(__fadd_rn(lo, 12582912.0f));
+        b1 = __float_as_uint(__fadd_rn(hi, 12582912.0f));
+    }
+}
 template <bool CLAMP> __device__ __forceinline__ uint32_t code_bits(float v, float inv, float qmaxf)
 {
     float t = __fmul_rn(v, inv);
-    if (CLAMP) asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(t) : "f"(qmaxf)); // sign(t) * min(|t|, qmax)
+    if (CLAMP) asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(t) : "f"(qmaxf));
     return __float_as_uint(__fadd_rn(t, 12582912.0f));
 }
 __device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3)
@@ -172,23 +219,35 @@ __device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2,
     uint32_t hi = __byte_perm(b2, b3, 0x0040);
     return __byte_perm(lo, hi, 0x5410);
 }
-// Quantize N (8 or 16) consecutive-k values of this thread's token, k0 a multiple of N, and store
-// them into the A operand tile: byte offset (k/16) * 2048 + row * 16 + k % 16.
-template <int N, bool CLAMP>
-__device__ __forceinline__ void store_codes(uint32_t a_tile, int row, int k0, const uint32_t *v, float inv, float qmaxf)
+// Store N (4, 8 or 16) consecutive-k codes of this thread's token, k0 a multiple of N, into the A
+// operand tile: byte offset (k/16) * 2048 + row * 16 + k % 16.  w holds N/4 packed words.
+template <int N> __device__ __forceinline__ void store_code_words(uint32_t a_tile, int row, int k0, const uint32_t *w)
 {
-    uint32_t w[N / 4];
-#pragma unroll
-    for (int j = 0; j < N / 4; ++j)
-        w[j] = pack4(code_bits<CLAMP>(__uint_as_float(v[4 * j]), inv, qmaxf),
-                     code_bits<CLAMP>(__uint_as_float(v[4 * j + 1]), inv, qmaxf),
-                     code_bits<CLAMP>(__uint_as_float(v[4 * j + 2]), inv, qmaxf),
-                     code_bits<CLAMP>(__uint_as_float(v[4 * j + 3]), inv, qmaxf));
     const uint32_t addr = a_tile + (k0 >> 4) * 2048 + row * 16 + (k0 & 15);
     if constexpr (N == 16)
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-    else
+    else if constexpr (N == 8)
         asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(w[0]), "r"(w[1]) : "memory");
+    else
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(w[0]) : "memory");
+}
+// Quantize G consecutive tensor-memory columns of chunk `ch` starting at column position p0 (even
+// positions hold features p0/2 + k, odd positions features CH/2 + p0/2 + k) and store the codes.
+template <int G, int CH, bool CLAMP>
+__device__ __forceinline__ void quantize_store(uint32_t a_tile, int row, int ch, int p0, const uint32_t *u, float inv, float qmaxf)
+{
+    const f32x2 inv2 = pack2(inv, inv);
+    uint32_t even[G / 2], odd[G / 2];
+#pragma unroll
+    for (int k = 0; k < G / 2; ++k) code_bits2<CLAMP>(pack2u(u[2 * k], u[2 * k + 1]), inv2, qmaxf, even[k], odd[k]);
+    uint32_t we[G / 8], wo[G / 8];
+#pragma unroll
+    for (int j = 0; j < G / 8; ++j) {
+        we[j] = pack4(even[4 * j], even[4 * j + 1], even[4 * j + 2], even[4 * j + 3]);
+        wo[j] = pack4(odd[4 * j], odd[4 * j + 1], odd[4 * j + 2], odd[4 * j + 3]);
+    }
+    store_code_words<G / 2>(a_tile, row, ch * CH + p0 / 2, we);
+    store_code_words<G / 2>(a_tile, row, ch * CH + CH / 2 + p0 / 2, wo);
 }
 
 template <int N> __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[N])
@@ -213,97 +272,121 @@ __device__ __forceinline__ float4 lds128(uint32_t addr)
     return v;
 }
 
-// One butterfly: (a, b) -> (a + b, a - b).
-__device__ __forceinline__ void bfly(float &a, float &b)
-{
-    const float x = a, y = b;
-    a = __fadd_rn(x, y);
-    b = __fsub_rn(x, y);
-}
-
 // Pass 1 of one chunk, in place: v holds CH int32 accumulators (or nothing, for layer 1) on entry
 // and, on exit, the fp32 activations after the butterfly stages with strides 1 .. CH/2.
-// `sine4(j, out)` produces the four activations 4j .. 4j+3.  The work is ordered as a software
-// pipeline - the sines of group j+1 are issued before the stride-1/2 butterflies of group j, the
-// stride-4/8 butterflies follow every fourth group - so that the special-function unit (one sine
-// per 8 issue cycles and scheduler) is fed evenly instead of in one burst per chunk.  Each
-// element still goes through the stages in the order 1, 2, 4, ...: the sums are unchanged.
-template <int CH, class Sine4> __device__ __forceinline__ void chunk_pipeline(uint32_t (&v)[CH], Sine4 sine4)
+// Tensor-memory column 2i of the chunk is feature i, column 2i+1 feature i + CH/2, so the
+// register pair (v[2i], v[2i+1]) goes through the stages with strides 1 .. CH/4 as one packed
+// value; the stride-CH/2 stage is the butterfly between its two halves.
+// `sine8(j, out)` produces the four pairs 4j .. 4j+3.  The work is ordered as a software pipeline -
+// the sines of group j+1 are issued before the stride-1/2 butterflies of group j, the stride-4/8
+// butterflies follow every fourth group - so that the special-function unit (one sine per 8 issue
+// cycles and scheduler) is fed evenly instead of in one burst per chunk.  Each element still goes
+// through the stages in the order 1, 2, 4, ...: the sums are unchanged.
+template <int CH, class Sine8> __device__ __forceinline__ void chunk_pipeline(uint32_t (&v)[CH], Sine8 sine8)
 {
-    float f[CH];
-    sine4(0, &f[0]);
+    constexpr int NP = CH / 2;
+    f32x2 P[NP];
+    sine8(0, &P[0]);
 #pragma unroll
-    for (int j = 0; j < CH / 4; ++j) {
-        if (j + 1 < CH / 4) sine4(j + 1, &f[4 * (j + 1)]);
-        bfly(f[4 * j], f[4 * j + 1]);
-        bfly(f[4 * j + 2], f[4 * j + 3]);
-        bfly(f[4 * j], f[4 * j + 2]);
-        bfly(f[4 * j + 1], f[4 * j + 3]);
+    for (int j = 0; j < NP / 4; ++j) {
+        if (j + 1 < NP / 4) sine8(j + 1, &P[4 * (j + 1)]);
+        bfly2(P[4 * j], P[4 * j + 1]);
+        bfly2(P[4 * j + 2], P[4 * j + 3]);
+        bfly2(P[4 * j], P[4 * j + 2]);
+        bfly2(P[4 * j + 1], P[4 * j + 3]);
         if ((j & 3) == 3) {
             const int base = 4 * (j - 3);
 #pragma unroll
             for (int h = 4; h <= 8; h <<= 1) {
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    if ((i & h) == 0) bfly(f[base + i], f[base + i + h]);
+                    if ((i & h) == 0) bfly2(P[base + i], P[base + i + h]);
             }
         }
     }
 #pragma unroll
-    for (int h = 16; h < CH; h <<= 1) {
+    for (int h = 16; h < NP; h <<= 1) {
 #pragma unroll
-        for (int i = 0; i < CH; ++i)
-            if ((i & h) == 0) bfly(f[i], f[i + h]);
+        for (int i = 0; i < NP; ++i)
+            if ((i & h) == 0) bfly2(P[i], P[i + h]);
     }
 #pragma unroll
-    for (int i = 0; i < CH; ++i) v[i] = __float_as_uint(f[i]);
+    for (int i = 0; i < NP; ++i) {
+        float a, b;
+        unpack2(P[i], a, b);
+        v[2 * i] = __float_as_uint(__fadd_rn(a, b));
+        v[2 * i + 1] = __float_as_uint(__fsub_rn(a, b));
+    }
 }
 
-// Hidden layer: dequantize + bias + sine of the CH channels starting at m0.  Constants come
-// from shared memory: area A = cA, B = cB, C = cA_lo, each W words.
+// Hidden layer: dequantize + bias + sine of the CH columns starting at column m0.  Constants come
+// from shared memory in column order: area A = cA, B = cB, C = cA_lo, each W words.
 template <int W, int CH, bool PER_TOKEN, int MODE>
 __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH])
 {
-    chunk_pipeline<CH>(v, [&](int j, float *out) {
-        const float4 a = lds128(cbase + (m0 + 4 * j) * 4);
-        const float4 b = lds128(cbase + (W + m0 + 4 * j) * 4);
-        float4 lo = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (MODE == EPI_SINE_WIDE) lo = lds128(cbase + (2 * W + m0 + 4 * j) * 4);
-        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w}, lv[4] = {lo.x, lo.y, lo.z, lo.w};
+    chunk_pipeline<CH>(v, [&](int j, f32x2 *out) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            float c_hi = av[e], c_lo = lv[e];
-            if (PER_TOKEN) token_const(av[e], lv[e], s_x, c_hi, c_lo);
-            out[e] = epilogue(MODE, (float)(int)v[4 * j + e], c_hi, c_lo, bv[e]);
+        for (int q = 0; q < 2; ++q) {
+            const int i = 8 * j + 4 * q; // four columns = two pairs
+            const float4 a = lds128(cbase + (m0 + i) * 4);
+            const float4 b = lds128(cbase + (W + m0 + i) * 4);
+            if (MODE == EPI_SINE_FAST && !PER_TOKEN) {
+                // x = fma(acc, cA, cB) for two columns at once, then the sine of each
+                float x0, x1, x2, x3;
+                unpack2(fma2(pack2((float)(int)v[i], (float)(int)v[i + 1]), pack2(a.x, a.y), pack2(b.x, b.y)), x0, x1);
+                unpack2(fma2(pack2((float)(int)v[i + 2], (float)(int)v[i + 3]), pack2(a.z, a.w), pack2(b.z, b.w)), x2, x3);
+                out[2 * q] = pack2(sin_approx(x0), sin_approx(x1));
+                out[2 * q + 1] = pack2(sin_approx(x2), sin_approx(x3));
+            } else {
+                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (MODE == EPI_SINE_WIDE) lo = lds128(cbase + (2 * W + m0 + i) * 4);
+                const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w}, lv[4] = {lo.x, lo.y, lo.z, lo.w};
+                float y[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float c_hi = av[e], c_lo = lv[e];
+                    if (PER_TOKEN) token_const(av[e], lv[e], s_x, c_hi, c_lo);
+                    y[e] = epilogue(MODE, (float)(int)v[i + e], c_hi, c_lo, bv[e]);
+                }
+                out[2 * q] = pack2(y[0], y[1]);
+                out[2 * q + 1] = pack2(y[2], y[3]);
+            }
         }
     });
 }
 
-// Layer 1 for CH channels starting at m0.  Fixed-point mode: areas A = P, B = B, C = Q.
+// Layer 1 for the CH columns starting at column m0.  Fixed-point mode: areas A = P, B = B, C = Q.
 // Float mode (per-token scales): A = cA, B = cB, C = cA_lo, D = the weight codes, one word per
-// channel, and acc = dp4a(codes of the token, codes of the channel).
+// column, and acc = dp4a(codes of the token, codes of the column's feature).
 template <int W, int CH, bool PER_TOKEN>
 __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int qd, uint32_t qx, float s_x, uint32_t (&v)[CH])
 {
-    chunk_pipeline<CH>(v, [&](int j, float *out) {
-        const float4 A = lds128(cbase + (m0 + 4 * j) * 4);
-        const float4 B = lds128(cbase + (W + m0 + 4 * j) * 4);
-        const float4 Cc = lds128(cbase + (2 * W + m0 + 4 * j) * 4);
-        const float Av[4] = {A.x, A.y, A.z, A.w}, Bv[4] = {B.x, B.y, B.z, B.w}, Cv[4] = {Cc.x, Cc.y, Cc.z, Cc.w};
-        if constexpr (!PER_TOKEN) {
+    chunk_pipeline<CH>(v, [&](int j, f32x2 *out) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                out[e] = sine_fixed(qs, qd, __float_as_uint(Av[e]), __float_as_uint(Cv[e]), __float_as_uint(Bv[e]));
-        } else {
-            const float4 wq = lds128(cbase + (3 * W + m0 + 4 * j) * 4);
-            const float wv[4] = {wq.x, wq.y, wq.z, wq.w};
+        for (int q = 0; q < 2; ++q) {
+            const int i = 8 * j + 4 * q;
+            const float4 A = lds128(cbase + (m0 + i) * 4);
+            const float4 B = lds128(cbase + (W + m0 + i) * 4);
+            const float4 Cc = lds128(cbase + (2 * W + m0 + i) * 4);
+            const float Av[4] = {A.x, A.y, A.z, A.w}, Bv[4] = {B.x, B.y, B.z, B.w}, Cv[4] = {Cc.x, Cc.y, Cc.z, Cc.w};
+            float y[4];
+            if constexpr (!PER_TOKEN) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float c_hi, c_lo;
-                token_const(Av[e], Cv[e], s_x, c_hi, c_lo);
-                const int acc = __dp4a((int)qx, (int)__float_as_uint(wv[e]), 0);
-                out[e] = epilogue(EPI_SINE_WIDE, (float)acc, c_hi, c_lo, Bv[e]);
+                for (int e = 0; e < 4; ++e)
+                    y[e] = sine_fixed(qs, qd, __float_as_uint(Av[e]), __float_as_uint(Cv[e]), __float_as_uint(Bv[e]));
+            } else {
+                const float4 wq = lds128(cbase + (3 * W + m0 + i) * 4);
+                const float wv[4] = {wq.x, wq.y, wq.z, wq.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float c_hi, c_lo;
+                    token_const(Av[e], Cv[e], s_x, c_hi, c_lo);
+                    const int acc = __dp4a((int)qx, (int)__float_as_uint(wv[e]), 0);
+                    y[e] = epilogue(EPI_SINE_WIDE, (float)acc, c_hi, c_lo, Bv[e]);
+                }
             }
+            out[2 * q] = pack2(y[0], y[1]);
+            out[2 * q + 1] = pack2(y[2], y[3]);
         }
     });
 }
@@ -338,7 +421,6 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
 {
     using C = Cfg<W>;
     constexpr int NCH = C::NCH, G = C::G, CH = C::CH;
-    constexpr int SN = (G >= 16) ? 16 : 8; // codes per shared-memory store
     ptx::tmem_wait_st();
     ptx::tc_fence_before();
     if (!slot_barrier(c)) return false;
@@ -351,17 +433,18 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
         ptx::tmem_wait_ld();
-        // strides CH, 2 CH, ...: the chunk index is the butterfly index
+        // strides CH, 2 CH, ...: the chunk index is the butterfly index; two columns per instruction
 #pragma unroll
         for (int h = 1; h < NCH; h <<= 1) {
 #pragma unroll
             for (int ch = 0; ch < NCH; ++ch) {
                 if ((ch & h) == 0) {
 #pragma unroll
-                    for (int i = 0; i < G; ++i) {
-                        float a = __uint_as_float(u[ch][i]), b = __uint_as_float(u[ch + h][i]);
-                        u[ch][i] = __float_as_uint(__fadd_rn(a, b));
-                        u[ch + h][i] = __float_as_uint(__fsub_rn(a, b));
+                    for (int i = 0; i < G; i += 2) {
+                        f32x2 a = pack2u(u[ch][i], u[ch][i + 1]), b = pack2u(u[ch + h][i], u[ch + h][i + 1]);
+                        bfly2(a, b);
+                        unpack2u(a, u[ch][i], u[ch][i + 1]);
+                        unpack2u(b, u[ch + h][i], u[ch + h][i + 1]);
                     }
                 }
             }
@@ -375,11 +458,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
             }
         } else {
 #pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-#pragma unroll
-                for (int i = 0; i < G; i += SN)
-                    store_codes<SN, true>(c.a_tile, c.row, ch * CH + g * G + i, &u[ch][i], static_inv, c.qmaxf);
-            }
+            for (int ch = 0; ch < NCH; ++ch) quantize_store<G, CH, true>(c.a_tile, c.row, ch, g * G, u[ch], static_inv, c.qmaxf);
         }
     }
     if (!PER_TOKEN) {
@@ -408,11 +487,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
             for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
             ptx::tmem_wait_ld();
 #pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-#pragma unroll
-                for (int i = 0; i < G; i += SN)
-                    store_codes<SN, false>(c.a_tile, c.row, ch * CH + g * G + i, &u[ch][i], inv, c.qmaxf);
-            }
+            for (int ch = 0; ch < NCH; ++ch) quantize_store<G, CH, false>(c.a_tile, c.row, ch, g * G, u[ch], inv, c.qmaxf);
         }
     }
     ptx::fence_proxy_async();
@@ -686,11 +761,12 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
             const uint32_t *srcB = fixed ? ly.fxB : reinterpret_cast<const uint32_t *>(ly.cB);
             const uint32_t *srcC = fixed ? ly.fxQ : reinterpret_cast<const uint32_t *>(ly.cA_lo);
             const int areas = (l == 0) ? (fixed ? 3 : 4) : (ly.epi_mode == EPI_SINE_WIDE ? 3 : 2);
-            for (int i = threadIdx.x; i < W; i += kThreads) {
-                d[i] = __ldg(srcA + i);
-                d[W + i] = __ldg(srcB + i);
-                if (areas >= 3) d[2 * W + i] = __ldg(srcC + i);
-                if (areas >= 4) d[3 * W + i] = __ldg(ly.qw_k4m + i);
+            for (int i = threadIdx.x; i < W; i += kThreads) { // i: tensor-memory column, m: its feature
+                const int m = fused_feature(i, W);
+                d[i] = __ldg(srcA + m);
+                d[W + i] = __ldg(srcB + m);
+                if (areas >= 3) d[2 * W + i] = __ldg(srcC + m);
+                if (areas >= 4) d[3 * W + i] = __ldg(ly.qw_k4m + m);
             }
         }
     }

@@ -76,6 +76,7 @@ struct PrepArgs {
     const float *W, *b;
     int d_out, d_in, K, M, Mt;
     int bits, per_channel;
+    int permute_rows;      // 1: rows of the tensor-core image in fused_column order (layers 2 .. L-1)
     int sine;              // hidden or first layer
     int first;             // layer 1: no phase bound from the weights (coordinates are unbounded)
     double omega0;
@@ -96,6 +97,21 @@ __host__ __device__ inline size_t umma_offset(int n, int k, int K, int slab_rows
 {
     return (size_t)(n / slab_rows) * slab_rows * K + (size_t)(k >> 4) * slab_rows * 16 +
            (size_t)(n % slab_rows) * 16 + (k & 15);
+}
+// Columns of a hidden layer's output are processed by the fused kernel in register chunks of
+// fused_chunk(W) columns, and inside a chunk the features i and i + chunk/2 sit in adjacent
+// tensor-memory columns (2i, 2i+1) so that they form the two halves of a packed fp32x2 register.
+// fused_column(m, W) is the tensor-memory column (= row of the weight image) of output feature m.
+__host__ __device__ inline int fused_chunk(int W) { return W == 64 ? 32 : 64; }
+__host__ __device__ inline int fused_column(int m, int W)
+{
+    const int ch = fused_chunk(W), c = m / ch, f = m % ch;
+    return c * ch + (f < ch / 2 ? 2 * f : 2 * (f - ch / 2) + 1);
+}
+__host__ __device__ inline int fused_feature(int col, int W)
+{
+    const int ch = fused_chunk(W), c = col / ch, j = col % ch;
+    return c * ch + (j >> 1) + (j & 1) * (ch / 2);
 }
 // Rows per slab for a layer with K inputs and Mt (padded) outputs: slabs hold at most 64 KB.
 inline int fused_slab_rows(int K, int Mt)

@@ -11,10 +11,13 @@ template <int PIPE> __global__ void __launch_bounds__(256) scalar_pipe_kernel(in
 {
     float v[kChains];
     uint32_t u[kChains];
+    unsigned long long w[kChains], k2;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(k2) : "f"(seed * 1e-3f));
 #pragma unroll
     for (int c = 0; c < kChains; ++c) {
         v[c] = seed + (float)(threadIdx.x + c) * 1e-3f;
         u[c] = threadIdx.x * 2654435761u + c;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(w[c]) : "f"(v[c]), "f"(seed));
     }
     for (int i = 0; i < iters; ++i) {
 #pragma unroll
@@ -28,12 +31,14 @@ template <int PIPE> __global__ void __launch_bounds__(256) scalar_pipe_kernel(in
                 else if (PIPE == DHQ_PIPE_F2I) asm volatile("cvt.rni.s32.f32 %0, %1;" : "=r"(u[c]) : "f"(__uint_as_float((u[c] & 0x007fffffu) | 0x3f800000u)));
                 else if (PIPE == DHQ_PIPE_PRMT) asm volatile("prmt.b32 %0, %0, %1, 0x5140;" : "+r"(u[c]) : "r"(u[(c + 1) % kChains]));
                 else if (PIPE == DHQ_PIPE_FMNMX) v[c] = fmaxf(fminf(v[c], seed), -seed);
+                else if (PIPE == DHQ_PIPE_FADD2) asm volatile("add.rn.f32x2 %0, %0, %1;" : "+l"(w[c]) : "l"(k2));
+                else if (PIPE == DHQ_PIPE_FFMA2) asm volatile("fma.rn.f32x2 %0, %0, %1, %1;" : "+l"(w[c]) : "l"(k2));
             }
         }
     }
     float acc = 0.f;
 #pragma unroll
-    for (int c = 0; c < kChains; ++c) acc += v[c] + __uint_as_float(u[c] & 0x3fffffffu);
+    for (int c = 0; c < kChains; ++c) acc += v[c] + __uint_as_float(u[c] & 0x3fffffffu) + __uint_as_float((uint32_t)(w[c] >> 32) & 0x3fffffffu);
     if (acc == 123.456f) sink[0] = acc; // keeps the loop alive
 }
 
@@ -123,6 +128,8 @@ extern "C" int dhq_measure_pipe(int pipe, int iters, void *stream, double *ops_p
         case DHQ_PIPE_F2I: e = run_scalar<DHQ_PIPE_F2I>(blocks, iters, sink, st); break;
         case DHQ_PIPE_PRMT: e = run_scalar<DHQ_PIPE_PRMT>(blocks, iters, sink, st); break;
         case DHQ_PIPE_FMNMX: e = run_scalar<DHQ_PIPE_FMNMX>(blocks, iters, sink, st); break;
+        case DHQ_PIPE_FADD2: e = run_scalar<DHQ_PIPE_FADD2>(blocks, iters, sink, st); break;
+        case DHQ_PIPE_FFMA2: e = run_scalar<DHQ_PIPE_FFMA2>(blocks, iters, sink, st); break;
         case DHQ_PIPE_TENSOR_I8:
             e = cudaFuncSetAttribute(tensor_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tensor_smem);
             if (e == cudaSuccess) {
@@ -145,7 +152,7 @@ extern "C" int dhq_measure_pipe(int pipe, int iters, void *stream, double *ops_p
             if (flag) rc = 1;
             ops = (double)sms * iters * 8.0 * 2.0 * 128 * 256 * 32;
         } else {
-            double per_thread = (double)iters * 8 * kChains * (pipe == DHQ_PIPE_FMNMX ? 2 : 1);
+            double per_thread = (double)iters * 8 * kChains * ((pipe == DHQ_PIPE_FMNMX || pipe == DHQ_PIPE_FADD2 || pipe == DHQ_PIPE_FFMA2) ? 2 : 1);
             ops = per_thread * 256.0 * blocks;
         }
         *ops_per_s = ops / ((double)t * 1e-3);
