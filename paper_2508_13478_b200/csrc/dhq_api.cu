@@ -158,7 +158,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             d.K = (l == 1) ? 4 : w;
             d.M = (l == L) ? 4 : w;
             d.Mt = d.M < 16 ? 16 : d.M;
-            d.slab_rows = fused_slab_rows(d.K, d.Mt);
+            d.slab_k = fused_slab_k(d.K, d.Mt);
             d.d_in = cfg->dims[l - 1];
             d.d_out = cfg->dims[l];
             if (l == 1) d.epi_mode = per_token ? EPI_SINE_WIDE : EPI_SINE_FIXED; // coordinates are not bounded by the weights

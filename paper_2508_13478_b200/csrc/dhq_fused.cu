@@ -42,6 +42,7 @@ constexpr int kMmaWarp = 16, kLoadWarp = 17;
 constexpr int kThreads = 18 * 32;
 constexpr int kMaxStages = 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull; // 2 s per wait
+constexpr uint32_t kCopyBytes = 8192; // bytes per bulk copy of a weight slab
 constexpr int kMinSmem = 120 * 1024; // more than half an SM's shared memory: one CTA per SM
 
 // Work split for a hidden width W.
@@ -53,8 +54,10 @@ template <int W> struct Cfg {
     static constexpr int CPT = NCH / R;                        // chunks per thread
     static constexpr int G = (64 / NCH < CH / R) ? 64 / NCH : CH / R; // positions per pass-2 group
     static constexpr int GPT = CH / (G * R);                   // groups per thread
-    static constexpr int PIECES = (W == 512) ? 4 : 1;          // MMAs per layer along N
-    static constexpr int PW = W / PIECES;                      // N of one MMA = rows of one weight slab
+    static constexpr int KSLABS = (W == 512) ? 4 : 1;          // weight slabs per layer along K
+    static constexpr int SLABK = W / KSLABS;                   // k per slab (= fused_slab_k)
+    static constexpr int NHALF = (W == 512) ? 2 : 1;           // MMAs along N (an MMA has N <= 256)
+    static constexpr int NW = W / NHALF;                       // N of one MMA
     static constexpr int SLOT_THREADS = R * kTile;
     static constexpr int TMEM_COLS_PER_SLOT = 512 / SLOTS;
 };
@@ -104,12 +107,12 @@ struct SmemMap {
 __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words)
 {
     const int slots = (W == 512) ? 1 : 2;
-    const int pw = (W == 512) ? 128 : W;
+    const int slab_k = (W == 512) ? 128 : W;
     SmemMap m;
     uint32_t off = 0;
     m.a_tile[0] = off; off += kTile * W;
     m.a_tile[1] = off; if (slots == 2) off += kTile * W;
-    m.ring = off; off += (uint32_t)n_stages * pw * W;
+    m.ring = off; off += (uint32_t)n_stages * slab_k * W;
     m.last_w = off; off += 16 * W;
     m.consts = off; off += (uint32_t)const_words * 4;
     m.amax = off; off += 2 * 4 * kTile * 4;
@@ -517,7 +520,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     c.qmaxf = p.qmaxf;
     c.abort_flag = abort_flag;
     c.status = p.status;
-    const uint32_t bar_acc = smem_base + sm.acc_full + 8 * (slot * 4 + (sub * C::PIECES) / C::R);
+    const uint32_t bar_acc = smem_base + sm.acc_full + 8 * (slot * 4);
     const uint32_t bar_last = smem_base + sm.acc_last + 8 * slot;
     const uint32_t consts = smem_base + sm.consts;
     uint32_t acc_parity = 0, last_parity = 0;
@@ -554,7 +557,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
             next_s = __ldg(p.layer[1].act + 1);
             next_inv = __ldg(p.layer[1].act + 2);
         }
-#pragma unroll 1
+#pragma unroll
         for (int cc = 0; cc < C::CPT; ++cc) {
             const int ch = sub * C::CPT + cc;
             uint32_t v[CH];
@@ -575,7 +578,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
             }
             const uint32_t cbase = consts + ly.c_off * 4;
             const bool fast = ly.epi_mode == EPI_SINE_FAST;
-#pragma unroll 1
+#pragma unroll
             for (int cc = 0; cc < C::CPT; ++cc) {
                 const int ch = sub * C::CPT + cc;
                 uint32_t v[CH];
@@ -618,55 +621,64 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
 {
     using C = Cfg<W>;
     uint32_t codes_parity[2] = {0, 0};
-    const uint32_t idesc_hidden = ptx::idesc_i8(kTile, C::PW), idesc_last = ptx::idesc_i8(kTile, 16);
-    const uint32_t slab = C::PW * W;
+    const uint32_t idesc_hidden = ptx::idesc_i8(kTile, C::NW), idesc_last = ptx::idesc_i8(kTile, 16);
+    const uint32_t slab = W * C::SLABK;
+    // each K step of 32 advances a descriptor's start-address field (bits 0-13, 16-byte units) by
+    // two core-matrix columns
+    const uint64_t a_step = (uint64_t)((2 * kTile * 16) >> 4);
     long long use = 0; // ring uses so far (streaming mode)
     bool ok = true;
     for (long long r = 0; ok; ++r) {
         const long long tile0 = ((long long)blockIdx.x + r * gridDim.x) * C::SLOTS;
         if (tile0 >= p.n_tiles) break;
         const int active = (C::SLOTS == 2 && tile0 + 1 < p.n_tiles) ? 2 : 1;
-        for (int l = 2; l <= p.L && ok; ++l) {
-            const int pieces = (l < p.L) ? C::PIECES : 1;
-            for (int pc = 0; pc < pieces && ok; ++pc) {
-                uint32_t b_addr, n_rows, idesc;
-                int stage = 0;
-                if (l < p.L) {
-                    const int slab_id = (l - 2) * C::PIECES + pc;
-                    stage = p.resident ? slab_id : (int)(use % p.n_stages);
-                    const uint32_t par = p.resident ? 0u : (uint32_t)((use / p.n_stages) & 1);
-                    if (!wait_bar<100>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
-                    b_addr = smem_base + sm.ring + (uint32_t)stage * slab;
-                    n_rows = C::PW;
-                    idesc = idesc_hidden;
-                } else {
-                    if (!wait_bar<100>(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
-                    b_addr = smem_base + sm.last_w;
-                    n_rows = 16;
-                    idesc = idesc_last;
-                }
+        for (int l = 2; l < p.L && ok; ++l) {
+            for (int ksl = 0; ksl < C::KSLABS && ok; ++ksl) {
+                const int slab_id = (l - 2) * C::KSLABS + ksl;
+                const int stage = p.resident ? slab_id : (int)(use % p.n_stages);
+                const uint32_t par = p.resident ? 0u : (uint32_t)((use / p.n_stages) & 1);
+                if (!wait_bar<100>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
+                const uint32_t b_addr = smem_base + sm.ring + (uint32_t)stage * slab;
                 for (int s = 0; s < active; ++s) {
-                    if (pc == 0) {
+                    if (ksl == 0) {
                         if (!wait_bar<100>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
                         codes_parity[s] ^= 1;
                         ptx::tc_fence_after();
                     }
-                    const uint32_t a_addr = smem_base + sm.a_tile[s];
-                    const uint32_t d = tmem_base + (uint32_t)(s * C::TMEM_COLS_PER_SLOT) + (l < p.L ? pc * C::PW : 0);
-#pragma unroll 1
-                    for (int ks = 0; ks < W / 32; ++ks) {
-                        uint64_t ad = ptx::smem_desc(a_addr + ks * 2 * (kTile * 16), kTile * 16, 128);
-                        uint64_t bd = ptx::smem_desc(b_addr + ks * 2 * (n_rows * 16), n_rows * 16, 128);
-                        ptx::mma_i8(d, ad, bd, idesc, ks > 0 ? 1u : 0u);
+                    const uint64_t ad0 = ptx::smem_desc(smem_base + sm.a_tile[s] + ksl * (C::SLABK / 16) * (kTile * 16), kTile * 16, 128);
+#pragma unroll
+                    for (int half = 0; half < C::NHALF; ++half) {
+                        const uint32_t d = tmem_base + (uint32_t)(s * C::TMEM_COLS_PER_SLOT + half * C::NW);
+                        const uint64_t bd0 = ptx::smem_desc(b_addr + half * C::NW * 16, W * 16, 128);
+                        const uint64_t b_step = (uint64_t)((2 * W * 16) >> 4);
+#pragma unroll
+                        for (int ks = 0; ks < C::SLABK / 32; ++ks)
+                            ptx::mma_i8(d, ad0 + ks * a_step, bd0 + ks * b_step, idesc_hidden, (ksl > 0 || ks > 0) ? 1u : 0u);
                     }
-                    ptx::mma_commit(l < p.L ? smem_base + sm.acc_full + 8 * (s * 4 + pc) : smem_base + sm.acc_last + 8 * s);
+                    if (ksl == C::KSLABS - 1) ptx::mma_commit(smem_base + sm.acc_full + 8 * (s * 4));
                 }
                 if (!ok) break;
-                if (l < p.L && !p.resident) {
+                if (!p.resident) {
                     ptx::mma_commit(smem_base + sm.w_empty + 8 * stage);
                     ++use;
                 }
             }
+        }
+        if (!ok) break;
+        // last layer: N = 16, its weights stay in shared memory
+        if (!wait_bar<100>(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
+        for (int s = 0; s < active; ++s) {
+            if (!wait_bar<100>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
+            codes_parity[s] ^= 1;
+            ptx::tc_fence_after();
+            const uint32_t d = tmem_base + (uint32_t)(s * C::TMEM_COLS_PER_SLOT);
+            const uint64_t ad0 = ptx::smem_desc(smem_base + sm.a_tile[s], kTile * 16, 128);
+            const uint64_t bd0 = ptx::smem_desc(smem_base + sm.last_w, 16 * 16, 128);
+            const uint64_t b_step = (uint64_t)((2 * 16 * 16) >> 4);
+#pragma unroll
+            for (int ks = 0; ks < W / 32; ++ks)
+                ptx::mma_i8(d, ad0 + ks * a_step, bd0 + ks * b_step, idesc_last, ks > 0 ? 1u : 0u);
+            ptx::mma_commit(smem_base + sm.acc_last + 8 * s);
         }
     }
     if (!ok) { // give the MMAs already issued a bounded time to finish before TMEM is released
@@ -680,10 +692,10 @@ template <int W>
 __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
 {
     using C = Cfg<W>;
-    const uint32_t slab = C::PW * W;
+    const uint32_t slab = W * C::SLABK;
     ptx::mbar_expect_tx(smem_base + sm.last_full, 16 * W);
     ptx::bulk_g2s(smem_base + sm.last_w, p.layer[p.L - 1].qw_umma, 16 * W, smem_base + sm.last_full);
-    const int slabs = (p.L - 2) * C::PIECES; // per tile round
+    const int slabs = (p.L - 2) * C::KSLABS; // per tile round
     if (slabs <= 0) return;
     long long rounds = 0;
     for (long long r = 0;; ++r) {
@@ -700,10 +712,14 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
             if (!wait_bar<100>(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
         }
         const int id = (int)(i % slabs);
-        const int l = 2 + id / C::PIECES, pc = id % C::PIECES;
+        const int l = 2 + id / C::KSLABS, pc = id % C::KSLABS;
         ptx::mbar_expect_tx(smem_base + sm.w_full + 8 * stage, slab);
-        ptx::bulk_g2s(smem_base + sm.ring + (uint32_t)stage * slab, p.layer[l - 1].qw_umma + (size_t)pc * slab, slab,
-                      smem_base + sm.w_full + 8 * stage);
+        // several copies in flight per slab: one large bulk copy did not reach the L2 bandwidth
+        for (uint32_t off = 0; off < slab; off += kCopyBytes) {
+            const uint32_t bytes = slab - off < kCopyBytes ? slab - off : kCopyBytes;
+            ptx::bulk_g2s(smem_base + sm.ring + (uint32_t)stage * slab + off,
+                          p.layer[l - 1].qw_umma + (size_t)pc * slab + off, bytes, smem_base + sm.w_full + 8 * stage);
+        }
         ++issued;
     }
     if (!ok || *abort_flag) { // let copies in flight land before the CTA may exit
@@ -842,9 +858,9 @@ dhq_status_t fused_create(dhq_handle_s *h)
         return DHQ_ERR_CUDA;
     // weight ring: as many slab stages as fit beside the A tiles and the constants; all hidden
     // layers resident if they fit
-    const int pieces = (h->w == 512) ? 4 : 1;
-    const int slabs = (h->L - 2) * pieces;
-    const size_t slab_bytes = (size_t)(h->w / pieces) * h->w;
+    const int kslabs = (h->w == 512) ? 4 : 1;
+    const int slabs = (h->L - 2) * kslabs;
+    const size_t slab_bytes = (size_t)(h->w / kslabs) * h->w;
     const size_t fixed = smem_map(h->w, 0, words).total + 1024;
     if (fixed > (size_t)max_optin) return DHQ_ERR_UNSUPPORTED;
     int stages = (int)(((size_t)max_optin - fixed) / slab_bytes);

@@ -14,7 +14,7 @@ constexpr int kDebugChunk = 65536; // tokens per pass of the layer-by-layer path
 struct LayerDev {
     int K = 0, M = 0;          // padded sizes as the definition pads them (K = 4 | w, M = w | 4)
     int Mt = 0;                // rows of the tensor-core weight tile (M rounded up to 16)
-    int slab_rows = 0;         // rows per contiguous slab of the tensor-core image
+    int slab_k = 0;            // k per contiguous slab of the tensor-core image
     int d_in = 0, d_out = 0;
     int epi_mode = EPI_LINEAR;
     float phase_bound = 0.f;   // omega0 * max_m (sum_k |W_mk| + |b_m|), hidden layers
@@ -88,16 +88,18 @@ cudaError_t launch_prepare(const PrepArgs &a, cudaStream_t st, int64_t *launches
 cudaError_t launch_finalize(const LayerDev &dev, int a_bits, int per_token, int sine, double omega0,
                             cudaStream_t st, int64_t *launches);
 
-// Byte offset of code (n, k) in the tensor-core shared-memory image of a weight matrix with K
-// codes per row: contiguous slabs of `slab_rows` rows; inside a slab the 16-byte k-groups are
-// the outer index and rows the inner one, i.e. 8-row x 16-byte core matrices stacked along rows
-// (128 bytes apart) and along k (slab_rows * 16 bytes apart) - the K-major, unswizzled operand
-// layout of tcgen05.mma.
-__host__ __device__ inline size_t umma_offset(int n, int k, int K, int slab_rows)
+// Byte offset of code (n, k) in the tensor-core shared-memory image of a weight matrix with `rows`
+// rows and K codes per row.  The image is a sequence of contiguous slabs of `slab_k` consecutive
+// k (all rows); inside a slab the 16-byte k-groups are the outer index and rows the inner one,
+// i.e. 8-row x 16-byte core matrices stacked along rows (128 bytes apart) and along k
+// (rows * 16 bytes apart) - the K-major, unswizzled operand layout of tcgen05.mma.
+__host__ __device__ inline size_t umma_offset(int n, int k, int rows, int slab_k)
 {
-    return (size_t)(n / slab_rows) * slab_rows * K + (size_t)(k >> 4) * slab_rows * 16 +
-           (size_t)(n % slab_rows) * 16 + (k & 15);
+    return (size_t)(k / slab_k) * rows * slab_k + (size_t)((k % slab_k) >> 4) * rows * 16 + (size_t)n * 16 + (k & 15);
 }
+// Codes per row in one slab: a 512 x 512 layer is streamed in four slabs of 128 k (64 KB each);
+// narrower layers are one slab.
+__host__ __device__ inline int fused_slab_k(int K, int rows) { return (K == 512 && rows == 512) ? 128 : (K < 16 ? 16 : K); }
 // Columns of a hidden layer's output are processed by the fused kernel in register chunks of
 // fused_chunk(W) columns, and inside a chunk the features i and i + chunk/2 sit in adjacent
 // tensor-memory columns (2i, 2i+1) so that they form the two halves of a packed fp32x2 register.
@@ -113,13 +115,6 @@ __host__ __device__ inline int fused_feature(int col, int W)
     const int ch = fused_chunk(W), c = col / ch, j = col % ch;
     return c * ch + (j >> 1) + (j & 1) * (ch / 2);
 }
-// Rows per slab for a layer with K inputs and Mt (padded) outputs: slabs hold at most 64 KB.
-inline int fused_slab_rows(int K, int Mt)
-{
-    int rows = 65536 / (K < 16 ? 16 : K);
-    return rows < Mt ? rows : Mt;
-}
-
 // Fused tensor-core forward.
 dhq_status_t fused_create(dhq_handle_s *h);
 void fused_destroy(dhq_handle_s *h);

@@ -90,7 +90,7 @@ __global__ void prep_quant_kernel(PrepArgs a)
             ((int8_t *)a.dev.qw_k4m)[((size_t)(k >> 2) * M + m) * 4 + (k & 3)] = (int8_t)q;
         }
         const int row = a.permute_rows ? fused_column(m, M) : m;
-        a.dev.qw_umma[umma_offset(row, k, K, a.dev.slab_rows)] = (uint8_t)(int8_t)q;
+        a.dev.qw_umma[umma_offset(row, k, Mt, a.dev.slab_k)] = (uint8_t)(int8_t)q;
     }
 }
 
