@@ -4,9 +4,9 @@
 // One persistent CTA per SM, 18 warps:
 //   warps 0-15  epilogue warps.  Width <= 256: two "slots" of 8 warps, each slot has one tile of
 //               128 tokens in flight (its own A operand tile and 256 tensor-memory columns), so
-//               that one slot's CUDA-core work overlaps the other slot's MMA.  Width 512: one slot
-//               of 16 warps, the layer's MMA split in four N = 128 pieces so that the epilogue of
-//               piece j overlaps the MMA of piece j+1.
+//               that one slot's CUDA-core work overlaps the other slot's MMA; the second slot
+//               starts half a layer period late.  Width 512: one slot of 16 warps; a layer's
+//               weights arrive as four K slabs of 128 and each slab feeds two N = 256 MMAs.
 //               A token (row) is a tensor-memory lane; R = 2 (or 4) threads from different warps
 //               share a row and split its columns.
 //   warp 16     issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in tensor memory).
@@ -527,6 +527,14 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     const FusedLayer &l1 = p.layer[0];
     const float qmaxf = p.qmaxf;
 
+    if (C::SLOTS == 2 && slot == 1 && p.n_tiles > 1 && p.resident) {
+        // Start the second slot about half a layer period after the first, so that one slot's
+        // sine-heavy pass 1 and MMA wait fall on the other slot's pass 2 instead of both slots
+        // asking for the same pipe at the same time.  The offset then keeps itself.  Not when the
+        // weights are streamed: there both slots should consume a slab while it is in the ring.
+        const unsigned long long t0 = ptx::globaltimer(), delay = (3500ull * W * W) / (256 * 256);
+        while (ptx::globaltimer() - t0 < delay) __nanosleep(64);
+    }
     for (long long r = 0;; ++r) {
         const long long tile = ((long long)blockIdx.x + r * gridDim.x) * C::SLOTS + slot;
         if (tile >= p.n_tiles) break;
