@@ -177,6 +177,8 @@ def run_ours(args, workload):
 
     weights, biases = workload.network()
     coords_np = workload.coords()
+    if args.limit_coords > 0:
+        coords_np = np.ascontiguousarray(coords_np[: args.limit_coords])
     n, d_L = coords_np.shape[0], workload.dims[-1]
     W = [torch.from_numpy(w).cuda() for w in weights]
     B = [torch.from_numpy(b).cuda() for b in biases]
@@ -262,6 +264,48 @@ def run_ours(args, workload):
         dist.destroy_process_group()
 
 
+def run_sweep(args, workload):
+    """Batch-size sweep of the workload's network: n = 2^12 .. 2^24 coordinates, activation
+    scales frozen once on the workload's own grid (so a coordinate's result does not depend on
+    the batch).  One JSON line with the throughput curve; single GPU."""
+    import torch
+    import paper_2508_13478_b200 as dhq
+
+    torch.cuda.set_device(0)
+    weights, biases = workload.network()
+    d_L = workload.dims[-1]
+    h = dhq.dhq_prepare(workload.dims, [torch.from_numpy(w).cuda() for w in weights],
+                        [torch.from_numpy(b).cuda() for b in biases], workload.omega0, workload.w_bits,
+                        workload.a_bits, workload.w_gran, workload.a_gran)
+    dhq.dhq_calibrate(h, torch.from_numpy(workload.coords()).cuda())
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    points = []
+    for k in range(12, 25):
+        coords = torch.from_numpy(dhq_inputs.sweep_grid(k)).cuda()
+        n = coords.shape[0]
+        out = torch.empty((n, d_L), dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            dhq.dhq_forward(h, coords, out)
+        times = []
+        for _ in range(args.sweep_reps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            dhq.dhq_forward(h, coords, out)
+            b.record(stream)
+            b.synchronize()
+            times.append(a.elapsed_time(b))
+        ms = float(np.median(times))
+        points.append({"log2_n": k, "n": n, "ms": ms, "coords_per_s": n / (ms * 1e-3)})
+    status = dhq.dhq_last_status(h)
+    dhq.dhq_destroy(h)
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": 1, "data": "synthetic",
+                      "config": {"workload": workload.name, "dims": list(workload.dims), "sweep": "n = 2^12 .. 2^24",
+                                 "l2": "flushed before every timed call", "timing": f"median of {args.sweep_reps} calls"},
+                      "device_status": status, "sweep": points}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -270,10 +314,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C2", choices=sorted(dhq_inputs.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--limit-coords", type=int, default=0,
+                    help="use only the first N coordinates of the workload's grid (profiling captures)")
+    ap.add_argument("--sweep", action="store_true", help="batch-size sweep 2^12..2^24 instead of the timed steps")
+    ap.add_argument("--sweep-reps", type=int, default=20)
     args = ap.parse_args()
     workload = dhq_inputs.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, workload)
+    elif args.sweep:
+        run_sweep(args, workload)
     else:
         run_ours(args, workload)
 
