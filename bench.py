@@ -37,13 +37,14 @@ SM_COUNT = 148
 FP32_LANES_PER_SM = 128
 
 
-def alu_laneops_per_coord(dims) -> float:
+def alu_laneops_per_coord(dims, rotate=True) -> float:
     """Plain-ALU lane operations the method needs per coordinate: per element of every hidden
-    activation vector log2(w) butterfly adds plus 7 (int->float, scale+bias fma, 2 for the sine's
-    range handling, quantizer multiply, rounding, packing/abs-max)."""
+    activation vector log2(w) butterfly adds (none without the rotation) plus 7 (int->float,
+    scale+bias fma, 2 for the sine's range handling, quantizer multiply, rounding,
+    packing/abs-max)."""
     w = dims[1]
     hidden_vectors = len(dims) - 2
-    return float(hidden_vectors * w * (7 + int(np.log2(w))))
+    return float(hidden_vectors * w * (7 + (int(np.log2(w)) if rotate else 0)))
 
 
 class ClockSampler:
@@ -106,12 +107,12 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
-def time_oracle(workload, steps, warmup, sample_tokens):
+def time_oracle(workload, steps, warmup, sample_tokens, rotate=True):
     """The CPU oracle, as it stands, on `sample_tokens` coordinates of the workload."""
     from oracle import dhq_oracle as orc
     weights, biases = workload.network()
     net = orc.prepare(weights, biases, workload.dims, workload.omega0, workload.w_bits, workload.a_bits,
-                      workload.w_gran, workload.a_gran)
+                      workload.w_gran, workload.a_gran, rotate=rotate)
     coords = workload.coords()[:sample_tokens]
     if workload.a_gran == 0:
         orc.calibrate(net, coords)
@@ -131,7 +132,7 @@ def run_reference(args, workload):
     sample = min(workload.n, 16384)
     steps = max(1, min(args.steps, 5))
     warmup = min(args.warmup, 1)
-    value, dt, cores = time_oracle(workload, steps, warmup, sample)
+    value, dt, cores = time_oracle(workload, steps, warmup, sample, args.rotation == "input")
     desc = f"first {sample} coordinates of the {workload.grid[0]}x{workload.grid[1]} grid per step"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -183,7 +184,7 @@ def run_ours(args, workload):
     W = [torch.from_numpy(w).cuda() for w in weights]
     B = [torch.from_numpy(b).cuda() for b in biases]
     h = dhq.dhq_prepare(workload.dims, W, B, workload.omega0, workload.w_bits, workload.a_bits,
-                        workload.w_gran, workload.a_gran)
+                        workload.w_gran, workload.a_gran, rotation=0 if args.rotation == "input" else 2)
     coords = torch.from_numpy(coords_np).cuda()
     out = torch.empty((n, d_L), dtype=torch.float32, device="cuda")
     coords_host = torch.from_numpy(coords_np).pin_memory()
@@ -235,7 +236,7 @@ def run_ours(args, workload):
             pass
         sm_max = float(peaks.get("sm_max_mhz", 1965.0))
         alu_peak = SM_COUNT * FP32_LANES_PER_SM * sm_max * 1e6 / 1e12            # T lane-ops/s
-        achieved = alu_laneops_per_coord(workload.dims) * n / (ms_per_step * 1e-3) / 1e12
+        achieved = alu_laneops_per_coord(workload.dims, args.rotation == "input") * n / (ms_per_step * 1e-3) / 1e12
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -243,7 +244,7 @@ def run_ours(args, workload):
             "data": "synthetic",
             "config": {"workload": workload.name, "dims": list(workload.dims), "coords_per_step": n,
                        "bits": [workload.w_bits, workload.a_bits], "w_gran": workload.w_gran,
-                       "a_gran": workload.a_gran, "l2": "flushed between steps (256 MB write)",
+                       "a_gran": workload.a_gran, "rotation": args.rotation, "l2": "flushed between steps (256 MB write)",
                        "parallelism": f"{world} independent replica(s)"},
             "clocks": clocks.summary(),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * 8, "d2h_bytes_per_step": n * d_L * 4},
@@ -255,7 +256,7 @@ def run_ours(args, workload):
         }
         if world == 1 and not args.no_cpu_baseline:
             sample = min(n, 65536)
-            v, dt, cores = time_oracle(workload, 1, 1, sample)
+            v, dt, cores = time_oracle(workload, 1, 1, sample, args.rotation == "input")
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                     "sample": f"first {sample} coordinates of the grid, one pass ({dt:.1f} s)"}
         print(json.dumps(line), flush=True)
@@ -276,7 +277,8 @@ def run_sweep(args, workload):
     d_L = workload.dims[-1]
     h = dhq.dhq_prepare(workload.dims, [torch.from_numpy(w).cuda() for w in weights],
                         [torch.from_numpy(b).cuda() for b in biases], workload.omega0, workload.w_bits,
-                        workload.a_bits, workload.w_gran, workload.a_gran)
+                        workload.a_bits, workload.w_gran, workload.a_gran,
+                        rotation=0 if args.rotation == "input" else 2)
     dhq.dhq_calibrate(h, torch.from_numpy(workload.coords()).cuda())
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
@@ -314,6 +316,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C2", choices=sorted(dhq_inputs.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rotation", default="input", choices=["input", "none"],
+                    help="input = DHQ; none = the same path without the Hadamard rotation (uniform quantizer)")
     ap.add_argument("--limit-coords", type=int, default=0,
                     help="use only the first N coordinates of the workload's grid (profiling captures)")
     ap.add_argument("--sweep", action="store_true", help="batch-size sweep 2^12..2^24 instead of the timed steps")

@@ -56,6 +56,7 @@ LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X
     a.a_bits = h->cfg.a_bits;
     a.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
     a.epi_mode = d.epi_mode;
+    a.rotate = h->cfg.rotation == DHQ_ROT_INPUT;
     a.qw_k4m = d.qw_k4m; a.cA = d.cA; a.cA_lo = d.cA_lo; a.cB = d.cB; a.act = d.act;
     a.fxP = d.fxP; a.fxQ = d.fxQ; a.fxB = d.fxB;
     return a;
@@ -132,7 +133,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     for (int l = 1; l < L; ++l)
         if (cfg->dims[l] != w) return DHQ_ERR_UNSUPPORTED;
     if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits < 2 || cfg->a_bits > 8) return DHQ_ERR_UNSUPPORTED;
-    if (cfg->rotation != DHQ_ROT_INPUT) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->rotation != DHQ_ROT_INPUT && cfg->rotation != DHQ_ROT_NONE) return DHQ_ERR_UNSUPPORTED;
     if ((cfg->w_gran != DHQ_GRAN_TENSOR && cfg->w_gran != DHQ_GRAN_CHANNEL_OR_TOKEN) ||
         (cfg->a_gran != DHQ_GRAN_TENSOR && cfg->a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN))
         return DHQ_ERR_INVALID_ARG;
@@ -179,6 +180,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             a.per_channel = cfg->w_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
             a.sine = l < L; a.first = l == 1;
             a.permute_rows = (l > 1 && l < L) ? 1 : 0;
+            a.rotate = cfg->rotation == DHQ_ROT_INPUT;
             a.omega0 = (double)cfg->omega0;
             a.dev = d;
             a.phase_bound = d_bounds + (l - 1);

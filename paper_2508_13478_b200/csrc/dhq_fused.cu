@@ -285,10 +285,17 @@ __device__ __forceinline__ float4 lds128(uint32_t addr)
 // butterflies follow every fourth group - so that the special-function unit (one sine per 8 issue
 // cycles and scheduler) is fed evenly instead of in one burst per chunk.  Each element still goes
 // through the stages in the order 1, 2, 4, ...: the sums are unchanged.
-template <int CH, class Sine8> __device__ __forceinline__ void chunk_pipeline(uint32_t (&v)[CH], Sine8 sine8)
+template <int CH, bool ROT, class Sine8> __device__ __forceinline__ void chunk_pipeline(uint32_t (&v)[CH], Sine8 sine8)
 {
     constexpr int NP = CH / 2;
     f32x2 P[NP];
+    if constexpr (!ROT) { // no rotation (plain uniform quantization): activations only
+#pragma unroll
+        for (int j = 0; j < NP / 4; ++j) sine8(j, &P[4 * j]);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) unpack2u(P[i], v[2 * i], v[2 * i + 1]);
+        return;
+    }
     sine8(0, &P[0]);
 #pragma unroll
     for (int j = 0; j < NP / 4; ++j) {
@@ -324,10 +331,10 @@ template <int CH, class Sine8> __device__ __forceinline__ void chunk_pipeline(ui
 
 // Hidden layer: dequantize + bias + sine of the CH columns starting at column m0.  Constants come
 // from shared memory in column order: area A = cA, B = cB, C = cA_lo, each W words.
-template <int W, int CH, bool PER_TOKEN, int MODE>
+template <int W, int CH, bool PER_TOKEN, bool ROT, int MODE>
 __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH])
 {
-    chunk_pipeline<CH>(v, [&](int j, f32x2 *out) {
+    chunk_pipeline<CH, ROT>(v, [&](int j, f32x2 *out) {
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int i = 8 * j + 4 * q; // four columns = two pairs
@@ -361,10 +368,10 @@ __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, 
 // Layer 1 for the CH columns starting at column m0.  Fixed-point mode: areas A = P, B = B, C = Q.
 // Float mode (per-token scales): A = cA, B = cB, C = cA_lo, D = the weight codes, one word per
 // column, and acc = dp4a(codes of the token, codes of the column's feature).
-template <int W, int CH, bool PER_TOKEN>
+template <int W, int CH, bool PER_TOKEN, bool ROT>
 __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int qd, uint32_t qx, float s_x, uint32_t (&v)[CH])
 {
-    chunk_pipeline<CH>(v, [&](int j, f32x2 *out) {
+    chunk_pipeline<CH, ROT>(v, [&](int j, f32x2 *out) {
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int i = 8 * j + 4 * q;
@@ -419,7 +426,7 @@ __device__ __forceinline__ bool slot_barrier(SlotCtx &c)
 // Passes 2 and 3: remaining butterfly stages across chunks, quantizer, store of the codes, and the
 // arrival on the "codes ready" barrier.  Returns false if a wait ran out.  s_out receives the
 // token's activation scale of the next layer.
-template <int W, bool PER_TOKEN>
+template <int W, bool PER_TOKEN, bool ROT>
 __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float static_inv, float &s_out)
 {
     using C = Cfg<W>;
@@ -438,7 +445,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
         ptx::tmem_wait_ld();
         // strides CH, 2 CH, ...: the chunk index is the butterfly index; two columns per instruction
 #pragma unroll
-        for (int h = 1; h < NCH; h <<= 1) {
+        for (int h = 1; h < (ROT ? NCH : 1); h <<= 1) {
 #pragma unroll
             for (int ch = 0; ch < NCH; ++ch) {
                 if ((ch & h) == 0) {
@@ -499,7 +506,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
     return true;
 }
 
-template <int W, bool PER_TOKEN>
+template <int W, bool PER_TOKEN, bool ROT>
 __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
@@ -547,8 +554,11 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
             float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
             x = xy.x; y = xy.y;
         }
-        float r0 = __fadd_rn(x, y), r1 = __fsub_rn(x, y), r2 = __fadd_rn(0.f, 0.f), r3 = __fsub_rn(0.f, 0.f);
-        float e0 = __fadd_rn(r0, r2), e2 = __fsub_rn(r0, r2), e1 = __fadd_rn(r1, r3), e3 = __fsub_rn(r1, r3);
+        float e0 = x, e1 = y, e2 = 0.f, e3 = 0.f;
+        if (ROT) {
+            float r0 = __fadd_rn(x, y), r1 = __fsub_rn(x, y), r2 = __fadd_rn(0.f, 0.f), r3 = __fsub_rn(0.f, 0.f);
+            e0 = __fadd_rn(r0, r2); e2 = __fsub_rn(r0, r2); e1 = __fadd_rn(r1, r3); e3 = __fsub_rn(r1, r3);
+        }
         float s_x, inv_x;
         if (PER_TOKEN) {
             float a = fmaxf(fmaxf(fabsf(e0), fabsf(e1)), fmaxf(fabsf(e2), fabsf(e3)));
@@ -569,10 +579,10 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
         for (int cc = 0; cc < C::CPT; ++cc) {
             const int ch = sub * C::CPT + cc;
             uint32_t v[CH];
-            layer1_chunk<W, CH, PER_TOKEN>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v);
+            layer1_chunk<W, CH, PER_TOKEN, ROT>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v);
             tmem_st<CH>(c.taddr + ch * CH, v);
         }
-        if (!finish_layer<W, PER_TOKEN>(c, next_s, next_inv, s_x)) return;
+        if (!finish_layer<W, PER_TOKEN, ROT>(c, next_s, next_inv, s_x)) return;
 
         // ---------------- layers 2 .. L on the tensor core
         for (int l = 2; l < p.L; ++l) {
@@ -592,11 +602,11 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
                 uint32_t v[CH];
                 tmem_ld<CH>(c.taddr + ch * CH, v);
                 ptx::tmem_wait_ld();
-                if (fast) hidden_chunk<W, CH, PER_TOKEN, EPI_SINE_FAST>(cbase, ch * CH, s_x, v);
-                else hidden_chunk<W, CH, PER_TOKEN, EPI_SINE_WIDE>(cbase, ch * CH, s_x, v);
+                if (fast) hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_FAST>(cbase, ch * CH, s_x, v);
+                else hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_WIDE>(cbase, ch * CH, s_x, v);
                 tmem_st<CH>(c.taddr + ch * CH, v);
             }
-            if (!finish_layer<W, PER_TOKEN>(c, next_s, next_inv, s_x)) return;
+            if (!finish_layer<W, PER_TOKEN, ROT>(c, next_s, next_inv, s_x)) return;
         }
         {
             const FusedLayer &ly = p.layer[p.L - 1];
@@ -741,7 +751,7 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
     }
 }
 
-template <int W, bool PER_TOKEN>
+template <int W, bool PER_TOKEN, bool ROT>
 __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constant__ FusedParams p)
 {
     using C = Cfg<W>;
@@ -800,7 +810,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
+        epilogue_role<W, PER_TOKEN, ROT>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_role<W>(p, sm, smem_base, tmem_base, abort_flag);
     } else {
@@ -818,13 +828,18 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
 
 typedef void (*fused_fn)(const FusedParams);
 
-static fused_fn pick_kernel(int W, bool per_token)
+template <int W> static fused_fn pick_width(bool per_token, bool rot)
+{
+    if (rot) return per_token ? fused_kernel<W, true, true> : fused_kernel<W, false, true>;
+    return per_token ? fused_kernel<W, true, false> : fused_kernel<W, false, false>;
+}
+static fused_fn pick_kernel(int W, bool per_token, bool rot)
 {
     switch (W) {
-    case 64: return per_token ? fused_kernel<64, true> : fused_kernel<64, false>;
-    case 128: return per_token ? fused_kernel<128, true> : fused_kernel<128, false>;
-    case 256: return per_token ? fused_kernel<256, true> : fused_kernel<256, false>;
-    case 512: return per_token ? fused_kernel<512, true> : fused_kernel<512, false>;
+    case 64: return pick_width<64>(per_token, rot);
+    case 128: return pick_width<128>(per_token, rot);
+    case 256: return pick_width<256>(per_token, rot);
+    case 512: return pick_width<512>(per_token, rot);
     }
     return nullptr;
 }
@@ -857,7 +872,7 @@ dhq_status_t fused_create(dhq_handle_s *h)
         }
     }
     p.const_words = words;
-    fused_fn fn = pick_kernel(h->w, p.per_token);
+    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     if (!fn) return DHQ_ERR_UNSUPPORTED;
     int dev = 0, max_optin = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -897,7 +912,7 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     FusedParams p = fs->p;
     p.coords = coords; p.out = out; p.n = n;
     p.n_tiles = (n + kTile - 1) / kTile;
-    fused_fn fn = pick_kernel(h->w, p.per_token);
+    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     const int slots = (h->w == 512) ? 1 : 2;
     long long rounds_all = (p.n_tiles + slots - 1) / slots;
     int grid = (int)(rounds_all < fs->sm_count ? rounds_all : fs->sm_count);

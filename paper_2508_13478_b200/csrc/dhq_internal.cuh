@@ -60,6 +60,7 @@ struct LayerArgs {
     int a_bits;
     int per_token;
     int epi_mode;
+    int rotate;            // 0: DHQ_ROT_NONE, the layer input is quantized as it is
     int calib_only;        // 1: only take max |rotated input| into act[0] (bit pattern max)
     const uint32_t *qw_k4m;
     const float *cA, *cA_lo, *cB;
@@ -76,6 +77,7 @@ struct PrepArgs {
     const float *W, *b;
     int d_out, d_in, K, M, Mt;
     int bits, per_channel;
+    int rotate;            // 0: DHQ_ROT_NONE, weights are quantized as they are
     int permute_rows;      // 1: rows of the tensor-core image in fused_column order (layers 2 .. L-1)
     int sine;              // hidden or first layer
     int first;             // layer 1: no phase bound from the weights (coordinates are unbounded)

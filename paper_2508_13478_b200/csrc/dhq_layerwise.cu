@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
         if (a.dX && tok < a.n) a.dX[tok * K + k] = v;
     }
     // rotation: strides 1, 2, ..., K/2; pair (i, i+h) -> (x+y, x-y)
-    for (int h = 1; h < K; h <<= 1) {
+    for (int h = 1; h < (a.rotate ? K : 1); h <<= 1) {
         __syncthreads();
         for (int p = tid; p < TB * (K / 2); p += LW_THREADS) {
             int t = p / (K / 2), j = p % (K / 2);

@@ -29,7 +29,7 @@ __global__ void prep_rotate_kernel(PrepArgs a)
         atomicMax((unsigned int *)a.phase_bound, __float_as_uint(bound));
         a.dev.bias[m] = (m < a.d_out) ? a.b[m] : 0.0f;
     }
-    for (int h = 1; h < K; h <<= 1) {
+    for (int h = 1; h < (a.rotate ? K : 1); h <<= 1) {
         __syncthreads();
         for (int p = threadIdx.x; p < K / 2; p += blockDim.x) {
             int i = ((p & ~(h - 1)) << 1) | (p & (h - 1));
@@ -39,7 +39,7 @@ __global__ void prep_rotate_kernel(PrepArgs a)
         }
     }
     __syncthreads();
-    const float invK = 1.0f / (float)K; // power of two: exact
+    const float invK = a.rotate ? 1.0f / (float)K : 1.0f; // power of two: exact
     float amax = 0.f;
     for (int k = threadIdx.x; k < K; k += blockDim.x) {
         float v = __fmul_rn(row[k], invK);

@@ -59,6 +59,7 @@ extern "C" dhq_status_t dhq_forward_static_scratch(dhq_handle_t h, const float *
         a.a_bits = h->cfg.a_bits;
         a.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
         a.epi_mode = d.epi_mode;
+        a.rotate = h->cfg.rotation == DHQ_ROT_INPUT;
         a.qw_k4m = d.qw_k4m; a.cA = d.cA; a.cA_lo = d.cA_lo; a.cB = d.cB; a.act = d.act;
         a.fxP = d.fxP; a.fxQ = d.fxQ; a.fxB = d.fxB;
         a.Y = scratch + (size_t)((l - 1) & 1) * kHalf; // every row < n is written before it is read

@@ -13,10 +13,10 @@ def to_dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def prepare_pair(dims, weights, biases, omega0, w_bits, a_bits, w_gran, a_gran):
+def prepare_pair(dims, weights, biases, omega0, w_bits, a_bits, w_gran, a_gran, rotate=True):
     h = dhq.dhq_prepare(dims, [to_dev(w) for w in weights], [to_dev(b) for b in biases], omega0,
-                        w_bits, a_bits, w_gran, a_gran)
-    net = orc.prepare(weights, biases, dims, omega0, w_bits, a_bits, w_gran, a_gran)
+                        w_bits, a_bits, w_gran, a_gran, rotation=0 if rotate else 2)
+    net = orc.prepare(weights, biases, dims, omega0, w_bits, a_bits, w_gran, a_gran, rotate=rotate)
     return h, net
 
 

@@ -27,10 +27,10 @@ def _built():
     assert torch.cuda.is_available()
 
 
-def _p1(workload, coords_np, fused=True):
+def _p1(workload, coords_np, fused=True, rotate=True):
     weights, biases = workload.network()
     h, net = prepare_pair(workload.dims, weights, biases, workload.omega0, workload.w_bits,
-                          workload.a_bits, workload.w_gran, workload.a_gran)
+                          workload.a_bits, workload.w_gran, workload.a_gran, rotate=rotate)
     try:
         check_weights(h, net)
         cd = to_dev(coords_np)
@@ -96,6 +96,16 @@ def test_every_width_with_ragged_tail_and_several_rounds(width, a_gran):
     _p1(wl, coords)
 
 
+@pytest.mark.parametrize("name,count", [("C1", 4096), ("C2", 9000 + 5), ("C3", 9000 + 5), ("C5", 3000 + 7)])
+def test_no_rotation_variant_uniform_quantizer(name, count):
+    # DHQ_ROT_NONE: the uniform quantizer of the paper's comparison (Section IV-B), same path
+    # without the Hadamard rotation of weights and activations
+    w = dhq_inputs.WORKLOADS[name]
+    coords = w.coords()
+    idx = np.linspace(0, coords.shape[0] - 1, count).astype(np.int64)
+    _p1(w, np.ascontiguousarray(coords[idx]), rotate=False)
+
+
 def test_trained_like_weights_and_wide_phases():
     # bell-shaped hidden weights, two-peaked last layer (Section III-A), and a first layer scaled up
     # so that phases reach hundreds of radians
@@ -144,7 +154,7 @@ def test_unsupported_and_invalid_arguments():
         dhq.dhq_prepare((3, 64, 64, 64, 1), W, B)
     assert e.value.code == 2
     with pytest.raises(dhq.DhqError) as e:
-        dhq.dhq_prepare((2, 64, 64, 64, 1), W, B, rotation=1)
+        dhq.dhq_prepare((2, 64, 64, 64, 1), W, B, rotation=1)      # two-sided rotation: not implemented
     assert e.value.code == 2
     h = dhq.dhq_prepare(w.dims, W, B)
     try:
