@@ -31,6 +31,9 @@ import numpy as np  # noqa: E402
 
 import dhq_inputs  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one fused-kernel launch, from the ncu capture
+# summarised in profiles/fused_kernel_w256_C2.md (full C2 grid, rotation on).
+NCU_DRAM_BYTES_PER_LAUNCH = {("C2", "input", 65536): 780288 + 4096}
 METRIC = "coords/sec, fused W8A8 DHQ INR forward"
 UNIT = "coords/s"
 SM_COUNT = 148
@@ -250,7 +253,8 @@ def run_ours(args, workload):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * 8, "d2h_bytes_per_step": n * d_L * 4},
             "gpu_launches": launches,
             "roofline": {"bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "Tlaneop/s",
-                         "frac": achieved / alu_peak, "traffic": None,
+                         "frac": achieved / alu_peak,
+                         "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((workload.name, args.rotation, n)),
                          "peak_source": "148 SMs x 128 fp32 lanes x max SM clock (derived, not measured)"},
             "device_status": status,
         }

@@ -75,6 +75,37 @@ def test_c3_c4_c5_sampled_tokens(name, count):
     _p1(w, np.ascontiguousarray(coords[idx]))
 
 
+@pytest.mark.parametrize("name", ["C3", "C4-W4A4", "C5"])
+def test_full_size_launch_on_sampled_outputs(name):
+    # The launch bench.py times: the whole grid of the workload in one dhq_forward call.  The
+    # oracle cannot run millions of tokens, so 3,000 tokens sampled over the grid are checked: the
+    # full launch's outputs at those tokens must equal, bit for bit, a small launch over only those
+    # tokens (same handle, same frozen scales), and that small launch is checked stage by stage
+    # against the oracle.
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        check_weights(h, net)
+        grid = to_dev(w.coords())
+        if w.a_gran == 0:
+            dhq.dhq_calibrate(h, grid)                       # scales frozen on the full grid
+        full = torch.empty((w.n, w.dims[-1]), device="cuda")
+        dhq.dhq_forward(h, grid, full)
+        torch.cuda.synchronize()
+        assert dhq.dhq_last_status(h) == 0
+        assert torch.isfinite(full).all()
+        idx = np.unique(np.concatenate([np.linspace(0, w.n - 1, 2990).astype(np.int64),
+                                        np.arange(w.n - 10, w.n)]))      # includes the last tile
+        sample_np = np.ascontiguousarray(w.coords()[idx])
+        out_dbg, bufs = run_debug(h, net, to_dev(sample_np))
+        check_layers_against_oracle(h, net, sample_np, out_dbg, bufs, calib_is_this_set=False)
+        picked = full[torch.from_numpy(idx).cuda()]
+        assert torch.equal(picked.view(torch.int32), out_dbg.view(torch.int32))
+    finally:
+        dhq.dhq_destroy(h)
+
+
 @pytest.mark.parametrize("n", [1, 127, 128, 129, 255, 257, 1000])
 def test_ragged_tails_small_width(n):
     w = dhq_inputs.WORKLOADS["C1"]
