@@ -243,6 +243,52 @@ def test_free_running_end_to_end_report():
         dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("a_gran", [0, 1])
+def test_non_finite_coordinates_do_not_hang_or_disturb_other_tokens(a_gran):
+    w = dhq_inputs.WORKLOADS["C2"]
+    weights, biases = w.network()
+    h, _ = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 1, a_gran)
+    try:
+        good = w.coords()[:1000].copy()
+        if a_gran == 0:
+            dhq.dhq_calibrate(h, to_dev(good))
+        ref = torch.empty((1000, 3), device="cuda")
+        dhq.dhq_forward(h, to_dev(good), ref)
+        bad = good.copy()
+        bad[3] = [np.nan, 0.5]
+        bad[130] = [np.inf, -np.inf]
+        bad[700] = [1e30, -1e30]
+        out = torch.empty((1000, 3), device="cuda")
+        dhq.dhq_forward(h, to_dev(bad), out)
+        torch.cuda.synchronize()
+        assert dhq.dhq_last_status(h) == 0                     # no wait ran out, the kernel returned
+        keep = np.ones(1000, bool)
+        keep[[3, 130, 700]] = False                            # every other token is untouched
+        k = torch.from_numpy(keep).cuda()
+        assert torch.equal(out[k].view(torch.int32), ref[k].view(torch.int32))
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_forward_on_a_side_stream():
+    w = dhq_inputs.WORKLOADS["C1"]
+    weights, biases = w.network()
+    h, _ = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 0, 1)
+    try:
+        cd = to_dev(w.coords())
+        ref = torch.empty((w.n, 1), device="cuda")
+        dhq.dhq_forward(h, cd, ref)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        out = torch.zeros((w.n, 1), device="cuda")
+        with torch.cuda.stream(side):
+            dhq.dhq_forward(h, cd, out, stream=side)
+        side.synchronize()
+        assert torch.equal(out.view(torch.int32), ref.view(torch.int32))
+    finally:
+        dhq.dhq_destroy(h)
+
+
 def test_forward_host_buffers():
     w = dhq_inputs.WORKLOADS["C1"]
     weights, biases = w.network()
