@@ -140,7 +140,7 @@ def run_reference(args, workload):
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "int8 codes, int32 accumulate, fp64 epilogue", "data": "synthetic",
+        "vs_baseline": None, "dtype": "int8 (int64 accumulate, f64 epilogue)", "data": "synthetic",
         "config": {"workload": workload.name, "dims": list(workload.dims), "bits": [workload.w_bits, workload.a_bits]},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -243,7 +243,7 @@ def run_ours(args, workload):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int8 codes, int32 accumulate, fp32 epilogue",
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8 (int32 accumulate, f32 epilogue)",
             "data": "synthetic",
             "config": {"workload": workload.name, "dims": list(workload.dims), "coords_per_step": n,
                        "bits": [workload.w_bits, workload.a_bits], "w_gran": workload.w_gran,
