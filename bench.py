@@ -110,8 +110,20 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
-def time_oracle(workload, steps, warmup, sample_tokens, rotate=True):
-    """The CPU oracle, as it stands, on `sample_tokens` coordinates of the workload."""
+def work_per_coord(dims, rotate=True):
+    """Algorithmic work of the method per coordinate: int8 multiply-adds of all layers (the two
+    inputs padded to 4, the outputs of the last layer to 4), sines, and fp32 operations that only
+    the fp32 pipe can do (butterfly adds, dequantization fma, quantizer multiply, rounding add)."""
+    w, hidden_vectors, hidden_matmuls = dims[1], len(dims) - 2, len(dims) - 3
+    macs = 4 * w + hidden_matmuls * w * w + 4 * w
+    sines = hidden_vectors * w
+    fp32 = hidden_vectors * w * (3 + (int(np.log2(w)) if rotate else 0))
+    return macs, sines, fp32
+
+
+def time_oracle(workload, steps, warmup, sample_tokens, rotate=True, min_seconds=0.0):
+    """The CPU oracle, as it stands, on `sample_tokens` coordinates of the workload; with
+    min_seconds the passes repeat until that much CPU time has been measured."""
     from oracle import dhq_oracle as orc
     weights, biases = workload.network()
     net = orc.prepare(weights, biases, workload.dims, workload.omega0, workload.w_bits, workload.a_bits,
@@ -122,10 +134,12 @@ def time_oracle(workload, steps, warmup, sample_tokens, rotate=True):
     for _ in range(warmup):
         orc.forward(net, coords[: max(1, sample_tokens // 8)])
     t0 = time.perf_counter()
-    for _ in range(steps):
+    done = 0
+    while done < steps or time.perf_counter() - t0 < min_seconds:
         orc.forward(net, coords)
-    dt = (time.perf_counter() - t0) / steps
-    return coords.shape[0] / dt, dt, orc.threads()
+        done += 1
+    dt = (time.perf_counter() - t0) / done
+    return coords.shape[0] / dt, dt, orc.threads(), done
 
 
 def run_reference(args, workload):
@@ -135,7 +149,7 @@ def run_reference(args, workload):
     sample = min(workload.n, 16384)
     steps = max(1, min(args.steps, 5))
     warmup = min(args.warmup, 1)
-    value, dt, cores = time_oracle(workload, steps, warmup, sample, args.rotation == "input")
+    value, dt, cores, _ = time_oracle(workload, steps, warmup, sample, args.rotation == "input")
     desc = f"first {sample} coordinates of the {workload.grid[0]}x{workload.grid[1]} grid per step"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -250,7 +264,10 @@ def run_ours(args, workload):
                        "a_gran": workload.a_gran, "rotation": args.rotation, "l2": "flushed between steps (256 MB write)",
                        "parallelism": f"{world} independent replica(s)"},
             "clocks": clocks.summary(),
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * 8, "d2h_bytes_per_step": n * d_L * 4},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * 8, "d2h_bytes_per_step": n * d_L * 4,
+                    "ms_per_step": e2e_ms / args.steps,
+                    "route": "dhq_forward_host on pinned host buffers: the kernel reads the coordinates and writes "
+                             "the result over the host link through the buffers' device mapping, every step"},
             "gpu_launches": launches,
             "roofline": {"bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "Tlaneop/s",
                          "frac": achieved / alu_peak,
@@ -258,11 +275,25 @@ def run_ours(args, workload):
                          "peak_source": "148 SMs x 128 fp32 lanes x max SM clock (derived, not measured)"},
             "device_status": status,
         }
+        # The same launch against the other pipes' ceilings, each measured now on this GPU by the
+        # library's own micro-benchmarks (perfect-overlap model: each pipe alone).
+        macs, sines, fp32_ops = work_per_coord(workload.dims, args.rotation == "input")
+        per_s = n / (ms_per_step * 1e-3)
+        pipes = {}
+        for key, pipe, work in (("tensor_i8", "tensor_i8", 2.0 * macs), ("sfu_sine", "mufu_sin", float(sines)),
+                                ("fp32", "fadd", float(fp32_ops))):
+            try:
+                peak, _ = dhq.dhq_measure_pipe(pipe, 2000)
+                pipes[key] = {"achieved": work * per_s, "peak_measured": peak, "frac": work * per_s / peak,
+                              "unit": "op/s", "per_coord": work}
+            except Exception as exc:       # a failed micro-benchmark must not lose the bench line
+                pipes[key] = {"error": str(exc)}
+        line["pipes"] = pipes
         if world == 1 and not args.no_cpu_baseline:
             sample = min(n, 65536)
-            v, dt, cores = time_oracle(workload, 1, 1, sample, args.rotation == "input")
+            v, dt, cores, passes = time_oracle(workload, 1, 1, sample, args.rotation == "input", min_seconds=10.0)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                    "sample": f"first {sample} coordinates of the grid, one pass ({dt:.1f} s)"}
+                                    "sample": f"first {sample} coordinates of the grid, {passes} pass(es) of {dt:.1f} s"}
         print(json.dumps(line), flush=True)
     dhq.dhq_destroy(h)
     if world > 1:

@@ -142,10 +142,19 @@ DHQ_API dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n,
                                  void *stream);
 
 /*
- * As dhq_forward but with HOST buffers: copies coords to the device, runs the forward and
- * copies the result back, all enqueued on `stream` (pass pinned memory for the copies to be
- * asynchronous).  Uses staging buffers owned by the handle, grown on demand (this may allocate
- * and synchronize the first time a larger n is seen).
+ * As dhq_forward but with HOST buffers.  The call is ordered after earlier work on `stream`, and
+ * later work on `stream` waits for the result to be in out_host.
+ *   - Both buffers pinned (page-locked, e.g. cudaHostAlloc / cudaHostRegister) and the scales
+ *     already frozen: no staging and no copy call.  The fused kernel reads the coordinates and
+ *     writes the result through the buffers' device mapping, so the transfers over the host link
+ *     happen tile by tile inside the one launch, beside the arithmetic.
+ *   - Otherwise (pageable memory, or the first per-tensor call, which calibrates): the data is
+ *     staged in device buffers owned by the handle, grown on demand (this may allocate and
+ *     synchronize the first time a larger n is seen).  Larger n is cut into up to 8 launches, each
+ *     a whole number of tile rounds of the fused kernel, whose copies run on two streams owned
+ *     by the handle beside the kernels (streams and events are created on the first such call).
+ * Results do not depend on the route or the cut.  If a device-side wait times out in one launch,
+ * later launches of the same call still run; the status word read by dhq_last_status records it.
  */
 DHQ_API dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t n,
                                       float *out_host, void *stream);

@@ -116,6 +116,14 @@ void dhq_destroy(dhq_handle_t h)
     cudaFree(h->d_status);
     cudaFree(h->scratch[0]); cudaFree(h->scratch[1]);
     cudaFree(h->stage_in); cudaFree(h->stage_out);
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
+    if (h->ev_start) cudaEventDestroy(h->ev_start);
+    if (h->ev_done) cudaEventDestroy(h->ev_done);
+    for (int i = 0; i < dhq_handle_s::kHostChunks; ++i) {
+        if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+        if (h->ev_k[i]) cudaEventDestroy(h->ev_k[i]);
+    }
     delete h;
 }
 
@@ -272,6 +280,20 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     if (!h || n < 0 || (n > 0 && (!coords_host || !out_host))) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     cudaStream_t st = (cudaStream_t)stream;
+    // Pinned (page-locked, device-mapped) host buffers need no staging: the fused kernel reads the
+    // coordinates and writes the result through their device addresses, so the transfers happen
+    // inside the kernel, tile by tile, beside the arithmetic.  (Calibration reads the coordinates
+    // once per layer: it goes through the staged path below.)
+    if (h->calibrated && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
+        cudaPointerAttributes ai, ao;
+        void *di = nullptr, *dout = nullptr;
+        const bool mapped = cudaPointerGetAttributes(&ai, coords_host) == cudaSuccess && ai.type == cudaMemoryTypeHost &&
+                            cudaPointerGetAttributes(&ao, out_host) == cudaSuccess && ao.type == cudaMemoryTypeHost &&
+                            cudaHostGetDevicePointer(&di, const_cast<float *>(coords_host), 0) == cudaSuccess &&
+                            cudaHostGetDevicePointer(&dout, out_host, 0) == cudaSuccess && di && dout;
+        (void)cudaGetLastError(); // a failed query of pageable memory is not an error of this call
+        if (mapped) return fused_forward(h, static_cast<const float *>(di), n, static_cast<float *>(dout), st);
+    }
     if (n > h->stage_tokens) {
         CK(cudaDeviceSynchronize());
         cudaFree(h->stage_in); cudaFree(h->stage_out);
@@ -281,10 +303,55 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
             return DHQ_ERR_ALLOC;
         h->stage_tokens = n;
     }
-    CK(cudaMemcpyAsync(h->stage_in, coords_host, (size_t)n * 2 * sizeof(float), cudaMemcpyHostToDevice, st));
-    dhq_status_t s = dhq_forward(h, h->stage_in, n, h->stage_out, stream);
-    if (s != DHQ_OK) return s;
-    CK(cudaMemcpyAsync(out_host, h->stage_out, (size_t)n * h->d_L * sizeof(float), cudaMemcpyDeviceToHost, st));
+    // How many launches the call is cut into: each is a whole number of rounds of the fused kernel
+    // (one tile per slot of every SM), so that cutting costs only the launch prologue.
+    const int64_t round = fused_round_tokens(h);
+    const int64_t rounds = (n + round - 1) / round;
+    int chunks = (int)(rounds >= 16 ? 8 : rounds < 4 ? rounds : 4);
+    if (!h->calibrated) chunks = 1; // the first forward freezes the per-tensor scales on ALL of its coordinates
+    if (chunks <= 1) {
+        CK(cudaMemcpyAsync(h->stage_in, coords_host, (size_t)n * 2 * sizeof(float), cudaMemcpyHostToDevice, st));
+        dhq_status_t s = dhq_forward(h, h->stage_in, n, h->stage_out, stream);
+        if (s != DHQ_OK) return s;
+        CK(cudaMemcpyAsync(out_host, h->stage_out, (size_t)n * h->d_L * sizeof(float), cudaMemcpyDeviceToHost, st));
+        return DHQ_OK;
+    }
+    // Pipeline: the copy of chunk i+1 to the device and the copy of chunk i-1 back run on two
+    // streams of the handle beside the kernel of chunk i on the caller's stream.  The whole call
+    // is ordered after earlier work on `stream`, and `stream` ends up waiting for the last copy.
+    if (!h->pipe_ready) {
+        CK(cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking));
+        CK(cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking));
+        CK(cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&h->ev_done, cudaEventDisableTiming));
+        for (int i = 0; i < dhq_handle_s::kHostChunks; ++i) {
+            CK(cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
+            CK(cudaEventCreateWithFlags(&h->ev_k[i], cudaEventDisableTiming));
+        }
+        h->pipe_ready = true;
+    }
+    CK(cudaEventRecord(h->ev_start, st));
+    CK(cudaStreamWaitEvent(h->copy_in, h->ev_start, 0));
+    CK(cudaStreamWaitEvent(h->copy_out, h->ev_start, 0));
+    const int64_t base = rounds / chunks, extra = rounds % chunks;
+    int64_t t0 = 0;
+    for (int i = 0; i < chunks; ++i) {
+        int64_t cnt = (base + (i < extra ? 1 : 0)) * round;
+        if (cnt > n - t0) cnt = n - t0;
+        CK(cudaMemcpyAsync(h->stage_in + t0 * 2, coords_host + t0 * 2, (size_t)cnt * 2 * sizeof(float),
+                           cudaMemcpyHostToDevice, h->copy_in));
+        CK(cudaEventRecord(h->ev_in[i], h->copy_in));
+        CK(cudaStreamWaitEvent(st, h->ev_in[i], 0));
+        dhq_status_t s = fused_forward(h, h->stage_in + t0 * 2, cnt, h->stage_out + t0 * h->d_L, st);
+        if (s != DHQ_OK) return s;
+        CK(cudaEventRecord(h->ev_k[i], st));
+        CK(cudaStreamWaitEvent(h->copy_out, h->ev_k[i], 0));
+        CK(cudaMemcpyAsync(out_host + t0 * h->d_L, h->stage_out + t0 * h->d_L, (size_t)cnt * h->d_L * sizeof(float),
+                           cudaMemcpyDeviceToHost, h->copy_out));
+        t0 += cnt;
+    }
+    CK(cudaEventRecord(h->ev_done, h->copy_out));
+    CK(cudaStreamWaitEvent(st, h->ev_done, 0));
     return DHQ_OK;
 }
 

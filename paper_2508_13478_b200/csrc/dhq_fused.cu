@@ -905,6 +905,13 @@ void fused_destroy(dhq_handle_s *h)
     h->fused = nullptr;
 }
 
+int64_t fused_round_tokens(const dhq_handle_s *h)
+{
+    const FusedState *fs = static_cast<const FusedState *>(h->fused);
+    const int slots = (h->w == 512) ? 1 : 2;
+    return (int64_t)(fs ? fs->sm_count : 1) * slots * kTile;
+}
+
 dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st)
 {
     FusedState *fs = static_cast<FusedState *>(h->fused);

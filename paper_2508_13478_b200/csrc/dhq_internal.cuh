@@ -45,6 +45,11 @@ struct dhq_handle_s {
     int64_t scratch_tokens = 0;
     float *stage_in = nullptr, *stage_out = nullptr; // dhq_forward_host staging
     int64_t stage_tokens = 0;
+    // dhq_forward_host pipeline: copy streams and events, created on first use
+    static constexpr int kHostChunks = 8;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[kHostChunks] = {}, ev_k[kHostChunks] = {};
+    bool pipe_ready = false;
     int64_t launches = 0;
     void *fused = nullptr;          // state of the fused path (device parameter block)
 };
@@ -121,5 +126,8 @@ __host__ __device__ inline int fused_feature(int col, int W)
 dhq_status_t fused_create(dhq_handle_s *h);
 void fused_destroy(dhq_handle_s *h);
 dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st);
+// Coordinates one launch of the fused kernel works on at a time over the whole GPU (one tile per
+// slot of every SM): launches cut at multiples of this leave no SM idle.
+int64_t fused_round_tokens(const dhq_handle_s *h);
 
 } // namespace dhq

@@ -306,6 +306,58 @@ def test_forward_host_buffers():
         dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("name,n", [("C2", 65536), ("C2", 5 * 37888 + 777), ("C3", 17 * 37888 + 129), ("C5", 3 * 18944 + 1)])
+def test_forward_host_pinned_and_pageable(name, n):
+    """Host buffers with n spanning several tile rounds.  Pinned buffers are read and written by
+    the kernel itself through their device mapping; pageable buffers are staged and the call is
+    cut into launches whose copies overlap the kernels.  Either way the result must equal one
+    dhq_forward over device buffers: on the first call (which freezes per-tensor scales on all
+    coordinates) and on later ones, from the default stream and from a side stream."""
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h, _ = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        coords = w.coords()
+        reps = (n + coords.shape[0] - 1) // coords.shape[0]
+        coords = np.ascontiguousarray(np.tile(coords, (reps, 1))[:n])
+        d_L = w.dims[-1]
+        ch = torch.from_numpy(coords).pin_memory()
+        oh = torch.zeros((n, d_L)).pin_memory()
+        dhq.dhq_forward_host(h, ch, oh)                 # first call: calibrates (per tensor) on all of it
+        torch.cuda.synchronize()
+        ref = torch.empty((n, d_L), device="cuda")
+        dhq.dhq_forward(h, ch.cuda(), ref)
+        torch.cuda.synchronize()
+        ref_bits = ref.cpu().view(torch.int32)
+        assert torch.equal(oh.view(torch.int32), ref_bits)
+        oh.zero_()
+        before = dhq.dhq_launch_count(h)
+        dhq.dhq_forward_host(h, ch, oh)                 # pinned: one launch on the mapped buffers
+        torch.cuda.synchronize()
+        assert dhq.dhq_launch_count(h) - before == 1
+        assert torch.equal(oh.view(torch.int32), ref_bits)
+        side = torch.cuda.Stream()
+        oh.zero_()
+        with torch.cuda.stream(side):
+            dhq.dhq_forward_host(h, ch, oh, stream=side)
+        side.synchronize()
+        assert torch.equal(oh.view(torch.int32), ref_bits)
+        pageable = torch.zeros((n, d_L))
+        before = dhq.dhq_launch_count(h)
+        dhq.dhq_forward_host(h, torch.from_numpy(coords), pageable)     # staged, cut into launches
+        torch.cuda.synchronize()
+        assert dhq.dhq_launch_count(h) - before >= 2
+        assert torch.equal(pageable.view(torch.int32), ref_bits)
+        pageable.zero_()
+        with torch.cuda.stream(side):
+            dhq.dhq_forward_host(h, torch.from_numpy(coords), pageable, stream=side)
+        side.synchronize()
+        assert torch.equal(pageable.view(torch.int32), ref_bits)
+        assert dhq.dhq_last_status(h) == 0
+    finally:
+        dhq.dhq_destroy(h)
+
+
 def test_pipe_micro_benchmarks_run():
     for pipe in ("ffma", "mufu_sin", "tensor_i8"):
         ops, ms = dhq.dhq_measure_pipe(pipe, 200)
