@@ -288,6 +288,16 @@ def run_ours(args, workload):
                               "unit": "op/s", "per_coord": work}
             except Exception as exc:       # a failed micro-benchmark must not lose the bench line
                 pipes[key] = {"error": str(exc)}
+        if workload.dims[1] == 256:
+            # the kernel's own per-element loops (pass 1 + pass 2 of a hidden layer) run alone:
+            # what the arithmetic would reach with every wait hidden, in activation elements per second
+            try:
+                alone, _ = dhq.dhq_measure_pipe("pass12", 200)
+                elems = float((len(workload.dims) - 2) * workload.dims[1])
+                pipes["inner_loops_alone"] = {"achieved": elems * per_s, "peak_measured": alone, "frac": elems * per_s / alone,
+                                              "unit": "activation elements/s", "per_coord": elems}
+            except Exception as exc:
+                pipes["inner_loops_alone"] = {"error": str(exc)}
         line["pipes"] = pipes
         if world == 1 and not args.no_cpu_baseline:
             sample = min(n, 65536)

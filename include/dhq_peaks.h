@@ -29,7 +29,12 @@ typedef enum {
     DHQ_PIPE_FMNMX = 6,    /* fp32 min/max                                         */
     DHQ_PIPE_TENSOR_I8 = 7, /* tcgen05.mma kind::i8, 128x256x32, operands resident in shared memory */
     DHQ_PIPE_FADD2 = 8,    /* add.rn.f32x2: two fp32 adds per lane and instruction (counted as 2)   */
-    DHQ_PIPE_FFMA2 = 9     /* fma.rn.f32x2 (counted as 2)                                            */
+    DHQ_PIPE_FFMA2 = 9,    /* fma.rn.f32x2 (counted as 2)                                            */
+    /* The fused kernel's own per-element loops for a hidden layer of width 256, run alone (16 warps per
+     * SM, data in tensor memory, no MMA, no barrier, no tile loop); counted in activation elements:    */
+    DHQ_PIPE_PASS1 = 10,   /* dequantize + bias + sine + butterfly stages with stride < 64             */
+    DHQ_PIPE_PASS2 = 11,   /* butterfly stages 64 and 128 + quantizer + code stores to shared memory   */
+    DHQ_PIPE_PASS12 = 12   /* both, one after the other                                                */
 } dhq_pipe_t;
 
 /*
@@ -37,7 +42,7 @@ typedef enum {
  * `stream` after one warm-up launch; synchronizes.
  *   ops_per_s  host, receives operations per second: instructions x 32 lanes for the scalar
  *              pipes (an FMA counts as one), 2*M*N*K integer operations per MMA for the tensor
- *              pipe.
+ *              pipe, activation elements for the PASS loops.
  *   ms         host, receives the duration of the timed launch, or NULL.
  * Returns 0 on success, a negative value on a CUDA error or unknown pipe, 1 if the tensor-pipe
  * loop hit its bounded wait.

@@ -928,4 +928,103 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------- inner loops in isolation
+//
+// The per-element work of a hidden layer of width 256 without anything else the fused kernel
+// does: no MMA, no mbarrier, no tile loop.  16 warps per SM run, `iters` times, pass 1 (tensor
+// memory -> dequantize, sine, butterfly stages below 64 -> tensor memory), pass 2 (stages 64 and
+// 128, quantizer, code stores to shared memory) or both, each warp on its own lanes and columns
+// with the same functions and the same thread-to-data mapping as the kernel (R = 2).  The rate
+// this reaches is what the kernel's arithmetic could do if every wait were hidden.
+template <int WHICH> __global__ void __launch_bounds__(512, 1) pass_rate_kernel(int iters)
+{
+    constexpr int W = 256;
+    using C = Cfg<W>;
+    constexpr int CH = C::CH, NCH = C::NCH, G = C::G;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = ptx::smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *gen = smem_raw + (base - raw);
+    constexpr uint32_t kConsts = 2 * kTile * W, kHolder = kConsts + 3 * W * 4; // two A tiles, then cA | cB | cA_lo
+    float *cst = reinterpret_cast<float *>(gen + kConsts);
+    for (int i = threadIdx.x; i < 3 * W; i += blockDim.x) cst[i] = (i < W) ? 1e-5f : (i < 2 * W ? 0.3f : 0.f);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0) {
+        ptx::tmem_alloc(base + kHolder, 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(gen + kHolder);
+    const int quad = warp & 3, slot = warp >> 3, sub = (warp >> 2) & 1;
+    const uint32_t taddr = tmem + (uint32_t)(slot * C::TMEM_COLS_PER_SLOT) + ((uint32_t)(quad * 32) << 16);
+    {
+        uint32_t v[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) v[i] = (uint32_t)((lane * 37 + i * 11) % 2001 - 1000);
+        for (int cc = 0; cc < C::CPT; ++cc) tmem_st<CH>(taddr + (sub * C::CPT + cc) * CH, v);
+        ptx::tmem_wait_st();
+    }
+    __syncthreads();
+    for (int it = 0; it < iters; ++it) {
+        if (WHICH & 1) {
+#pragma unroll
+            for (int cc = 0; cc < C::CPT; ++cc) {
+                const int ch = sub * C::CPT + cc;
+                uint32_t v[CH];
+                tmem_ld<CH>(taddr + ch * CH, v);
+                ptx::tmem_wait_ld();
+                hidden_chunk<W, CH, false, true, EPI_SINE_FAST>(base + kConsts, ch * CH, 1.f, v);
+                tmem_st<CH>(taddr + ch * CH, v);
+            }
+            ptx::tmem_wait_st();
+        }
+        if (WHICH & 2) {
+#pragma unroll 1
+            for (int gg = 0; gg < C::GPT; ++gg) {
+                const int g = sub * C::GPT + gg;
+                uint32_t u[NCH][G];
+#pragma unroll
+                for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(taddr + ch * CH + g * G, u[ch]);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int h = 1; h < NCH; h <<= 1) {
+#pragma unroll
+                    for (int ch = 0; ch < NCH; ++ch) {
+                        if ((ch & h) == 0) {
+#pragma unroll
+                            for (int i = 0; i < G; i += 2) {
+                                f32x2 a = pack2u(u[ch][i], u[ch][i + 1]), b = pack2u(u[ch + h][i], u[ch + h][i + 1]);
+                                bfly2(a, b);
+                                unpack2u(a, u[ch][i], u[ch][i + 1]);
+                                unpack2u(b, u[ch + h][i], u[ch + h][i + 1]);
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int ch = 0; ch < NCH; ++ch)
+                    quantize_store<G, CH, true>(base + slot * (kTile * W), quad * 32 + lane, ch, g * G, u[ch], 1e-3f, 127.f);
+            }
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        ptx::tmem_dealloc(tmem, 512);
+    }
+}
+
+cudaError_t launch_pass_rate(int which, int sms, int iters, cudaStream_t st)
+{
+    const size_t smem = 2 * kTile * 256 + 3 * 256 * 4 + 64 + 1024 > (size_t)kMinSmem ? 2 * kTile * 256 + 3 * 256 * 4 + 64 + 1024 : (size_t)kMinSmem;
+    void (*fn)(int) = which == 1 ? pass_rate_kernel<1> : which == 2 ? pass_rate_kernel<2> : pass_rate_kernel<3>;
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    fn<<<sms, 512, smem, st>>>(iters);
+    return cudaGetLastError();
+}
+
 } // namespace dhq

@@ -129,5 +129,9 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
 // Coordinates one launch of the fused kernel works on at a time over the whole GPU (one tile per
 // slot of every SM): launches cut at multiples of this leave no SM idle.
 int64_t fused_round_tokens(const dhq_handle_s *h);
+// The fused kernel's per-element loops of a width-256 hidden layer in isolation (micro-benchmark):
+// which = 1 pass 1, 2 pass 2, 3 both; one block of 16 warps on each of `sms` SMs.  Each iteration
+// covers 256 tokens x 256 activation elements per SM.
+cudaError_t launch_pass_rate(int which, int sms, int iters, cudaStream_t st);
 
 } // namespace dhq

@@ -1,6 +1,7 @@
 // Micro-benchmarks of the pipes that bound the fused kernel (see include/dhq_peaks.h).
 #include <cuda_runtime.h>
 #include "../../include/dhq_peaks.h"
+#include "dhq_internal.cuh"
 #include "dhq_tmem.cuh"
 
 namespace dhq {
@@ -137,6 +138,9 @@ extern "C" int dhq_measure_pipe(int pipe, int iters, void *stream, double *ops_p
                 e = cudaGetLastError();
             }
             break;
+        case DHQ_PIPE_PASS1: e = launch_pass_rate(1, sms, iters, st); break;
+        case DHQ_PIPE_PASS2: e = launch_pass_rate(2, sms, iters, st); break;
+        case DHQ_PIPE_PASS12: e = launch_pass_rate(3, sms, iters, st); break;
         default: rc = -4;
         }
         if (e != cudaSuccess) rc = -5;
@@ -151,6 +155,8 @@ extern "C" int dhq_measure_pipe(int pipe, int iters, void *stream, double *ops_p
             cudaMemcpy(&flag, sink, sizeof(int), cudaMemcpyDeviceToHost);
             if (flag) rc = 1;
             ops = (double)sms * iters * 8.0 * 2.0 * 128 * 256 * 32;
+        } else if (pipe == DHQ_PIPE_PASS1 || pipe == DHQ_PIPE_PASS2 || pipe == DHQ_PIPE_PASS12) {
+            ops = (double)sms * iters * 256.0 * 256.0; // activation elements: two tiles of 128 tokens x 256 per SM and iteration
         } else {
             double per_thread = (double)iters * 8 * kChains * ((pipe == DHQ_PIPE_FMNMX || pipe == DHQ_PIPE_FADD2 || pipe == DHQ_PIPE_FFMA2) ? 2 : 1);
             ops = per_thread * 256.0 * blocks;

@@ -359,6 +359,6 @@ def test_forward_host_pinned_and_pageable(name, n):
 
 
 def test_pipe_micro_benchmarks_run():
-    for pipe in ("ffma", "mufu_sin", "tensor_i8"):
+    for pipe in ("ffma", "mufu_sin", "tensor_i8", "pass1", "pass2", "pass12"):
         ops, ms = dhq.dhq_measure_pipe(pipe, 200)
         assert ops > 1e11 and ms > 0
