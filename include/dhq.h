@@ -128,6 +128,30 @@ DHQ_API dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W,
 DHQ_API dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void *stream);
 
 /*
+ * The same calibration one layer at a time, for coordinate sets that are spread over several
+ * GPUs (coordinates are independent, Section III: f_theta maps each x to its y; each GPU holds a
+ * replica of the handle and a part of the set).  The frozen value of layer l is the maximum over
+ * ALL parts, and layer l+1 may only be measured once layer l is frozen, so the caller alternates,
+ * for l = 1..L:
+ *   dhq_calibrate_layer(h, l, part, n_part, stream)   measure this part: max |H_K x_l| into the handle;
+ *   dhq_get_act_absmax(h, l, &a, stream)              read it (synchronizes the stream);
+ *   a = maximum of a over the parts                   (one float: an all-reduce(max), or a host loop);
+ *   dhq_set_act_absmax(h, l, a, stream)               freeze layer l: scales and epilogue constants.
+ * After layer L the handle is calibrated exactly as by dhq_calibrate on the whole set (the
+ * maximum of non-negative floats does not depend on how the set was split).  n_part = 0 is
+ * allowed and contributes 0.  dhq_calibrate_layer(l) needs layers < l frozen (by this sequence or
+ * an earlier calibration): otherwise NOT_CALIBRATED.  Starting the sequence marks the handle as
+ * not calibrated until layer L is set.  With per-token activation scales all three are no-ops
+ * (dhq_get_act_absmax then returns whatever the handle holds).
+ *   absmax  host pointer (get) / finite value >= 0 (set).
+ * Errors: INVALID_ARG, NOT_CALIBRATED, ALLOC, CUDA.
+ */
+DHQ_API dhq_status_t dhq_calibrate_layer(dhq_handle_t h, int layer, const float *coords, int64_t n,
+                                         void *stream);
+DHQ_API dhq_status_t dhq_get_act_absmax(dhq_handle_t h, int layer, float *absmax, void *stream);
+DHQ_API dhq_status_t dhq_set_act_absmax(dhq_handle_t h, int layer, float absmax, void *stream);
+
+/*
  * The forward pass f_theta over n coordinates: one launch of the fused kernel, activations
  * never leave the SM between layers.
  *   coords device [n][2] fp32 (x, y per token), 8-byte aligned.

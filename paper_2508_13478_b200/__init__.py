@@ -7,8 +7,9 @@ functions raises.
 """
 from .binding import (  # noqa: F401
     DHQ_GRAN_TENSOR, DHQ_GRAN_CHANNEL_OR_TOKEN, DHQ_ROT_INPUT, DhqError, PIPES,
-    dhq_prepare, dhq_calibrate, dhq_forward, dhq_forward_host, dhq_forward_debug, dhq_forward_static_scratch,
+    dhq_prepare, dhq_calibrate, dhq_calibrate_layer, dhq_get_act_absmax, dhq_set_act_absmax, dhq_forward, dhq_forward_host, dhq_forward_debug, dhq_forward_static_scratch,
     DHQ_STATIC_MAX_TOKENS, dhq_get_layer,
     dhq_layer_dims, dhq_last_status, dhq_launch_count, dhq_destroy, dhq_status_string,
     dhq_measure_pipe, library_path, load_library,
 )
+from .sharded import calibrate_sharded, shard_range  # noqa: F401,E402

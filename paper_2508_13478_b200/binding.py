@@ -61,6 +61,9 @@ def load_library():
     vp, c_i, c_i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
     L.dhq_prepare.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(vp), ctypes.POINTER(vp), vp, ctypes.POINTER(vp)]
     L.dhq_calibrate.argtypes = [vp, vp, c_i64, vp]
+    L.dhq_calibrate_layer.argtypes = [vp, c_i, vp, c_i64, vp]
+    L.dhq_get_act_absmax.argtypes = [vp, c_i, ctypes.POINTER(ctypes.c_float), vp]
+    L.dhq_set_act_absmax.argtypes = [vp, c_i, ctypes.c_float, vp]
     L.dhq_forward.argtypes = [vp, vp, c_i64, vp, vp]
     L.dhq_forward_host.argtypes = [vp, vp, c_i64, vp, vp]
     L.dhq_forward_static_scratch.argtypes = [vp, vp, c_i64, vp, vp]
@@ -76,6 +79,8 @@ def load_library():
     L.dhq_status_string.argtypes = [c_i]
     L.dhq_status_string.restype = ctypes.c_char_p
     L.dhq_measure_pipe.argtypes = [c_i, c_i, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    for name in ("dhq_calibrate_layer", "dhq_get_act_absmax", "dhq_set_act_absmax"):
+        getattr(L, name).restype = c_i
     for name in ("dhq_prepare", "dhq_calibrate", "dhq_forward", "dhq_forward_host", "dhq_forward_debug",
                  "dhq_get_layer", "dhq_layer_dims", "dhq_last_status", "dhq_measure_pipe"):
         getattr(L, name).restype = c_i
@@ -124,6 +129,24 @@ def dhq_calibrate(handle, coords, stream=None):
     n = coords.shape[0]
     _check(load_library().dhq_calibrate(handle, _dev_ptr(coords, torch.float32, "coords"), n, _stream_ptr(stream)),
            "dhq_calibrate")
+
+
+def dhq_calibrate_layer(handle, layer, coords, stream=None):
+    """Measure layer `layer` (1-based) on this part of the calibration set; coords may be empty."""
+    n = 0 if coords is None else coords.shape[0]
+    ptr = _dev_ptr(coords, torch.float32, "coords") if n else None
+    _check(load_library().dhq_calibrate_layer(handle, int(layer), ptr, n, _stream_ptr(stream)), "dhq_calibrate_layer")
+
+
+def dhq_get_act_absmax(handle, layer, stream=None) -> float:
+    a = ctypes.c_float()
+    _check(load_library().dhq_get_act_absmax(handle, int(layer), ctypes.byref(a), _stream_ptr(stream)), "dhq_get_act_absmax")
+    return float(a.value)
+
+
+def dhq_set_act_absmax(handle, layer, absmax, stream=None):
+    _check(load_library().dhq_set_act_absmax(handle, int(layer), ctypes.c_float(float(absmax)), _stream_ptr(stream)),
+           "dhq_set_act_absmax")
 
 
 def dhq_forward(handle, coords, out, stream=None):

@@ -62,29 +62,39 @@ LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X
     return a;
 }
 
-dhq_status_t calibrate_impl(dhq_handle_s *h, const float *coords, int64_t n, cudaStream_t st)
+// One calibration pass: the maximum of |rotated input of layer l| over the given coordinates, with
+// layers < l run as they are frozen, is left in the layer's act[0] (not yet turned into scales).
+dhq_status_t calibrate_layer_pass(dhq_handle_s *h, int l, const float *coords, int64_t n, cudaStream_t st)
 {
     const int64_t chunk = n < kDebugChunk ? n : kDebugChunk;
     dhq_status_t s = ensure_scratch(h, chunk);
     if (s != DHQ_OK) return s;
-    for (int l = 1; l <= h->L; ++l) {
-        LayerDev &d = h->layer[l - 1];
-        CK(cudaMemsetAsync(d.act, 0, 4 * sizeof(float), st));
-        for (int64_t t0 = 0; t0 < n; t0 += chunk) {
-            int64_t cnt = n - t0 < chunk ? n - t0 : chunk;
-            const float *X = nullptr;
-            for (int j = 1; j <= l; ++j) {
-                LayerArgs a = layer_args(h, j, coords + t0 * 2, X, cnt);
-                if (j == l) a.calib_only = 1;
-                else a.Y = h->scratch[(j - 1) & 1];
-                CK(launch_layer(a, st));
-                h->launches++;
-                X = a.Y;
-            }
+    LayerDev &d = h->layer[l - 1];
+    CK(cudaMemsetAsync(d.act, 0, 4 * sizeof(float), st));
+    for (int64_t t0 = 0; t0 < n; t0 += chunk) {
+        int64_t cnt = n - t0 < chunk ? n - t0 : chunk;
+        const float *X = nullptr;
+        for (int j = 1; j <= l; ++j) {
+            LayerArgs a = layer_args(h, j, coords + t0 * 2, X, cnt);
+            if (j == l) a.calib_only = 1;
+            else a.Y = h->scratch[(j - 1) & 1];
+            CK(launch_layer(a, st));
+            h->launches++;
+            X = a.Y;
         }
-        CK(launch_finalize(d, h->cfg.a_bits, 0, l < h->L, (double)h->cfg.omega0, st, &h->launches));
+    }
+    return DHQ_OK;
+}
+
+dhq_status_t calibrate_impl(dhq_handle_s *h, const float *coords, int64_t n, cudaStream_t st)
+{
+    for (int l = 1; l <= h->L; ++l) {
+        dhq_status_t s = calibrate_layer_pass(h, l, coords, n, st);
+        if (s != DHQ_OK) return s;
+        CK(launch_finalize(h->layer[l - 1], h->cfg.a_bits, 0, l < h->L, (double)h->cfg.omega0, st, &h->launches));
     }
     h->calibrated = true;
+    h->calib_layers_done = h->L;
     return DHQ_OK;
 }
 
@@ -226,6 +236,43 @@ dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void 
     if (!h || !coords || n < 1) return DHQ_ERR_INVALID_ARG;
     if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
     return calibrate_impl(h, coords, n, (cudaStream_t)stream);
+}
+
+dhq_status_t dhq_calibrate_layer(dhq_handle_t h, int layer, const float *coords, int64_t n, void *stream)
+{
+    if (!h || layer < 1 || layer > h->L || n < 0 || (n > 0 && !coords)) return DHQ_ERR_INVALID_ARG;
+    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
+    if (layer > h->calib_layers_done + 1) return DHQ_ERR_NOT_CALIBRATED; // layers before it are not frozen yet
+    h->calibrated = false;
+    h->calib_layers_done = layer - 1;
+    if (n == 0) { // a rank without coordinates contributes the neutral element
+        CK(cudaMemsetAsync(h->layer[layer - 1].act, 0, 4 * sizeof(float), (cudaStream_t)stream));
+        return DHQ_OK;
+    }
+    return calibrate_layer_pass(h, layer, coords, n, (cudaStream_t)stream);
+}
+
+dhq_status_t dhq_get_act_absmax(dhq_handle_t h, int layer, float *absmax, void *stream)
+{
+    if (!h || layer < 1 || layer > h->L || !absmax) return DHQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    CK(cudaMemcpyAsync(absmax, h->layer[layer - 1].act, sizeof(float), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_set_act_absmax(dhq_handle_t h, int layer, float absmax, void *stream)
+{
+    if (!h || layer < 1 || layer > h->L || !(absmax >= 0.0f) || std::isinf(absmax)) return DHQ_ERR_INVALID_ARG;
+    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
+    if (layer > h->calib_layers_done + 1) return DHQ_ERR_NOT_CALIBRATED;
+    cudaStream_t st = (cudaStream_t)stream;
+    CK(cudaMemcpyAsync(h->layer[layer - 1].act, &absmax, sizeof(float), cudaMemcpyHostToDevice, st));
+    CK(cudaStreamSynchronize(st)); // `absmax` lives on this call's stack
+    CK(launch_finalize(h->layer[layer - 1], h->cfg.a_bits, 0, layer < h->L, (double)h->cfg.omega0, st, &h->launches));
+    h->calib_layers_done = layer;
+    h->calibrated = layer == h->L;
+    return DHQ_OK;
 }
 
 dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int64_t n, float *out,

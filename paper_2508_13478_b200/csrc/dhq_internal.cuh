@@ -39,6 +39,7 @@ struct dhq_handle_s {
     int L = 0, w = 0, d_L = 0;
     int device = 0;
     bool calibrated = false;
+    int calib_layers_done = 0;      // layers whose per-tensor activation scale is frozen (sharded calibration)
     dhq::LayerDev layer[dhq::kMaxLayers];
     int *d_status = nullptr;        // device status word
     float *scratch[2] = {nullptr, nullptr}; // ping-pong activations of the layer-by-layer path

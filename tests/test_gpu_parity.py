@@ -358,6 +358,57 @@ def test_forward_host_pinned_and_pageable(name, n):
         dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("name,parts", [("C2", 2), ("C1", 3)])
+def test_sharded_calibration_equals_whole_set(name, parts):
+    """The coordinate set split into contiguous blocks, one handle per block (as one GPU each would
+    hold), layer-by-layer calibration with the maximum exchanged on the host: the frozen values and
+    the outputs must equal, bit for bit, those of one handle calibrated on the whole set.  One
+    block is left empty on purpose in the three-way split."""
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    coords = w.coords()
+    L = len(w.dims) - 1
+    whole, _ = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, 0)
+    handles = [prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, 0)[0] for _ in range(parts)]
+    try:
+        cd = to_dev(coords)
+        dhq.dhq_calibrate(whole, cd)
+        if parts == 3:
+            bounds = [(0, 1000), (1000, 1000), (1000, w.n)]
+        else:
+            bounds = [dhq.shard_range(w.n, r, parts) for r in range(parts)]
+        blocks = [cd[lo:hi].contiguous() for lo, hi in bounds]
+        with pytest.raises(dhq.DhqError):
+            dhq.dhq_calibrate_layer(handles[0], 2, blocks[0])       # layer 1 is not frozen yet
+        for l in range(1, L + 1):
+            for h, blk in zip(handles, blocks):
+                dhq.dhq_calibrate_layer(h, l, blk)
+            a = max(dhq.dhq_get_act_absmax(h, l) for h in handles)
+            for h in handles:
+                dhq.dhq_set_act_absmax(h, l, a)
+        ref = torch.empty((w.n, w.dims[-1]), device="cuda")
+        dhq.dhq_forward(whole, cd, ref)
+        for h in handles:
+            for l in range(1, L + 1):
+                assert np.float32(dhq.dhq_get_layer(h, l)[2]).view(np.uint32) == np.float32(dhq.dhq_get_layer(whole, l)[2]).view(np.uint32)
+            out = torch.empty((w.n, w.dims[-1]), device="cuda")
+            dhq.dhq_forward(h, cd, out)
+            torch.cuda.synchronize()
+            assert torch.equal(out.view(torch.int32), ref.view(torch.int32))
+            assert dhq.dhq_last_status(h) == 0
+        # the helper with a host-side maximum over the emulated ranks gives the same values
+        again = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, 0)[0]
+        handles.append(again)
+        others = {l: dhq.dhq_get_layer(whole, l)[2] for l in range(1, L + 1)}
+        layer_no = iter(range(1, L + 1))
+        frozen = dhq.calibrate_sharded(again, blocks[0], L, allreduce_max=lambda v: max(v, others[next(layer_no)]))
+        assert [np.float32(v) for v in frozen] == [np.float32(others[l]) for l in range(1, L + 1)]
+    finally:
+        dhq.dhq_destroy(whole)
+        for h in handles:
+            dhq.dhq_destroy(h)
+
+
 def test_pipe_micro_benchmarks_run():
     for pipe in ("ffma", "mufu_sin", "tensor_i8", "pass1", "pass2", "pass12"):
         ops, ms = dhq.dhq_measure_pipe(pipe, 200)
