@@ -15,6 +15,11 @@
  *     s = a/qmax and inv = qmax/a both as IEEE fp32 divisions, q = clamp(rint(fl32(v*inv))) with
  *     round-half-to-even, a = 0 giving s = inv = 0.
  *   - The output layer has no activation (Section III-C); hidden layers apply sin(omega0 * z).
+ *   - rotate = 2 is the two-sided transform of Eq. 4-5 taken literally: W~ = H_M W H_K / (K M)
+ *     (rows rotated first, then columns, both as pinned fp32 pairwise sums, both scales exact
+ *     powers of two), and since H_M H_M = M I the layer output is z = H_M d + b with
+ *     d_m = s_w[m] s_x acc_m.  That second rotation decides no integer, so it is an explicit
+ *     fp64 matrix product.
  *
  * Parity pins (tests/test_oracle_*.py): Hadamard recursion vs closed form and H H^T = nI;
  * rotation vs an exact integer product and vs fp64; W x = (W H/K)(H x); Frobenius norm
@@ -155,7 +160,8 @@ ORC_API void dhq_orc_quantize(const float *v, int64_t count, float inv, int bits
 
 /*
  * Weight side (Eq. 4-5, input-side factor): pad W[d_out][d_in] with zeros to [M_pad][K_pad],
- * rotate each row (rotate != 0), scale by the exact 1/K_pad, quantize per tensor
+ * rotate each row (rotate != 0), scale by the exact 1/K_pad, for rotate = 2 also rotate each column
+ * and scale by the exact 1/M_pad, quantize per tensor
  * (per_channel = 0) or per output row.  Outputs: Wrot [M_pad][K_pad] fp32, q [M_pad][K_pad],
  * s_w [M_pad] (per-tensor: the same value repeated).
  */
@@ -180,6 +186,22 @@ ORC_API int dhq_orc_prepare_layer(const float *W, int d_out, int d_in, int M_pad
         for (size_t i = 0; i < cnt; ++i) Wrot[i] = Wrot[i] * invK;
     } else {
         memcpy(Wrot, padded, cnt * sizeof(float));
+    }
+    if (rotate == 2) {
+        /* output-side factor of Eq. 4: every column k becomes Tree(H_M column_k) / M */
+        int8_t *HM = (int8_t *)malloc((size_t)M_pad * M_pad);
+        float *colT = (float *)malloc(cnt * sizeof(float)), *rotT = (float *)malloc(cnt * sizeof(float));
+        if (!HM || !colT || !rotT || dhq_orc_hadamard(M_pad, HM) != 0) {
+            free(HM); free(colT); free(rotT); free(padded); free(H);
+            return -2;
+        }
+        for (int m = 0; m < M_pad; ++m)
+            for (int k = 0; k < K_pad; ++k) colT[(size_t)k * M_pad + m] = Wrot[(size_t)m * K_pad + k];
+        dhq_orc_rotate_rows(HM, M_pad, K_pad, colT, rotT);
+        float invM = 1.0f / (float)M_pad; /* power of two: exact */
+        for (int m = 0; m < M_pad; ++m)
+            for (int k = 0; k < K_pad; ++k) Wrot[(size_t)m * K_pad + k] = rotT[(size_t)k * M_pad + m] * invM;
+        free(HM); free(colT); free(rotT);
     }
     if (per_channel) {
         for (int m = 0; m < M_pad; ++m) {
@@ -231,6 +253,7 @@ ORC_API void dhq_orc_rotated_absmax(const float *X, int64_t n, int K_pad, int ro
  *   acc[m] = sum_k q[k] * qw[m][k]         -> acc   [n][M_pad] int64 (exact)
  *   z = s_w[m] * s_x * acc + b[m] in fp64; Y = sin(omega0 z) for hidden layers, z for the last
  *                                          -> Y     [n][M_pad] fp64
+ *   rotate = 2: z = H_M (s_w s_x acc) + b instead (fp64 matrix product)
  * Any output pointer may be NULL.  Returns 0, or -3 if an accumulator leaves the int32 range.
  */
 ORC_API int dhq_orc_layer(const float *X, int64_t n, int K_pad, int M_pad, const int32_t *qw,
@@ -239,8 +262,10 @@ ORC_API int dhq_orc_layer(const float *X, int64_t n, int K_pad, int M_pad, const
                           int32_t *codes, float *s_x, int64_t *acc, double *Y)
 {
     int8_t *H = (int8_t *)malloc((size_t)K_pad * K_pad);
-    if (!H || dhq_orc_hadamard(K_pad, H) != 0) {
+    int8_t *HM = (int8_t *)malloc((size_t)M_pad * M_pad);
+    if (!H || !HM || dhq_orc_hadamard(K_pad, H) != 0 || dhq_orc_hadamard(M_pad, HM) != 0) {
         free(H);
+        free(HM);
         return -2;
     }
     int overflow = 0;
@@ -249,6 +274,7 @@ ORC_API int dhq_orc_layer(const float *X, int64_t n, int K_pad, int M_pad, const
         float *scratch = (float *)malloc(sizeof(float) * (size_t)K_pad);
         float *xr = (float *)malloc(sizeof(float) * (size_t)K_pad);
         int32_t *q = (int32_t *)malloc(sizeof(int32_t) * (size_t)K_pad);
+        double *dq = (double *)malloc(sizeof(double) * (size_t)M_pad);
 #pragma omp for schedule(static)
         for (int64_t t = 0; t < n; ++t) {
             const float *x = X + t * K_pad;
@@ -270,16 +296,30 @@ ORC_API int dhq_orc_layer(const float *X, int64_t n, int K_pad, int M_pad, const
                     overflow = 1;
                 }
                 if (acc) acc[t * M_pad + m] = sum;
-                if (Y) {
+                if (rotate == 2) {
+                    dq[m] = (double)s_w[m] * (double)s * (double)sum; /* still in the rotated output basis */
+                } else if (Y) {
                     double z = (double)s_w[m] * (double)s * (double)sum + (double)b_pad[m];
                     Y[t * M_pad + m] = apply_sine ? sin(omega0 * z) : z;
+                }
+            }
+            if (rotate == 2 && Y) {
+                /* z = H_M d + b: undoes the output-side factor of W~ (H_M H_M = M I, the 1/M is in W~) */
+                for (int j = 0; j < M_pad; ++j) {
+                    const int8_t *hr = HM + (size_t)j * M_pad;
+                    double z = 0.0;
+                    for (int m = 0; m < M_pad; ++m) z += (hr[m] > 0) ? dq[m] : -dq[m];
+                    z += (double)b_pad[j];
+                    Y[t * M_pad + j] = apply_sine ? sin(omega0 * z) : z;
                 }
             }
         }
         free(scratch);
         free(xr);
         free(q);
+        free(dq);
     }
     free(H);
+    free(HM);
     return overflow ? -3 : 0;
 }

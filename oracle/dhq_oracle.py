@@ -142,12 +142,20 @@ class OracleNet:
     a_bits: int
     w_gran: int
     a_gran: int
-    rotate: bool
+    rotate: int           # 0: none, 1: input side (the hot path), 2: both sides (Eq. 4-5 literally)
     layers: list
 
 
+def _rot_mode(rotate) -> int:
+    if rotate in ("both", 2) and rotate is not True:
+        return 2
+    return int(bool(rotate))
+
+
 def prepare(weights, biases, dims, omega0, w_bits=8, a_bits=8, w_gran=0, a_gran=0, rotate=True) -> OracleNet:
-    """Weight-side fold and quantizer for every layer (Eq. 4-5, input-side factor)."""
+    """Weight-side fold and quantizer for every layer (Eq. 4-5: rotate=True the input-side factor,
+    rotate="both" the two-sided transform, rotate=False none)."""
+    mode = _rot_mode(rotate)
     L = len(dims) - 1
     layers = []
     for l in range(1, L + 1):
@@ -158,13 +166,13 @@ def prepare(weights, biases, dims, omega0, w_bits=8, a_bits=8, w_gran=0, a_gran=
         qw = np.empty((M_pad, K_pad), dtype=np.int32)
         s_w = np.empty(M_pad, dtype=np.float32)
         rc = lib().dhq_orc_prepare_layer(_p(W), d_out, d_in, M_pad, K_pad, w_bits, int(w_gran),
-                                         int(bool(rotate)), _p(Wrot), _p(qw), _p(s_w))
+                                         mode, _p(Wrot), _p(qw), _p(s_w))
         if rc != 0:
             raise RuntimeError(f"oracle prepare failed ({rc})")
         b_pad = np.zeros(M_pad, dtype=np.float32)
         b_pad[:d_out] = _f32(biases[l - 1])
         layers.append(OracleLayer(K_pad, M_pad, Wrot, qw, s_w, b_pad, sine=(l < L)))
-    return OracleNet(tuple(dims), float(omega0), w_bits, a_bits, int(w_gran), int(a_gran), bool(rotate), layers)
+    return OracleNet(tuple(dims), float(omega0), w_bits, a_bits, int(w_gran), int(a_gran), mode, layers)
 
 
 def pad_coords(coords) -> np.ndarray:
@@ -180,7 +188,7 @@ def rotated_absmax(net: OracleNet, l: int, X) -> np.ndarray:
     X = _f32(X)
     lay = net.layers[l - 1]
     amax = np.empty(X.shape[0], dtype=np.float32)
-    lib().dhq_orc_rotated_absmax(_p(X), X.shape[0], lay.K_pad, int(net.rotate), _p(amax))
+    lib().dhq_orc_rotated_absmax(_p(X), X.shape[0], lay.K_pad, int(net.rotate != 0), _p(amax))
     return amax
 
 

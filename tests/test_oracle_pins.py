@@ -328,3 +328,71 @@ def test_synthetic_inputs_have_the_distributions_the_paper_describes():
     assert (np.abs(y) > 0.8).mean() > (np.abs(y) < 0.2).mean()
     # generator self-check against the published first output of splitmix64 with seed 0
     assert int(dhq_inputs.splitmix64(0, 0, 1)[0]) == 0xE220A8397B1DCDAF
+
+
+# ---------------------------------------------------------------- two-sided transform (Eq. 4-5 literally)
+
+@pytest.mark.parametrize("shape", [(64, 2), (64, 64), (3, 256), (256, 256)])
+def test_two_sided_weight_transform_matches_eq5_and_keeps_the_product(shape):
+    d_out, d_in = shape
+    rng = np.random.default_rng(d_out * 77 + d_in)
+    W = rng.uniform(-0.1, 0.1, size=shape).astype(np.float32)
+    if d_in == 2:
+        weights, biases, dims, l = [W, np.zeros((1, d_out), np.float32)], [np.zeros(d_out, np.float32), np.zeros(1, np.float32)], (2, d_out, 1), 1
+    elif d_out <= 4:
+        weights, biases, dims, l = [np.zeros((d_in, 2), np.float32), W], [np.zeros(d_in, np.float32), np.zeros(d_out, np.float32)], (2, d_in, d_out), 2
+    else:
+        weights = [np.zeros((d_in, 2), np.float32), W, np.zeros((1, d_out), np.float32)]
+        biases = [np.zeros(d_in, np.float32), np.zeros(d_out, np.float32), np.zeros(1, np.float32)]
+        dims, l = (2, d_in, d_out, 1), 2
+    lay = orc.prepare(weights, biases, dims, 30.0, rotate="both").layers[l - 1]
+    K, M = lay.K_pad, lay.M_pad
+    Wp = np.zeros((M, K))
+    Wp[:d_out, :d_in] = W
+    Wrot = lay.Wrot.astype(np.float64)
+    # Eq. 5: W' = H_M W H_K / sqrt(M K); the oracle holds W' / sqrt(M K) (exact powers of two folded in)
+    assert np.allclose(Wrot * math.sqrt(M * K), odef.transform_2d(Wp), atol=2e-6)
+    # energy preservation (the sentence after Eq. 5)
+    assert math.isclose(np.linalg.norm(Wrot) * math.sqrt(M * K), np.linalg.norm(Wp), rel_tol=1e-5)
+    # the layer's product survives: H_M (W~ (H_K x)) = W x
+    x = rng.uniform(-1, 1, size=K)
+    x[d_in:] = 0
+    Wt = odef.transform_2d(Wp) / math.sqrt(M * K)
+    assert np.allclose(odef.hadamard(M) @ (Wt @ (odef.hadamard(K) @ x)), Wp @ x, rtol=1e-12, atol=1e-13)
+    # one-sided and two-sided folds differ exactly by the output-side factor
+    one = orc.prepare(weights, biases, dims, 30.0, rotate=True).layers[l - 1].Wrot.astype(np.float64)
+    assert np.allclose(Wrot, odef.hadamard(M) @ one / M, atol=1e-7)
+
+
+def test_two_sided_layer_brute_force_with_exact_rationals():
+    # 2 -> 4 -> 4, 3-bit codes, per-token scales: every stage recomputed with Python integers
+    # and Fractions from the oracle's own codes and scales; the second rotation must be applied
+    # to the dequantized values, before the bias.
+    rng = np.random.default_rng(11)
+    weights = [rng.uniform(-0.5, 0.5, (4, 2)).astype(np.float32), rng.uniform(-0.3, 0.3, (4, 4)).astype(np.float32)]
+    biases = [rng.uniform(-0.2, 0.2, 4).astype(np.float32), rng.uniform(-0.2, 0.2, 4).astype(np.float32)]
+    net = orc.prepare(weights, biases, (2, 4, 4), 30.0, w_bits=3, a_bits=3, a_gran=1, rotate="both")
+    H = closed_form(4)
+    X = rng.uniform(-1, 1, (50, 4)).astype(np.float32)
+    r = orc.layer(net, 2, X, want=("codes", "s_x", "acc", "Y"))
+    lay = net.layers[1]
+    for t in range(X.shape[0]):
+        q = [int(v) for v in r["codes"][t]]
+        acc = [sum(q[k] * int(lay.qw[m][k]) for k in range(4)) for m in range(4)]
+        assert acc == [int(v) for v in r["acc"][t]]
+        d = [Fraction(float(lay.s_w[m])) * Fraction(float(r["s_x"][t])) * acc[m] for m in range(4)]
+        for j in range(4):
+            z = sum(int(H[j][m]) * d[m] for m in range(4)) + Fraction(float(lay.b_pad[j]))
+            assert abs(float(z) - r["Y"][t][j]) <= 1e-15 * max(1.0, abs(float(z)))
+
+
+def test_two_sided_network_converges_to_the_unquantized_siren():
+    # the same limit as for the one-sided fold: a misplaced second rotation, a wrong scale (1/M), a
+    # bias added before the rotation or a rotated last layer leaves an error that does not shrink.
+    e8, _ = _net_error(8, rotate="both")
+    e12, _ = _net_error(12, rotate="both")
+    e16, g16 = _net_error(16, rotate="both")
+    assert e16 < 2e-4 and e12 < 4e-3
+    assert e12 < e8 / 4 and e16 < e12 / 4
+    _, g16_one = _net_error(16, rotate=True)
+    assert np.abs(g16 - g16_one).max() < 1e-3
