@@ -40,6 +40,11 @@ SM_COUNT = 148
 FP32_LANES_PER_SM = 128
 
 
+def rotations(mode: str) -> int:
+    """Hadamard rotations per hidden activation vector: 0 (none), 1 (input side), 2 (both sides)."""
+    return {"none": 0, "input": 1, "both": 2}[mode]
+
+
 def alu_laneops_per_coord(dims, rotate=True) -> float:
     """Plain-ALU lane operations the method needs per coordinate: per element of every hidden
     activation vector log2(w) butterfly adds (none without the rotation) plus 7 (int->float,
@@ -47,7 +52,7 @@ def alu_laneops_per_coord(dims, rotate=True) -> float:
     packing/abs-max)."""
     w = dims[1]
     hidden_vectors = len(dims) - 2
-    return float(hidden_vectors * w * (7 + (int(np.log2(w)) if rotate else 0)))
+    return float(hidden_vectors * w * (7 + int(rotate) * int(np.log2(w))))
 
 
 class ClockSampler:
@@ -117,7 +122,7 @@ def work_per_coord(dims, rotate=True):
     w, hidden_vectors, hidden_matmuls = dims[1], len(dims) - 2, len(dims) - 3
     macs = 4 * w + hidden_matmuls * w * w + 4 * w
     sines = hidden_vectors * w
-    fp32 = hidden_vectors * w * (3 + (int(np.log2(w)) if rotate else 0))
+    fp32 = hidden_vectors * w * (3 + int(rotate) * int(np.log2(w)))
     return macs, sines, fp32
 
 
@@ -149,7 +154,7 @@ def run_reference(args, workload):
     sample = min(workload.n, 16384)
     steps = max(1, min(args.steps, 5))
     warmup = min(args.warmup, 1)
-    value, dt, cores, _ = time_oracle(workload, steps, warmup, sample, args.rotation == "input")
+    value, dt, cores, _ = time_oracle(workload, steps, warmup, sample, rotations(args.rotation))
     desc = f"first {sample} coordinates of the {workload.grid[0]}x{workload.grid[1]} grid per step"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -201,7 +206,7 @@ def run_ours(args, workload):
     W = [torch.from_numpy(w).cuda() for w in weights]
     B = [torch.from_numpy(b).cuda() for b in biases]
     h = dhq.dhq_prepare(workload.dims, W, B, workload.omega0, workload.w_bits, workload.a_bits,
-                        workload.w_gran, workload.a_gran, rotation=0 if args.rotation == "input" else 2)
+                        workload.w_gran, workload.a_gran, rotation={"input": 0, "both": 1, "none": 2}[args.rotation])
     coords = torch.from_numpy(coords_np).cuda()
     out = torch.empty((n, d_L), dtype=torch.float32, device="cuda")
     coords_host = torch.from_numpy(coords_np).pin_memory()
@@ -253,7 +258,7 @@ def run_ours(args, workload):
             pass
         sm_max = float(peaks.get("sm_max_mhz", 1965.0))
         alu_peak = SM_COUNT * FP32_LANES_PER_SM * sm_max * 1e6 / 1e12            # T lane-ops/s
-        achieved = alu_laneops_per_coord(workload.dims, args.rotation == "input") * n / (ms_per_step * 1e-3) / 1e12
+        achieved = alu_laneops_per_coord(workload.dims, rotations(args.rotation)) * n / (ms_per_step * 1e-3) / 1e12
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -277,7 +282,7 @@ def run_ours(args, workload):
         }
         # The same launch against the other pipes' ceilings, each measured now on this GPU by the
         # library's own micro-benchmarks (perfect-overlap model: each pipe alone).
-        macs, sines, fp32_ops = work_per_coord(workload.dims, args.rotation == "input")
+        macs, sines, fp32_ops = work_per_coord(workload.dims, rotations(args.rotation))
         per_s = n / (ms_per_step * 1e-3)
         pipes = {}
         for key, pipe, work in (("tensor_i8", "tensor_i8", 2.0 * macs), ("sfu_sine", "mufu_sin", float(sines)),
@@ -301,7 +306,7 @@ def run_ours(args, workload):
         line["pipes"] = pipes
         if world == 1 and not args.no_cpu_baseline:
             sample = min(n, 65536)
-            v, dt, cores, passes = time_oracle(workload, 1, 1, sample, args.rotation == "input", min_seconds=10.0)
+            v, dt, cores, passes = time_oracle(workload, 1, 1, sample, rotations(args.rotation), min_seconds=10.0)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                     "sample": f"first {sample} coordinates of the grid, {passes} pass(es) of {dt:.1f} s"}
         print(json.dumps(line), flush=True)
@@ -323,7 +328,7 @@ def run_sweep(args, workload):
     h = dhq.dhq_prepare(workload.dims, [torch.from_numpy(w).cuda() for w in weights],
                         [torch.from_numpy(b).cuda() for b in biases], workload.omega0, workload.w_bits,
                         workload.a_bits, workload.w_gran, workload.a_gran,
-                        rotation=0 if args.rotation == "input" else 2)
+                        rotation={"input": 0, "both": 1, "none": 2}[args.rotation])
     dhq.dhq_calibrate(h, torch.from_numpy(workload.coords()).cuda())
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
@@ -361,8 +366,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C2", choices=sorted(dhq_inputs.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--rotation", default="input", choices=["input", "none"],
-                    help="input = DHQ; none = the same path without the Hadamard rotation (uniform quantizer)")
+    ap.add_argument("--rotation", default="input", choices=["input", "none", "both"],
+                    help="input = DHQ; none = the same path without the Hadamard rotation (uniform quantizer); "
+                         "both = the two-sided transform of Eq. 4-5, run layer by layer")
     ap.add_argument("--limit-coords", type=int, default=0,
                     help="use only the first N coordinates of the workload's grid (profiling captures)")
     ap.add_argument("--sweep", action="store_true", help="batch-size sweep 2^12..2^24 instead of the timed steps")

@@ -69,7 +69,11 @@ typedef enum { DHQ_GRAN_TENSOR = 0, DHQ_GRAN_CHANNEL_OR_TOKEN = 1 } dhq_gran_t;
 
 /* Which side of Eq. 4 is applied.  DHQ_ROT_INPUT is the DHQ path; DHQ_ROT_NONE skips the rotation
  * of weights and activations (the plain uniform quantizer the paper compares against, Section
- * IV-B) with everything else unchanged; DHQ_ROT_BOTH is declared but not implemented. */
+ * IV-B) with everything else unchanged.  DHQ_ROT_BOTH is Eq. 4-5 taken literally, W~ = H_M W H_K /
+ * (K M) (rows first, then columns, same fp32 butterfly order), with the layer output
+ * z = H_M (s_w s_x acc) + b: the output-side rotation is undone in fp64 after dequantization
+ * and before the bias.  It runs layer by layer (one kernel pass per layer, activations in device
+ * memory between layers), not in the fused kernel; dhq_forward_static_scratch does not take it. */
 typedef enum { DHQ_ROT_INPUT = 0, DHQ_ROT_BOTH = 1, DHQ_ROT_NONE = 2 } dhq_rot_t;
 
 typedef struct {
@@ -80,7 +84,7 @@ typedef struct {
     float omega0;       /* sine frequency of layers 1..L-1                                 */
     dhq_gran_t w_gran;
     dhq_gran_t a_gran;
-    dhq_rot_t rotation; /* DHQ_ROT_INPUT or DHQ_ROT_NONE                                   */
+    dhq_rot_t rotation; /* DHQ_ROT_INPUT, DHQ_ROT_NONE or DHQ_ROT_BOTH                     */
 } dhq_config_t;
 
 /*
@@ -109,8 +113,7 @@ typedef struct {
  * Allocates device memory; enqueues the preparation kernels on `stream` and returns.  W and b
  * may be released once that stream work has completed.
  * Errors: INVALID_ARG (NULL, n_layers out of range), UNSUPPORTED (dims[0] != 2, width not a
- * power of two in 64..512 or not uniform, d_L outside 1..4, bits outside 2..8, rotation
- * DHQ_ROT_BOTH), ALLOC, CUDA.
+ * power of two in 64..512 or not uniform, d_L outside 1..4, bits outside 2..8), ALLOC, CUDA.
  */
 DHQ_API dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W,
                                  const float *const *b, void *stream, dhq_handle_t *out);

@@ -147,7 +147,10 @@ class OracleNet:
 
 
 def _rot_mode(rotate) -> int:
-    if rotate in ("both", 2) and rotate is not True:
+    """True / 1: input side; False / 0: none; "both" / 2: both sides."""
+    if rotate is True or rotate is False:
+        return int(rotate)
+    if rotate == "both" or rotate == 2:
         return 2
     return int(bool(rotate))
 

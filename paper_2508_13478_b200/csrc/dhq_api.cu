@@ -56,7 +56,8 @@ LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X
     a.a_bits = h->cfg.a_bits;
     a.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
     a.epi_mode = d.epi_mode;
-    a.rotate = h->cfg.rotation == DHQ_ROT_INPUT;
+    a.rotate = h->cfg.rotation == DHQ_ROT_INPUT ? 1 : h->cfg.rotation == DHQ_ROT_BOTH ? 2 : 0;
+    a.s_w = d.s_w; a.bias = d.bias; a.omega0 = (double)h->cfg.omega0; a.sine = l < h->L;
     a.qw_k4m = d.qw_k4m; a.cA = d.cA; a.cA_lo = d.cA_lo; a.cB = d.cB; a.act = d.act;
     a.fxP = d.fxP; a.fxQ = d.fxQ; a.fxB = d.fxB;
     return a;
@@ -96,6 +97,35 @@ dhq_status_t calibrate_impl(dhq_handle_s *h, const float *coords, int64_t n, cud
     h->calibrated = true;
     h->calib_layers_done = h->L;
     return DHQ_OK;
+}
+
+// Layers 1..L one kernel pass each over tokens in chunks, activations in the handle's scratch.
+dhq_status_t layerwise_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st)
+{
+    const int64_t chunk = n < kDebugChunk ? n : kDebugChunk;
+    dhq_status_t s = ensure_scratch(h, chunk);
+    if (s != DHQ_OK) return s;
+    for (int64_t t0 = 0; t0 < n; t0 += chunk) {
+        int64_t cnt = n - t0 < chunk ? n - t0 : chunk;
+        const float *X = nullptr;
+        for (int l = 1; l <= h->L; ++l) {
+            LayerArgs a = layer_args(h, l, coords + t0 * 2, X, cnt);
+            a.Y = h->scratch[(l - 1) & 1];
+            if (l == h->L) a.out = out + t0 * h->d_L;
+            CK(launch_layer(a, st));
+            h->launches++;
+            X = a.Y;
+        }
+    }
+    return DHQ_OK;
+}
+
+// The forward pass of a calibrated handle: the fused kernel, or, for the two-sided transform, the
+// layer-by-layer kernels.
+dhq_status_t run_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st)
+{
+    if (h->cfg.rotation == DHQ_ROT_BOTH) return layerwise_forward(h, coords, n, out, st);
+    return fused_forward(h, coords, n, out, st);
 }
 
 } // namespace
@@ -151,7 +181,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     for (int l = 1; l < L; ++l)
         if (cfg->dims[l] != w) return DHQ_ERR_UNSUPPORTED;
     if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits < 2 || cfg->a_bits > 8) return DHQ_ERR_UNSUPPORTED;
-    if (cfg->rotation != DHQ_ROT_INPUT && cfg->rotation != DHQ_ROT_NONE) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->rotation != DHQ_ROT_INPUT && cfg->rotation != DHQ_ROT_NONE && cfg->rotation != DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
     if ((cfg->w_gran != DHQ_GRAN_TENSOR && cfg->w_gran != DHQ_GRAN_CHANNEL_OR_TOKEN) ||
         (cfg->a_gran != DHQ_GRAN_TENSOR && cfg->a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN))
         return DHQ_ERR_INVALID_ARG;
@@ -167,6 +197,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     dhq_status_t rc = DHQ_OK;
     float *d_bounds = nullptr;
     const bool per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
+    const bool both = cfg->rotation == DHQ_ROT_BOTH;
     do {
         if (cudaGetDevice(&h->device) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
         if (!dev_alloc(&h->d_status, 4) || !dev_alloc(&d_bounds, kMaxLayers)) { rc = DHQ_ERR_ALLOC; break; }
@@ -181,6 +212,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             d.d_in = cfg->dims[l - 1];
             d.d_out = cfg->dims[l];
             if (l == 1) d.epi_mode = per_token ? EPI_SINE_WIDE : EPI_SINE_FIXED; // coordinates are not bounded by the weights
+            if (both) d.epi_mode = EPI_BOTH;
             const size_t MK = (size_t)d.M * d.K;
             bool ok = dev_alloc(&d.w_rot, MK) && dev_alloc(&d.row_absmax, d.M) && dev_alloc(&d.qw, MK) &&
                       dev_alloc(&d.qw_k4m, MK / 4) && dev_alloc(&d.qw_umma, (size_t)d.Mt * (d.K < 16 ? 16 : d.K)) &&
@@ -198,7 +230,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             a.per_channel = cfg->w_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
             a.sine = l < L; a.first = l == 1;
             a.permute_rows = (l > 1 && l < L) ? 1 : 0;
-            a.rotate = cfg->rotation == DHQ_ROT_INPUT;
+            a.rotate = cfg->rotation == DHQ_ROT_INPUT ? 1 : both ? 2 : 0;
             a.omega0 = (double)cfg->omega0;
             a.dev = d;
             a.phase_bound = d_bounds + (l - 1);
@@ -215,12 +247,13 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
         for (int l = 1; l <= L; ++l) {
             LayerDev &d = h->layer[l - 1];
             d.phase_bound = bounds[l - 1];
-            if (l == L) d.epi_mode = EPI_LINEAR;
+            if (both) d.epi_mode = EPI_BOTH;
+            else if (l == L) d.epi_mode = EPI_LINEAR;
             else if (l == 1) {}
             else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit) ? EPI_SINE_FAST : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;
-        rc = fused_create(h);
+        if (!both) rc = fused_create(h); // the two-sided transform runs layer by layer (no fused kernel yet)
     } while (0);
     cudaFree(d_bounds);
     if (rc != DHQ_OK) {
@@ -318,7 +351,7 @@ dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *
         dhq_status_t s = calibrate_impl(h, coords, n, st);
         if (s != DHQ_OK) return s;
     }
-    return fused_forward(h, coords, n, out, st);
+    return run_forward(h, coords, n, out, st);
 }
 
 dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t n, float *out_host,
@@ -339,7 +372,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
                             cudaHostGetDevicePointer(&di, const_cast<float *>(coords_host), 0) == cudaSuccess &&
                             cudaHostGetDevicePointer(&dout, out_host, 0) == cudaSuccess && di && dout;
         (void)cudaGetLastError(); // a failed query of pageable memory is not an error of this call
-        if (mapped) return fused_forward(h, static_cast<const float *>(di), n, static_cast<float *>(dout), st);
+        if (mapped) return run_forward(h, static_cast<const float *>(di), n, static_cast<float *>(dout), st);
     }
     if (n > h->stage_tokens) {
         CK(cudaDeviceSynchronize());
@@ -389,7 +422,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
                            cudaMemcpyHostToDevice, h->copy_in));
         CK(cudaEventRecord(h->ev_in[i], h->copy_in));
         CK(cudaStreamWaitEvent(st, h->ev_in[i], 0));
-        dhq_status_t s = fused_forward(h, h->stage_in + t0 * 2, cnt, h->stage_out + t0 * h->d_L, st);
+        dhq_status_t s = run_forward(h, h->stage_in + t0 * 2, cnt, h->stage_out + t0 * h->d_L, st);
         if (s != DHQ_OK) return s;
         CK(cudaEventRecord(h->ev_k[i], st));
         CK(cudaStreamWaitEvent(h->copy_out, h->ev_k[i], 0));

@@ -66,12 +66,17 @@ struct LayerArgs {
     int a_bits;
     int per_token;
     int epi_mode;
-    int rotate;            // 0: DHQ_ROT_NONE, the layer input is quantized as it is
+    int rotate;            // 0: DHQ_ROT_NONE, the layer input is quantized as it is; 2: DHQ_ROT_BOTH (see s_w below)
     int calib_only;        // 1: only take max |rotated input| into act[0] (bit pattern max)
     const uint32_t *qw_k4m;
     const float *cA, *cA_lo, *cB;
     const uint32_t *fxP, *fxQ, *fxB;
     float *act;            // frozen absmax / s_x / inv (per-tensor mode)
+    // DHQ_ROT_BOTH: raw weight scales and biases [M], omega0 and whether the layer has a sine; the
+    // output is z = H_M (s_w s_x acc) + b, computed in fp64
+    const float *s_w, *bias;
+    double omega0;
+    int sine;
     float *Y;              // [n][M] or NULL
     float *out;            // [n][d_L] or NULL (last layer)
     float *dX; int8_t *dcodes; float *ds_x; int32_t *dacc; // dumps, may be NULL
@@ -83,7 +88,7 @@ struct PrepArgs {
     const float *W, *b;
     int d_out, d_in, K, M, Mt;
     int bits, per_channel;
-    int rotate;            // 0: DHQ_ROT_NONE, weights are quantized as they are
+    int rotate;            // 0: DHQ_ROT_NONE, weights are quantized as they are; 2: DHQ_ROT_BOTH, columns rotated too
     int permute_rows;      // 1: rows of the tensor-core image in fused_column order (layers 2 .. L-1)
     int sine;              // hidden or first layer
     int first;             // layer 1: no phase bound from the weights (coordinates are unbounded)

@@ -17,6 +17,7 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
     __shared__ __align__(16) int8_t cs[TB * 512];
     __shared__ float s_tok[TB], inv_tok[TB];
     __shared__ float blockmax[LW_THREADS / 32];
+    extern __shared__ double dq[];   // DHQ_ROT_BOTH only: [TB][M] dequantized values in the rotated output basis
 
     const int K = a.K, M = a.M, tid = threadIdx.x;
     const int64_t base = (int64_t)blockIdx.x * TB;
@@ -91,6 +92,17 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
             for (int t = 0; t < TB; ++t)
                 acc[t] = __dp4a(((const int *)cs)[t * K4 + k4], w, acc[t]);
         }
+        if (a.rotate == 2) {
+            // two-sided transform: keep d = s_w s_x acc of every token; the output follows below
+            const double sw = (double)a.s_w[m];
+#pragma unroll
+            for (int t = 0; t < TB; ++t) {
+                dq[t * M + m] = sw * (double)s_tok[t] * (double)acc[t];
+                int64_t tok = base + t;
+                if (a.dacc && tok < a.n) a.dacc[tok * M + m] = acc[t];
+            }
+            continue;
+        }
         const float cA = a.cA[m], cAl = a.cA_lo[m], cB = a.cB[m];
 #pragma unroll
         for (int t = 0; t < TB; ++t) {
@@ -108,13 +120,52 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
             if (a.out && m < a.d_L) a.out[tok * a.d_L + m] = y;
         }
     }
+    if (a.rotate != 2) return;
+    // z = H_M d + b (H_M H_M = M I, and the 1/M is in the weights): fp64 butterfly over the M outputs.
+    // The sum of up to 512 terms reaches phases of tens of radians that must stay within 1e-5 of
+    // the fp64 definition; an fp32 butterfly does not (about 1e-7 rms per radian of phase).
+    for (int h = 1; h < M; h <<= 1) {
+        __syncthreads();
+        for (int p = tid; p < TB * (M / 2); p += LW_THREADS) {
+            int t = p / (M / 2), j = p % (M / 2);
+            int i = t * M + (((j & ~(h - 1)) << 1) | (j & (h - 1)));
+            double x = dq[i], y = dq[i + h];
+            dq[i] = x + y;
+            dq[i + h] = x - y;
+        }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < TB * M; idx += LW_THREADS) {
+        int t = idx / M, j = idx % M;
+        int64_t tok = base + t;
+        if (tok >= a.n) continue;
+        double z = dq[idx] + (double)a.bias[j];
+        float y;
+        if (a.sine) {
+            // phase reduced to [-pi, pi] in fp64, then the hardware sine on an fp32 argument
+            const double two_pi = 6.283185307179586476925287;
+            double ph = a.omega0 * z;
+            ph -= two_pi * rint(ph * (1.0 / two_pi));
+            y = sin_approx((float)ph);
+        } else {
+            y = (float)z;
+        }
+        if (a.Y) a.Y[tok * M + j] = y;
+        if (a.out && j < a.d_L) a.out[tok * a.d_L + j] = y;
+    }
 }
 
 cudaError_t launch_layer(const LayerArgs &a, cudaStream_t st)
 {
     if (a.n <= 0) return cudaSuccess;
     int64_t blocks = (a.n + TB - 1) / TB;
-    layer_kernel<<<(unsigned)blocks, LW_THREADS, 0, st>>>(a);
+    size_t dyn = 0;
+    if (a.rotate == 2 && !a.calib_only) {
+        dyn = (size_t)TB * a.M * sizeof(double); // up to 64 KB beside the 41 KB of static shared memory
+        cudaError_t e = cudaFuncSetAttribute(layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TB * 512 * (int)sizeof(double));
+        if (e != cudaSuccess) return e;
+    }
+    layer_kernel<<<(unsigned)blocks, LW_THREADS, dyn, st>>>(a);
     return cudaGetLastError();
 }
 

@@ -13,7 +13,8 @@ enum EpiMode : int {
     EPI_LINEAR = 0,    // last layer: z = c * acc + b
     EPI_SINE_FAST = 1, // hidden layer whose phase is provably small: sin.approx(fma(acc, c, B))
     EPI_SINE_WIDE = 2, // large phases: compensated phase and explicit 2*pi reduction
-    EPI_SINE_FIXED = 3 // first layer with a per-tensor activation scale: phase in 32-bit fixed point
+    EPI_SINE_FIXED = 3, // first layer with a per-tensor activation scale: phase in 32-bit fixed point
+    EPI_BOTH = 4       // two-sided transform: the layer kernel undoes the output-side rotation in fp64
 };
 
 // Largest |omega0 z| for which EPI_SINE_FAST keeps the result within 1e-5 of an exact sine:

@@ -57,6 +57,44 @@ __global__ void prep_rotate_kernel(PrepArgs a)
     }
 }
 
+// DHQ_ROT_BOTH, output-side factor of Eq. 4: one block per column k; the column of the row-rotated
+// weights goes through the same fp32 butterfly over the M rows and is scaled by the exact 1/M.
+__global__ void prep_rotate_cols_kernel(PrepArgs a)
+{
+    extern __shared__ float col[];
+    const int k = blockIdx.x, K = a.K, M = a.M;
+    for (int m = threadIdx.x; m < M; m += blockDim.x) col[m] = a.dev.w_rot[(size_t)m * K + k];
+    for (int h = 1; h < M; h <<= 1) {
+        __syncthreads();
+        for (int p = threadIdx.x; p < M / 2; p += blockDim.x) {
+            int i = ((p & ~(h - 1)) << 1) | (p & (h - 1));
+            float x = col[i], y = col[i + h];
+            col[i] = __fadd_rn(x, y);
+            col[i + h] = __fsub_rn(x, y);
+        }
+    }
+    __syncthreads();
+    const float invM = 1.0f / (float)M; // power of two: exact
+    for (int m = threadIdx.x; m < M; m += blockDim.x) a.dev.w_rot[(size_t)m * K + k] = __fmul_rn(col[m], invM);
+}
+
+// Row absmax of the final rotated weights (after the column pass).
+__global__ void prep_row_absmax_kernel(PrepArgs a)
+{
+    __shared__ float red[32];
+    const int m = blockIdx.x, K = a.K;
+    float amax = 0.f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) amax = fmaxf(amax, fabsf(a.dev.w_rot[(size_t)m * K + k]));
+    for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float r = 0.f;
+        for (int i = 0; i < (blockDim.x + 31) / 32; ++i) r = fmaxf(r, red[i]);
+        a.dev.row_absmax[m] = r;
+    }
+}
+
 // One block: per-tensor or per-row scales.
 __global__ void prep_scales_kernel(PrepArgs a)
 {
@@ -135,6 +173,12 @@ cudaError_t launch_prepare(const PrepArgs &a, cudaStream_t st, int64_t *launches
 {
     int threads = a.K / 2 < 32 ? 32 : a.K / 2;
     prep_rotate_kernel<<<a.M, threads, a.K * sizeof(float), st>>>(a);
+    if (a.rotate == 2) {
+        int tc = a.M / 2 < 32 ? 32 : a.M / 2;
+        prep_rotate_cols_kernel<<<a.K, tc, a.M * sizeof(float), st>>>(a);
+        prep_row_absmax_kernel<<<a.M, 128, 0, st>>>(a);
+        *launches += 2;
+    }
     prep_scales_kernel<<<1, 256, 0, st>>>(a);
     int total = a.Mt * a.K;
     prep_quant_kernel<<<(total + 255) / 256, 256, 0, st>>>(a);

@@ -44,7 +44,7 @@ extern "C" dhq_status_t dhq_forward_static_scratch(dhq_handle_t h, const float *
     if (n > DHQ_STATIC_MAX_TOKENS) return DHQ_ERR_TOO_LARGE;
     if (n == 0) return DHQ_OK;
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
-    if (h->w > kMaxWidth) return DHQ_ERR_UNSUPPORTED;
+    if (h->w > kMaxWidth || h->cfg.rotation == DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
     float *scratch = nullptr;
     dhq_status_t s = scratch_for_current_device(&scratch);
     if (s != DHQ_OK) return s;

@@ -15,7 +15,7 @@ def to_dev(a):
 
 def prepare_pair(dims, weights, biases, omega0, w_bits, a_bits, w_gran, a_gran, rotate=True):
     h = dhq.dhq_prepare(dims, [to_dev(w) for w in weights], [to_dev(b) for b in biases], omega0,
-                        w_bits, a_bits, w_gran, a_gran, rotation=0 if rotate else 2)
+                        w_bits, a_bits, w_gran, a_gran, rotation=1 if rotate == "both" else 0 if rotate else 2)
     net = orc.prepare(weights, biases, dims, omega0, w_bits, a_bits, w_gran, a_gran, rotate=rotate)
     return h, net
 

@@ -137,6 +137,39 @@ def test_no_rotation_variant_uniform_quantizer(name, count):
     _p1(w, np.ascontiguousarray(coords[idx]), rotate=False)
 
 
+@pytest.mark.parametrize("name,count", [("C1", 4096), ("C2", 9000 + 5), ("C3", 6000 + 3), ("C4-W4A4", 3000 + 1), ("C5", 2000 + 9)])
+def test_two_sided_transform_layer_by_layer(name, count):
+    # DHQ_ROT_BOTH: Eq. 4-5 literally.  Weight codes and scales, activation codes, scales and
+    # accumulators bit-exact; the outputs (output-side rotation undone in fp64) within 1e-5.
+    w = dhq_inputs.WORKLOADS[name]
+    coords = w.coords()
+    idx = np.linspace(0, coords.shape[0] - 1, count).astype(np.int64)
+    _p1(w, np.ascontiguousarray(coords[idx]), rotate="both")
+
+
+def test_two_sided_transform_wide_phases_host_buffers_and_static_scratch():
+    dims = (2, 256, 256, 256, 3)
+    weights, biases = dhq_inputs.trained_like_init(dims, 30.0, 12)
+    weights[0] = (weights[0] * 4).astype(np.float32)          # phases of hundreds of radians
+    weights[1] = (weights[1] * 6).astype(np.float32)
+    coords = dhq_inputs.grid_coords(40, 50)
+    h, net = prepare_pair(dims, weights, biases, 30.0, 8, 8, 1, 1, rotate="both")
+    try:
+        check_weights(h, net)
+        out_dbg, bufs = run_debug(h, net, to_dev(coords))
+        check_layers_against_oracle(h, net, coords, out_dbg, bufs)
+        ch = torch.from_numpy(coords).pin_memory()
+        oh = torch.zeros((coords.shape[0], 3)).pin_memory()
+        dhq.dhq_forward_host(h, ch, oh)
+        torch.cuda.synchronize()
+        assert torch.equal(oh.view(torch.int32), out_dbg.cpu().view(torch.int32))
+        with pytest.raises(dhq.DhqError) as e:
+            dhq.dhq_forward_static_scratch(h, to_dev(coords[:100]), torch.empty((100, 3), device="cuda"))
+        assert e.value.code == 2
+    finally:
+        dhq.dhq_destroy(h)
+
+
 def test_trained_like_weights_and_wide_phases():
     # bell-shaped hidden weights, two-peaked last layer (Section III-A), and a first layer scaled up
     # so that phases reach hundreds of radians
@@ -185,7 +218,7 @@ def test_unsupported_and_invalid_arguments():
         dhq.dhq_prepare((3, 64, 64, 64, 1), W, B)
     assert e.value.code == 2
     with pytest.raises(dhq.DhqError) as e:
-        dhq.dhq_prepare((2, 64, 64, 64, 1), W, B, rotation=1)      # two-sided rotation: not implemented
+        dhq.dhq_prepare((2, 64, 64, 64, 1), W, B, rotation=7)      # no such rotation mode
     assert e.value.code == 2
     h = dhq.dhq_prepare(w.dims, W, B)
     try:
