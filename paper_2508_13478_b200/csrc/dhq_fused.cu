@@ -131,16 +131,25 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
 }
 
 // Bounded wait.  Returns false when the wait ran out or another role already gave up.  Between
-// tries the thread sleeps, so that a waiting warp leaves the issue slots to the working ones;
-// the time limit and the abort flag are looked at every 64 tries.
-template <int SLEEP_NS>
+// tries the thread either sleeps (SLEEP_NS), so that a waiting warp leaves the issue slots to the
+// working ones, or, with HINT_NS > 0, stays suspended inside the try itself for up to that long;
+// the time limit and the abort flag are looked at every 64 tries.  Which form is faster was
+// measured per role: the single-thread MMA and copy roles and the epilogue warps of the
+// per-token kernels (two more barriers per layer) do better suspended, the epilogue warps of the
+// per-tensor kernels sleeping.
+constexpr int kHintNs = 2000;
+template <int SLEEP_NS, int HINT_NS = 0>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
     for (uint32_t tries = 1;; ++tries) {
-        __nanosleep(SLEEP_NS);
-        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (HINT_NS > 0) {
+            if (ptx::mbar_try_wait_hint(bar, parity, HINT_NS)) return true;
+        } else {
+            __nanosleep(SLEEP_NS);
+            if (ptx::mbar_try_wait(bar, parity)) return true;
+        }
         if ((tries & 63) == 0) {
             if (*abort_flag) return false;
             const unsigned long long now = ptx::globaltimer();
@@ -154,9 +163,10 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 // The same for a whole warp: every lane takes the same decision.
+template <bool SUSPEND>
 __device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
-    return __all_sync(0xffffffffu, wait_bar<32>(bar, parity, abort_flag, status));
+    return __all_sync(0xffffffffu, wait_bar<32, SUSPEND ? kHintNs : 0>(bar, parity, abort_flag, status));
 }
 
 // Two fp32 values in one 64-bit register pair, and the packed sm_100 arithmetic on them: one
@@ -415,10 +425,10 @@ struct SlotCtx {
     int *status;
 };
 
-__device__ __forceinline__ bool slot_barrier(SlotCtx &c)
+template <bool SUSPEND> __device__ __forceinline__ bool slot_barrier(SlotCtx &c)
 {
     ptx::mbar_arrive(c.bar_sync);
-    bool ok = wait_bar_warp(c.bar_sync, c.sync_parity, c.abort_flag, c.status);
+    bool ok = wait_bar_warp<SUSPEND>(c.bar_sync, c.sync_parity, c.abort_flag, c.status);
     c.sync_parity ^= 1;
     return ok;
 }
@@ -433,7 +443,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
     constexpr int NCH = C::NCH, G = C::G, CH = C::CH;
     ptx::tmem_wait_st();
     ptx::tc_fence_before();
-    if (!slot_barrier(c)) return false;
+    if (!slot_barrier<PER_TOKEN>(c)) return false;
     ptx::tc_fence_after();
     float amax = 0.f;
 #pragma unroll 1
@@ -478,7 +488,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
         asm volatile("st.shared.f32 [%0], %1;" ::"r"(c.amax_addr + (c.sub * kTile + c.row) * 4), "f"(amax) : "memory");
         ptx::tmem_wait_st();
         ptx::tc_fence_before();
-        if (!slot_barrier(c)) return false;
+        if (!slot_barrier<PER_TOKEN>(c)) return false;
         ptx::tc_fence_after();
 #pragma unroll
         for (int r = 0; r < C::R; ++r) {
@@ -587,7 +597,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
         // ---------------- layers 2 .. L on the tensor core
         for (int l = 2; l < p.L; ++l) {
             const FusedLayer &ly = p.layer[l - 1];
-            if (!wait_bar_warp(bar_acc, acc_parity, abort_flag, p.status)) return;
+            if (!wait_bar_warp<PER_TOKEN>(bar_acc, acc_parity, abort_flag, p.status)) return;
             acc_parity ^= 1;
             ptx::tc_fence_after();
             if (!PER_TOKEN) {
@@ -610,7 +620,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
         }
         {
             const FusedLayer &ly = p.layer[p.L - 1];
-            if (!wait_bar_warp(bar_last, last_parity, abort_flag, p.status)) return;
+            if (!wait_bar_warp<PER_TOKEN>(bar_last, last_parity, abort_flag, p.status)) return;
             last_parity ^= 1;
             ptx::tc_fence_after();
             if (sub == 0) {
@@ -655,11 +665,11 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
                 const int slab_id = (l - 2) * C::KSLABS + ksl;
                 const int stage = p.resident ? slab_id : (int)(use % p.n_stages);
                 const uint32_t par = p.resident ? 0u : (uint32_t)((use / p.n_stages) & 1);
-                if (!wait_bar<100>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
+                if (!wait_bar<0, kHintNs>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
                 const uint32_t b_addr = smem_base + sm.ring + (uint32_t)stage * slab;
                 for (int s = 0; s < active; ++s) {
                     if (ksl == 0) {
-                        if (!wait_bar<100>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
+                        if (!wait_bar<0, kHintNs>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
                         codes_parity[s] ^= 1;
                         ptx::tc_fence_after();
                     }
@@ -684,9 +694,9 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
         }
         if (!ok) break;
         // last layer: N = 16, its weights stay in shared memory
-        if (!wait_bar<100>(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
+        if (!wait_bar<0, kHintNs>(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
         for (int s = 0; s < active; ++s) {
-            if (!wait_bar<100>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
+            if (!wait_bar<0, kHintNs>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
             codes_parity[s] ^= 1;
             ptx::tc_fence_after();
             const uint32_t d = tmem_base + (uint32_t)(s * C::TMEM_COLS_PER_SLOT);
@@ -727,7 +737,7 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
         const int stage = (int)(i % p.n_stages);
         if (i >= p.n_stages) {
             uint32_t par = (uint32_t)(((i / p.n_stages) - 1) & 1);
-            if (!wait_bar<100>(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
+            if (!wait_bar<0, kHintNs>(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
         }
         const int id = (int)(i % slabs);
         const int l = 2 + id / C::KSLABS, pc = id % C::KSLABS;
