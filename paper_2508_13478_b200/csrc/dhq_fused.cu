@@ -62,6 +62,16 @@ template <int W> struct Cfg {
     static constexpr int TMEM_COLS_PER_SLOT = 512 / SLOTS;
 };
 
+// Tile of slot `slot` of this CTA in its round r.  Normally the slots of a CTA take adjacent tiles.
+// A launch with fewer tiles than CTAs x slots is spread instead: the tiles go round-robin first
+// over the CTAs, then over the slots, so that it covers as many SMs as it has tiles (one busy slot
+// each) before any SM gets a second tile.
+template <bool SPREAD> __device__ __forceinline__ long long tile_index(long long r, int slot, int slots)
+{
+    return SPREAD ? (r * slots + slot) * (long long)gridDim.x + blockIdx.x
+                  : ((long long)blockIdx.x + r * gridDim.x) * slots + slot;
+}
+
 struct FusedLayer {
     const uint8_t *qw_umma;
     const uint32_t *qw_k4m;
@@ -516,7 +526,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
     return true;
 }
 
-template <int W, bool PER_TOKEN, bool ROT>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD>
 __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
@@ -544,7 +554,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     const FusedLayer &l1 = p.layer[0];
     const float qmaxf = p.qmaxf;
 
-    if (C::SLOTS == 2 && slot == 1 && p.n_tiles > 1 && p.resident) {
+    if (C::SLOTS == 2 && slot == 1 && tile_index<SPREAD>(0, 1, 2) < p.n_tiles && p.resident) {
         // Start the second slot about half a layer period after the first, so that one slot's
         // sine-heavy pass 1 and MMA wait fall on the other slot's pass 2 instead of both slots
         // asking for the same pipe at the same time.  The offset then keeps itself.  Not when the
@@ -553,7 +563,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
         while (ptx::globaltimer() - t0 < delay) __nanosleep(64);
     }
     for (long long r = 0;; ++r) {
-        const long long tile = ((long long)blockIdx.x + r * gridDim.x) * C::SLOTS + slot;
+        const long long tile = tile_index<SPREAD>(r, slot, C::SLOTS);
         if (tile >= p.n_tiles) break;
         const long long tok = tile * kTile + c.row;
         const bool valid = tok < p.n;
@@ -643,7 +653,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     }
 }
 
-template <int W>
+template <int W, bool SPREAD>
 __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, uint32_t tmem_base,
                          volatile int *abort_flag)
 {
@@ -657,9 +667,8 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
     long long use = 0; // ring uses so far (streaming mode)
     bool ok = true;
     for (long long r = 0; ok; ++r) {
-        const long long tile0 = ((long long)blockIdx.x + r * gridDim.x) * C::SLOTS;
-        if (tile0 >= p.n_tiles) break;
-        const int active = (C::SLOTS == 2 && tile0 + 1 < p.n_tiles) ? 2 : 1;
+        if (tile_index<SPREAD>(r, 0, C::SLOTS) >= p.n_tiles) break;
+        const int active = (C::SLOTS == 2 && tile_index<SPREAD>(r, 1, C::SLOTS) < p.n_tiles) ? 2 : 1;
         for (int l = 2; l < p.L && ok; ++l) {
             for (int ksl = 0; ksl < C::KSLABS && ok; ++ksl) {
                 const int slab_id = (l - 2) * C::KSLABS + ksl;
@@ -716,7 +725,7 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
     }
 }
 
-template <int W>
+template <int W, bool SPREAD>
 __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
 {
     using C = Cfg<W>;
@@ -727,7 +736,7 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
     if (slabs <= 0) return;
     long long rounds = 0;
     for (long long r = 0;; ++r) {
-        if (((long long)blockIdx.x + r * gridDim.x) * C::SLOTS >= p.n_tiles) break;
+        if (tile_index<SPREAD>(r, 0, C::SLOTS) >= p.n_tiles) break;
         ++rounds;
     }
     const long long total = p.resident ? slabs : rounds * slabs;
@@ -761,7 +770,7 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
     }
 }
 
-template <int W, bool PER_TOKEN, bool ROT>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD>
 __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constant__ FusedParams p)
 {
     using C = Cfg<W>;
@@ -820,11 +829,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN, ROT>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
+        epilogue_role<W, PER_TOKEN, ROT, SPREAD>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
-        if (lane == 0) mma_role<W>(p, sm, smem_base, tmem_base, abort_flag);
+        if (lane == 0) mma_role<W, SPREAD>(p, sm, smem_base, tmem_base, abort_flag);
     } else {
-        if (lane == 0) load_role<W>(p, sm, smem_base, abort_flag);
+        if (lane == 0) load_role<W, SPREAD>(p, sm, smem_base, abort_flag);
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -838,18 +847,19 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
 
 typedef void (*fused_fn)(const FusedParams);
 
-template <int W> static fused_fn pick_width(bool per_token, bool rot)
+template <int W, bool SPREAD> static fused_fn pick_width(bool per_token, bool rot)
 {
-    if (rot) return per_token ? fused_kernel<W, true, true> : fused_kernel<W, false, true>;
-    return per_token ? fused_kernel<W, true, false> : fused_kernel<W, false, false>;
+    if (rot) return per_token ? fused_kernel<W, true, true, SPREAD> : fused_kernel<W, false, true, SPREAD>;
+    return per_token ? fused_kernel<W, true, false, SPREAD> : fused_kernel<W, false, false, SPREAD>;
 }
-static fused_fn pick_kernel(int W, bool per_token, bool rot)
+// spread: the tile-to-CTA mapping for launches smaller than one tile per slot of every SM (tile_index)
+static fused_fn pick_kernel(int W, bool per_token, bool rot, bool spread)
 {
     switch (W) {
-    case 64: return pick_width<64>(per_token, rot);
-    case 128: return pick_width<128>(per_token, rot);
-    case 256: return pick_width<256>(per_token, rot);
-    case 512: return pick_width<512>(per_token, rot);
+    case 64: return spread ? pick_width<64, true>(per_token, rot) : pick_width<64, false>(per_token, rot);
+    case 128: return spread ? pick_width<128, true>(per_token, rot) : pick_width<128, false>(per_token, rot);
+    case 256: return spread ? pick_width<256, true>(per_token, rot) : pick_width<256, false>(per_token, rot);
+    case 512: return spread ? pick_width<512, true>(per_token, rot) : pick_width<512, false>(per_token, rot);
     }
     return nullptr;
 }
@@ -882,8 +892,9 @@ dhq_status_t fused_create(dhq_handle_s *h)
         }
     }
     p.const_words = words;
-    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
-    if (!fn) return DHQ_ERR_UNSUPPORTED;
+    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false);
+    fused_fn fn_spread = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, true);
+    if (!fn || !fn_spread) return DHQ_ERR_UNSUPPORTED;
     int dev = 0, max_optin = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
@@ -904,7 +915,8 @@ dhq_status_t fused_create(dhq_handle_s *h)
     size_t bytes = smem_map(h->w, p.n_stages, words).total + 1024;
     if (bytes < (size_t)kMinSmem) bytes = kMinSmem;
     fs->smem_bytes = bytes;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(fn_spread, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
         return DHQ_ERR_CUDA;
     return DHQ_OK;
 }
@@ -929,10 +941,11 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     FusedParams p = fs->p;
     p.coords = coords; p.out = out; p.n = n;
     p.n_tiles = (n + kTile - 1) / kTile;
-    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     const int slots = (h->w == 512) ? 1 : 2;
-    long long rounds_all = (p.n_tiles + slots - 1) / slots;
-    int grid = (int)(rounds_all < fs->sm_count ? rounds_all : fs->sm_count);
+    const bool spread = slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
+    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread);
+    const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
+    int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, kThreads, fs->smem_bytes, st>>>(p);
     h->launches++;
     return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;
