@@ -6,7 +6,9 @@
 //               128 tokens in flight (its own A operand tile and 256 tensor-memory columns), so
 //               that one slot's CUDA-core work overlaps the other slot's MMA; the second slot
 //               starts half a layer period late.  Width 512: one slot of 16 warps; a layer's
-//               weights arrive as four K slabs of 128 and each slab feeds two N = 256 MMAs.
+//               weights arrive as eight pieces (256 output columns x 128 k, the first half of the
+//               columns first), each feeding N = 256 MMAs; a thread has one chunk in each half
+//               and starts on the first while the second half's weights and MMAs are under way.
 //               A token (row) is a tensor-memory lane; R = 2 (or 4) threads from different warps
 //               share a row and split its columns.
 //   warp 16     issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in tensor memory).
@@ -58,6 +60,8 @@ template <int W> struct Cfg {
     static constexpr int SLABK = W / KSLABS;                   // k per slab (= fused_slab_k)
     static constexpr int NHALF = (W == 512) ? 2 : 1;           // MMAs along N (an MMA has N <= 256)
     static constexpr int NW = W / NHALF;                       // N of one MMA
+    static constexpr int PIECES = KSLABS * NHALF;              // weight pieces per layer (ring units)
+    static constexpr int PIECE_BYTES = SLABK * NW;             // 64 KB (width 256), 32 KB (width 512)
     static constexpr int SLOT_THREADS = R * kTile;
     static constexpr int TMEM_COLS_PER_SLOT = 512 / SLOTS;
 };
@@ -70,6 +74,14 @@ template <bool SPREAD> __device__ __forceinline__ long long tile_index(long long
 {
     return SPREAD ? (r * slots + slot) * (long long)gridDim.x + blockIdx.x
                   : ((long long)blockIdx.x + r * gridDim.x) * slots + slot;
+}
+
+// Chunk cc of the thread with index `sub` among the R threads of a row.  Width 512 gives every
+// thread one chunk in each half of the columns (the halves' accumulators complete one after the
+// other); otherwise a thread's chunks are adjacent.
+template <int W> __device__ __forceinline__ int chunk_of(int sub, int cc)
+{
+    return (W == 512) ? cc * Cfg<W>::R + sub : sub * Cfg<W>::CPT + cc;
 }
 
 struct FusedLayer {
@@ -117,12 +129,12 @@ struct SmemMap {
 __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words)
 {
     const int slots = (W == 512) ? 1 : 2;
-    const int slab_k = (W == 512) ? 128 : W;
+    const uint32_t piece_bytes = (W == 512) ? 128u * 256u : (uint32_t)W * W;
     SmemMap m;
     uint32_t off = 0;
     m.a_tile[0] = off; off += kTile * W;
     m.a_tile[1] = off; if (slots == 2) off += kTile * W;
-    m.ring = off; off += (uint32_t)n_stages * slab_k * W;
+    m.ring = off; off += (uint32_t)n_stages * piece_bytes;
     m.last_w = off; off += 16 * W;
     m.consts = off; off += (uint32_t)const_words * 4;
     m.amax = off; off += 2 * 4 * kTile * 4;
@@ -597,7 +609,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
         }
 #pragma unroll
         for (int cc = 0; cc < C::CPT; ++cc) {
-            const int ch = sub * C::CPT + cc;
+            const int ch = chunk_of<W>(sub, cc);
             uint32_t v[CH];
             layer1_chunk<W, CH, PER_TOKEN, ROT>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v);
             tmem_st<CH>(c.taddr + ch * CH, v);
@@ -608,7 +620,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
         for (int l = 2; l < p.L; ++l) {
             const FusedLayer &ly = p.layer[l - 1];
             if (!wait_bar_warp<PER_TOKEN>(bar_acc, acc_parity, abort_flag, p.status)) return;
-            acc_parity ^= 1;
+            if constexpr (C::NHALF == 1) acc_parity ^= 1;
             ptx::tc_fence_after();
             if (!PER_TOKEN) {
                 next_s = __ldg(p.layer[l].act + 1);
@@ -618,7 +630,16 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
             const bool fast = ly.epi_mode == EPI_SINE_FAST;
 #pragma unroll
             for (int cc = 0; cc < C::CPT; ++cc) {
-                const int ch = sub * C::CPT + cc;
+                const int ch = chunk_of<W>(sub, cc);
+                if constexpr (C::NHALF == 2) {
+                    // width 512: the thread's second chunk lies in the second half of the output columns,
+                    // whose MMAs run while the first chunk is worked on
+                    if (cc == 1) {
+                        if (!wait_bar_warp<PER_TOKEN>(bar_acc + 8, acc_parity, abort_flag, p.status)) return;
+                        acc_parity ^= 1;
+                        ptx::tc_fence_after();
+                    }
+                }
                 uint32_t v[CH];
                 tmem_ld<CH>(c.taddr + ch * CH, v);
                 ptx::tmem_wait_ld();
@@ -660,7 +681,7 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
     using C = Cfg<W>;
     uint32_t codes_parity[2] = {0, 0};
     const uint32_t idesc_hidden = ptx::idesc_i8(kTile, C::NW), idesc_last = ptx::idesc_i8(kTile, 16);
-    const uint32_t slab = W * C::SLABK;
+    const uint32_t slab = C::PIECE_BYTES;
     // each K step of 32 advances a descriptor's start-address field (bits 0-13, 16-byte units) by
     // two core-matrix columns
     const uint64_t a_step = (uint64_t)((2 * kTile * 16) >> 4);
@@ -670,6 +691,33 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
         if (tile_index<SPREAD>(r, 0, C::SLOTS) >= p.n_tiles) break;
         const int active = (C::SLOTS == 2 && tile_index<SPREAD>(r, 1, C::SLOTS) < p.n_tiles) ? 2 : 1;
         for (int l = 2; l < p.L && ok; ++l) {
+            if constexpr (C::NHALF == 2) {
+                // width 512: eight pieces per layer, the four k-pieces of output columns 0..255 first;
+                // each half of the accumulator is committed on its own barrier as soon as it is complete
+                for (int pc = 0; pc < C::PIECES && ok; ++pc) {
+                    const int half = pc / C::KSLABS, ksl = pc % C::KSLABS;
+                    const int stage = (int)(use % p.n_stages);
+                    const uint32_t par = (uint32_t)((use / p.n_stages) & 1);
+                    if (!wait_bar<0, kHintNs>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
+                    if (pc == 0) {
+                        if (!wait_bar<0, kHintNs>(smem_base + sm.codes_full, codes_parity[0], abort_flag, p.status)) { ok = false; break; }
+                        codes_parity[0] ^= 1;
+                        ptx::tc_fence_after();
+                    }
+                    const uint32_t b_addr = smem_base + sm.ring + (uint32_t)stage * C::PIECE_BYTES;
+                    const uint64_t ad0 = ptx::smem_desc(smem_base + sm.a_tile[0] + ksl * (C::SLABK / 16) * (kTile * 16), kTile * 16, 128);
+                    const uint32_t d = tmem_base + (uint32_t)(half * C::NW);
+                    const uint64_t bd0 = ptx::smem_desc(b_addr, C::NW * 16, 128);
+                    const uint64_t b_step = (uint64_t)((2 * C::NW * 16) >> 4);
+#pragma unroll
+                    for (int ks = 0; ks < C::SLABK / 32; ++ks)
+                        ptx::mma_i8(d, ad0 + ks * a_step, bd0 + ks * b_step, idesc_hidden, (ksl > 0 || ks > 0) ? 1u : 0u);
+                    if (ksl == C::KSLABS - 1) ptx::mma_commit(smem_base + sm.acc_full + 8 * half);
+                    ptx::mma_commit(smem_base + sm.w_empty + 8 * stage);
+                    ++use;
+                }
+                continue;
+            }
             for (int ksl = 0; ksl < C::KSLABS && ok; ++ksl) {
                 const int slab_id = (l - 2) * C::KSLABS + ksl;
                 const int stage = p.resident ? slab_id : (int)(use % p.n_stages);
@@ -729,10 +777,10 @@ template <int W, bool SPREAD>
 __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
 {
     using C = Cfg<W>;
-    const uint32_t slab = W * C::SLABK;
+    const uint32_t slab = C::PIECE_BYTES;
     ptx::mbar_expect_tx(smem_base + sm.last_full, 16 * W);
     ptx::bulk_g2s(smem_base + sm.last_w, p.layer[p.L - 1].qw_umma, 16 * W, smem_base + sm.last_full);
-    const int slabs = (p.L - 2) * C::KSLABS; // per tile round
+    const int slabs = (p.L - 2) * C::PIECES; // per tile round
     if (slabs <= 0) return;
     long long rounds = 0;
     for (long long r = 0;; ++r) {
@@ -749,7 +797,7 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
             if (!wait_bar<0, kHintNs>(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
         }
         const int id = (int)(i % slabs);
-        const int l = 2 + id / C::KSLABS, pc = id % C::KSLABS;
+        const int l = 2 + id / C::PIECES, pc = id % C::PIECES;
         ptx::mbar_expect_tx(smem_base + sm.w_full + 8 * stage, slab);
         // several copies in flight per slab: one large bulk copy did not reach the L2 bandwidth
         for (uint32_t off = 0; off < slab; off += kCopyBytes) {
@@ -902,9 +950,9 @@ dhq_status_t fused_create(dhq_handle_s *h)
         return DHQ_ERR_CUDA;
     // weight ring: as many slab stages as fit beside the A tiles and the constants; all hidden
     // layers resident if they fit
-    const int kslabs = (h->w == 512) ? 4 : 1;
-    const int slabs = (h->L - 2) * kslabs;
-    const size_t slab_bytes = (size_t)(h->w / kslabs) * h->w;
+    const int pieces = (h->w == 512) ? 8 : 1;
+    const int slabs = (h->L - 2) * pieces;
+    const size_t slab_bytes = (h->w == 512) ? (size_t)128 * 256 : (size_t)h->w * h->w;
     const size_t fixed = smem_map(h->w, 0, words).total + 1024;
     if (fixed > (size_t)max_optin) return DHQ_ERR_UNSUPPORTED;
     int stages = (int)(((size_t)max_optin - fixed) / slab_bytes);

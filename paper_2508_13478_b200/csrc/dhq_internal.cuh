@@ -108,10 +108,15 @@ cudaError_t launch_finalize(const LayerDev &dev, int a_bits, int per_token, int 
 // (rows * 16 bytes apart) - the K-major, unswizzled operand layout of tcgen05.mma.
 __host__ __device__ inline size_t umma_offset(int n, int k, int rows, int slab_k)
 {
+    // A 512 x 512 layer is cut once more, along its rows: eight pieces of 256 rows x 128 k (32 KB),
+    // the four k-pieces of rows 0..255 first, so that the first half of the output columns can be
+    // finished (and worked on) while the second half's weights still stream in.
+    if (rows == 512 && slab_k == 128)
+        return (size_t)((n >> 8) * 4 + k / 128) * 32768 + (size_t)((k % 128) >> 4) * 4096 + (size_t)(n & 255) * 16 + (k & 15);
     return (size_t)(k / slab_k) * rows * slab_k + (size_t)((k % slab_k) >> 4) * rows * 16 + (size_t)n * 16 + (k & 15);
 }
-// Codes per row in one slab: a 512 x 512 layer is streamed in four slabs of 128 k (64 KB each);
-// narrower layers are one slab.
+// Codes per row in one slab: a 512 x 512 layer is streamed in slabs of 128 k (each cut in two
+// 32 KB pieces of 256 rows, see umma_offset); narrower layers are one slab.
 __host__ __device__ inline int fused_slab_k(int K, int rows) { return (K == 512 && rows == 512) ? 128 : (K < 16 ? 16 : K); }
 // Columns of a hidden layer's output are processed by the fused kernel in register chunks of
 // fused_chunk(W) columns, and inside a chunk the features i and i + chunk/2 sit in adjacent
