@@ -116,6 +116,7 @@ struct FusedState {
 struct SmemMap {
     uint32_t a_tile[2];
     uint32_t ring, last_w, consts, amax;
+    uint32_t xy;         // [2 slots][4 threads of a row][128 rows] float2: coordinates fetched ahead
     uint32_t acc_full;   // [2 slots][4 pieces]
     uint32_t acc_last;   // [2]
     uint32_t codes_full; // [2]
@@ -138,6 +139,7 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
     m.last_w = off; off += 16 * W;
     m.consts = off; off += (uint32_t)const_words * 4;
     m.amax = off; off += 2 * 4 * kTile * 4;
+    m.xy = off; if (W != 512) off += 2 * 4 * kTile * 8; // width 512 does not fetch ahead and needs the room for its weight ring
     m.acc_full = off; off += 8 * 8;
     m.acc_last = off; off += 8 * 2;
     m.codes_full = off; off += 8 * 2;
@@ -538,7 +540,7 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
     return true;
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD>
 __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
@@ -562,6 +564,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     const uint32_t bar_acc = smem_base + sm.acc_full + 8 * (slot * 4);
     const uint32_t bar_last = smem_base + sm.acc_last + 8 * slot;
     const uint32_t consts = smem_base + sm.consts;
+    const uint32_t xy_addr = smem_base + sm.xy + (uint32_t)(((slot * 4 + sub) * kTile + c.row) * 8);
     uint32_t acc_parity = 0, last_parity = 0;
     const FusedLayer &l1 = p.layer[0];
     const float qmaxf = p.qmaxf;
@@ -582,9 +585,15 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
 
         // ---------------- layer 1 on the CUDA cores: x~ = H_4 [x, y, 0, 0]
         float x = 0.f, y = 0.f;
-        if (valid) {
-            float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
-            x = xy.x; y = xy.y;
+        if (!AHEAD || r == 0) {
+            if (valid) {
+                float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
+                x = xy.x; y = xy.y;
+            }
+        } else {
+            // copied into shared memory by this thread while the previous tile was in its hidden layers
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            if (valid) asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x), "=f"(y) : "r"(xy_addr));
         }
         float e0 = x, e1 = y, e2 = 0.f, e3 = 0.f;
         if (ROT) {
@@ -615,6 +624,17 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
             tmem_st<CH>(c.taddr + ch * CH, v);
         }
         if (!finish_layer<W, PER_TOKEN, ROT>(c, next_s, next_inv, s_x)) return;
+        if constexpr (AHEAD) {
+            // The next tile's coordinates start their way into shared memory now.  An asynchronous
+            // copy holds neither a register nor one of the warp's dependency barriers while it is in
+            // flight (a plain load issued this early slowed the layers down: they wait on the barrier
+            // it occupies).  Not earlier than this: at the start of a launch every tile's first fetch
+            // is under way.  Only for coordinates in device memory: from mapped host memory the
+            // 8-byte asynchronous copies were slower than the plain load at the tile's start.
+            const long long tok_next = tile_index<SPREAD>(r + 1, slot, C::SLOTS) * kTile + c.row;
+            if (tok_next < p.n)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(xy_addr), "l"(reinterpret_cast<const float2 *>(p.coords) + tok_next) : "memory");
+        }
 
         // ---------------- layers 2 .. L on the tensor core
         for (int l = 2; l < p.L; ++l) {
@@ -818,7 +838,7 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
     }
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD>
 __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constant__ FusedParams p)
 {
     using C = Cfg<W>;
@@ -877,7 +897,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN, ROT, SPREAD>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
+        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_role<W, SPREAD>(p, sm, smem_base, tmem_base, abort_flag);
     } else {
@@ -895,19 +915,26 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
 
 typedef void (*fused_fn)(const FusedParams);
 
-template <int W, bool SPREAD> static fused_fn pick_width(bool per_token, bool rot)
+template <int W, bool SPREAD, bool AHEAD> static fused_fn pick_flags(bool per_token, bool rot)
 {
-    if (rot) return per_token ? fused_kernel<W, true, true, SPREAD> : fused_kernel<W, false, true, SPREAD>;
-    return per_token ? fused_kernel<W, true, false, SPREAD> : fused_kernel<W, false, false, SPREAD>;
+    if (rot) return per_token ? fused_kernel<W, true, true, SPREAD, AHEAD> : fused_kernel<W, false, true, SPREAD, AHEAD>;
+    return per_token ? fused_kernel<W, true, false, SPREAD, AHEAD> : fused_kernel<W, false, false, SPREAD, AHEAD>;
 }
-// spread: the tile-to-CTA mapping for launches smaller than one tile per slot of every SM (tile_index)
-static fused_fn pick_kernel(int W, bool per_token, bool rot, bool spread)
+template <int W, bool AHEAD_OK> static fused_fn pick_width(bool per_token, bool rot, bool spread, bool ahead)
+{
+    if (AHEAD_OK && ahead) return spread ? pick_flags<W, true, AHEAD_OK>(per_token, rot) : pick_flags<W, false, AHEAD_OK>(per_token, rot);
+    return spread ? pick_flags<W, true, false>(per_token, rot) : pick_flags<W, false, false>(per_token, rot);
+}
+// spread: the tile-to-CTA mapping for launches smaller than one tile per slot of every SM (tile_index);
+// ahead: coordinates of the next tile copied to shared memory early (device memory only; width 512
+// gained nothing from it and has no such variant)
+static fused_fn pick_kernel(int W, bool per_token, bool rot, bool spread, bool ahead)
 {
     switch (W) {
-    case 64: return spread ? pick_width<64, true>(per_token, rot) : pick_width<64, false>(per_token, rot);
-    case 128: return spread ? pick_width<128, true>(per_token, rot) : pick_width<128, false>(per_token, rot);
-    case 256: return spread ? pick_width<256, true>(per_token, rot) : pick_width<256, false>(per_token, rot);
-    case 512: return spread ? pick_width<512, true>(per_token, rot) : pick_width<512, false>(per_token, rot);
+    case 64: return pick_width<64, true>(per_token, rot, spread, ahead);
+    case 128: return pick_width<128, true>(per_token, rot, spread, ahead);
+    case 256: return pick_width<256, true>(per_token, rot, spread, ahead);
+    case 512: return pick_width<512, false>(per_token, rot, spread, ahead);
     }
     return nullptr;
 }
@@ -940,9 +967,8 @@ dhq_status_t fused_create(dhq_handle_s *h)
         }
     }
     p.const_words = words;
-    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false);
-    fused_fn fn_spread = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, true);
-    if (!fn || !fn_spread) return DHQ_ERR_UNSUPPORTED;
+    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false, false);
+    if (!fn) return DHQ_ERR_UNSUPPORTED;
     int dev = 0, max_optin = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
@@ -963,9 +989,11 @@ dhq_status_t fused_create(dhq_handle_s *h)
     size_t bytes = smem_map(h->w, p.n_stages, words).total + 1024;
     if (bytes < (size_t)kMinSmem) bytes = kMinSmem;
     fs->smem_bytes = bytes;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(fn_spread, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
-        return DHQ_ERR_CUDA;
+    for (int v = 0; v < 4; ++v) { // every variant of this handle's kernel
+        fused_fn f = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, (v & 1) != 0, (v & 2) != 0);
+        if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+            return DHQ_ERR_CUDA;
+    }
     return DHQ_OK;
 }
 
@@ -991,7 +1019,10 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     p.n_tiles = (n + kTile - 1) / kTile;
     const int slots = (h->w == 512) ? 1 : 2;
     const bool spread = slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
-    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread);
+    cudaPointerAttributes at;
+    const bool on_host = cudaPointerGetAttributes(&at, coords) == cudaSuccess && at.type == cudaMemoryTypeHost;
+    (void)cudaGetLastError();
+    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, kThreads, fs->smem_bytes, st>>>(p);
