@@ -1,7 +1,7 @@
 // Fused forward kernel: the whole quantized INR (Sections III-B and III-C of the paper) for
 // tiles of 128 coordinates without activations leaving the SM between layers.
 //
-// One persistent CTA per SM, 18 warps:
+// One persistent CTA per SM, 18 warps (19 at width 512):
 //   warps 0-15  epilogue warps.  Width <= 256: two "slots" of 8 warps, each slot has one tile of
 //               128 tokens in flight (its own A operand tile and 256 tensor-memory columns), so
 //               that one slot's CUDA-core work overlaps the other slot's MMA; the second slot
@@ -12,6 +12,8 @@
 //               A token (row) is a tensor-memory lane; R = 2 (or 4) threads from different warps
 //               share a row and split its columns.
 //   warp 16     issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in tensor memory).
+//   warp 18     (width 512) brings each tile's coordinates into shared memory with one bulk copy,
+//               a tile ahead.
 //   warp 17     brings the packed weight codes into shared memory with bulk async copies: once,
 //               if every hidden layer fits (they then stay resident), else through a ring that
 //               is refilled slab by slab from L2.
@@ -40,8 +42,8 @@ namespace dhq {
 
 constexpr int kTile = 128;
 constexpr int kEpiWarps = 16;
-constexpr int kMmaWarp = 16, kLoadWarp = 17;
-constexpr int kThreads = 18 * 32;
+constexpr int kMmaWarp = 16, kLoadWarp = 17, kXyWarp = 18;
+constexpr int kThreads = 18 * 32; // width 512 runs one more warp (Cfg::THREADS)
 constexpr int kMaxStages = 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull; // 2 s per wait
 constexpr uint32_t kCopyBytes = 8192; // bytes per bulk copy of a weight slab
@@ -63,6 +65,10 @@ template <int W> struct Cfg {
     static constexpr int PIECES = KSLABS * NHALF;              // weight pieces per layer (ring units)
     static constexpr int PIECE_BYTES = SLABK * NW;             // 64 KB (width 256), 32 KB (width 512)
     static constexpr int SLOT_THREADS = R * kTile;
+    // Width 512: the coordinates of a whole tile arrive by one bulk copy issued by a 19th warp (measured:
+    // 2.6 % faster, 6.7 % from mapped host memory; narrower networks lost 4-7 % to the extra barrier).
+    static constexpr bool BULK_XY = (W == 512);
+    static constexpr int THREADS = kThreads + (BULK_XY ? 32 : 0);
     static constexpr int TMEM_COLS_PER_SLOT = 512 / SLOTS;
 };
 
@@ -101,6 +107,7 @@ struct FusedParams {
     int L, W, d_L, per_token;
     float qmaxf;
     int n_stages, resident;
+    int bulk_xy;         // coords 16-byte aligned: whole tiles may arrive by bulk copy (width 512)
     int const_words;
     int *status;
     FusedLayer layer[kMaxLayers];
@@ -122,6 +129,7 @@ struct SmemMap {
     uint32_t codes_full; // [2]
     uint32_t slot_sync;  // [2 slots][4 lane quadrants]
     uint32_t last_full, drain;
+    uint32_t xy_full, xy_empty; // [2 slots] each: coordinates by bulk copy
     uint32_t w_full, w_empty; // [kMaxStages] each
     uint32_t tmem_holder, abort_flag;
     uint32_t total;
@@ -139,12 +147,14 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
     m.last_w = off; off += 16 * W;
     m.consts = off; off += (uint32_t)const_words * 4;
     m.amax = off; off += 2 * 4 * kTile * 4;
-    m.xy = off; if (W != 512) off += 2 * 4 * kTile * 8; // width 512 does not fetch ahead and needs the room for its weight ring
+    m.xy = off; off += (W != 512) ? 2 * 4 * kTile * 8 : kTile * 8; // per-thread entries, or one tile for the bulk copy
     m.acc_full = off; off += 8 * 8;
     m.acc_last = off; off += 8 * 2;
     m.codes_full = off; off += 8 * 2;
     m.slot_sync = off; off += 8 * 8;
     m.last_full = off; off += 8;
+    m.xy_full = off; if (W == 512) off += 16;
+    m.xy_empty = off; if (W == 512) off += 16;
     m.drain = off; off += 8;
     m.w_full = off; off += 8 * kMaxStages;
     m.w_empty = off; off += 8 * kMaxStages;
@@ -566,6 +576,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     const uint32_t consts = smem_base + sm.consts;
     const uint32_t xy_addr = smem_base + sm.xy + (uint32_t)(((slot * 4 + sub) * kTile + c.row) * 8);
     uint32_t acc_parity = 0, last_parity = 0;
+    [[maybe_unused]] uint32_t xy_k = 0; // tiles taken from the bulk-copy buffer so far
     const FusedLayer &l1 = p.layer[0];
     const float qmaxf = p.qmaxf;
 
@@ -585,6 +596,18 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
 
         // ---------------- layer 1 on the CUDA cores: x~ = H_4 [x, y, 0, 0]
         float x = 0.f, y = 0.f;
+        if constexpr (C::BULK_XY) {
+            if (p.bulk_xy && (tile + 1) * kTile <= p.n) {
+                // the whole tile was brought to shared memory by one bulk copy, a tile ahead
+                if (!wait_bar_warp<PER_TOKEN>(smem_base + sm.xy_full + 8 * slot, xy_k & 1u, abort_flag, p.status)) return;
+                ++xy_k;
+                asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x), "=f"(y) : "r"(smem_base + sm.xy + (uint32_t)((slot * kTile + c.row) * 8)));
+                ptx::mbar_arrive(smem_base + sm.xy_empty + 8 * slot);
+            } else if (valid) { // ragged last tile, or coordinates not 16-byte aligned
+                float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
+                x = xy.x; y = xy.y;
+            }
+        } else
         if (!AHEAD || r == 0) {
             if (valid) {
                 float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
@@ -838,8 +861,36 @@ __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem
     }
 }
 
+// Width 512.  Coordinates: one bulk copy per whole tile (1 KB) into the slot's buffer, issued as
+// soon as the slot's threads have taken the previous tile's coordinates out of it.
+template <int W, bool SPREAD>
+__device__ void xy_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
+{
+    using C = Cfg<W>;
+    if (!p.bulk_xy) return;
+    uint32_t k[2] = {0, 0};
+    bool ok = true;
+    for (long long r = 0; ok; ++r) {
+        if (tile_index<SPREAD>(r, 0, C::SLOTS) >= p.n_tiles) break;
+        for (int s = 0; s < C::SLOTS && ok; ++s) {
+            const long long tile = tile_index<SPREAD>(r, s, C::SLOTS);
+            if (tile >= p.n_tiles || (tile + 1) * kTile > p.n) continue; // none, or ragged: the threads load it themselves
+            if (k[s] > 0 && !wait_bar<0, kHintNs>(smem_base + sm.xy_empty + 8 * s, (k[s] - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+            ptx::mbar_expect_tx(smem_base + sm.xy_full + 8 * s, kTile * 8);
+            ptx::bulk_g2s(smem_base + sm.xy + (uint32_t)(s * kTile * 8), p.coords + tile * kTile * 2, kTile * 8, smem_base + sm.xy_full + 8 * s);
+            ++k[s];
+        }
+    }
+    if (!ok || *abort_flag) { // let a copy in flight land before the CTA may exit
+        const unsigned long long t0 = ptx::globaltimer();
+        for (int s = 0; s < C::SLOTS; ++s)
+            if (k[s] > 0)
+                while (!ptx::mbar_try_wait(smem_base + sm.xy_full + 8 * s, (k[s] - 1) & 1u) && ptx::globaltimer() - t0 < kWaitLimitNs) {}
+    }
+}
+
 template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD>
-__global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constant__ FusedParams p)
+__global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_constant__ FusedParams p)
 {
     using C = Cfg<W>;
     extern __shared__ uint8_t smem_raw[];
@@ -860,6 +911,12 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
             for (int q = 0; q < 4; ++q) ptx::mbar_init(smem_base + sm.slot_sync + 8 * (s * 4 + q), C::R * 32);
         }
         ptx::mbar_init(smem_base + sm.last_full, 1);
+        if constexpr (C::BULK_XY) {
+            for (int s2 = 0; s2 < 2; ++s2) {
+                ptx::mbar_init(smem_base + sm.xy_full + 8 * s2, 1);
+                ptx::mbar_init(smem_base + sm.xy_empty + 8 * s2, C::SLOT_THREADS);
+            }
+        }
         ptx::mbar_init(smem_base + sm.drain, 1);
         for (int i = 0; i < kMaxStages; ++i) {
             ptx::mbar_init(smem_base + sm.w_full + 8 * i, 1);
@@ -882,7 +939,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
             const uint32_t *srcB = fixed ? ly.fxB : reinterpret_cast<const uint32_t *>(ly.cB);
             const uint32_t *srcC = fixed ? ly.fxQ : reinterpret_cast<const uint32_t *>(ly.cA_lo);
             const int areas = (l == 0) ? (fixed ? 3 : 4) : (ly.epi_mode == EPI_SINE_WIDE ? 3 : 2);
-            for (int i = threadIdx.x; i < W; i += kThreads) { // i: tensor-memory column, m: its feature
+            for (int i = threadIdx.x; i < W; i += C::THREADS) { // i: tensor-memory column, m: its feature
                 const int m = fused_feature(i, W);
                 d[i] = __ldg(srcA + m);
                 d[W + i] = __ldg(srcB + m);
@@ -900,8 +957,12 @@ __global__ void __launch_bounds__(kThreads, 1) fused_kernel(const __grid_constan
         epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_role<W, SPREAD>(p, sm, smem_base, tmem_base, abort_flag);
-    } else {
+    } else if (warp == kLoadWarp) {
         if (lane == 0) load_role<W, SPREAD>(p, sm, smem_base, abort_flag);
+    } else {
+        if constexpr (C::BULK_XY) {
+            if (lane == 0) xy_role<W, SPREAD>(p, sm, smem_base, abort_flag);
+        }
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -1017,6 +1078,7 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     FusedParams p = fs->p;
     p.coords = coords; p.out = out; p.n = n;
     p.n_tiles = (n + kTile - 1) / kTile;
+    p.bulk_xy = (((uintptr_t)coords) & 15) == 0;
     const int slots = (h->w == 512) ? 1 : 2;
     const bool spread = slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
     cudaPointerAttributes at;
@@ -1025,7 +1087,7 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
-    fn<<<grid, kThreads, fs->smem_bytes, st>>>(p);
+    fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
     h->launches++;
     return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;
 }
