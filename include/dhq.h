@@ -174,7 +174,8 @@ DHQ_API dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n,
  *   - Both buffers pinned (page-locked, e.g. cudaHostAlloc / cudaHostRegister) and the scales
  *     already frozen: no staging and no copy call.  The fused kernel reads the coordinates and
  *     writes the result through the buffers' device mapping, so the transfers over the host link
- *     happen tile by tile inside the one launch, beside the arithmetic.
+ *     happen tile by tile inside the one launch, beside the arithmetic (with out_host 16-byte
+ *     aligned, each whole tile of results leaves by one bulk store).
  *   - Otherwise (pageable memory, or the first per-tensor call, which calibrates): the data is
  *     staged in device buffers owned by the handle, grown on demand (this may allocate and
  *     synchronize the first time a larger n is seen).  Larger n is cut into up to 8 launches, each

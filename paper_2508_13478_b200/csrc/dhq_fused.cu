@@ -108,6 +108,7 @@ struct FusedParams {
     float qmaxf;
     int n_stages, resident;
     int bulk_xy;         // coords 16-byte aligned: whole tiles may arrive by bulk copy (width 512)
+    int bulk_out;        // out 16-byte aligned: whole tiles may leave by bulk store (host-buffer variant)
     int const_words;
     int *status;
     FusedLayer layer[kMaxLayers];
@@ -124,6 +125,7 @@ struct SmemMap {
     uint32_t a_tile[2];
     uint32_t ring, last_w, consts, amax;
     uint32_t xy;         // [2 slots][4 threads of a row][128 rows] float2: coordinates fetched ahead
+    uint32_t out_tile;   // [2 slots][128 rows][4] fp32: a tile's results before their bulk store (width <= 256)
     uint32_t acc_full;   // [2 slots][4 pieces]
     uint32_t acc_last;   // [2]
     uint32_t codes_full; // [2]
@@ -148,6 +150,7 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
     m.consts = off; off += (uint32_t)const_words * 4;
     m.amax = off; off += 2 * 4 * kTile * 4;
     m.xy = off; off += (W != 512) ? 2 * 4 * kTile * 8 : kTile * 8; // per-thread entries, or one tile for the bulk copy
+    m.out_tile = off; if (W != 512) off += 2 * kTile * 4 * 4; // placed here, among the 16-byte aligned areas: a bulk store reads it
     m.acc_full = off; off += 8 * 8;
     m.acc_last = off; off += 8 * 2;
     m.codes_full = off; off += 8 * 2;
@@ -701,20 +704,38 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
                 uint32_t u[4];
                 ptx::tmem_ld4(c.taddr, u);
                 ptx::tmem_wait_ld();
+                // Host-buffer variant: a whole tile's results (128 x d_L floats, contiguous in `out`) are
+                // collected in shared memory and leave by one bulk store: over the host link one large
+                // write instead of 128 x d_L four-byte ones.  The slot's 128 sub-0 threads meet on a named
+                // barrier before and after filling the buffer; its first thread issues the store.
+                const bool by_bulk = !AHEAD && !C::BULK_XY && p.bulk_out && (tile + 1) * kTile <= p.n;
+                const uint32_t ot = smem_base + sm.out_tile + (uint32_t)(slot * kTile * 16);
+                if (by_bulk) {
+                    if (c.row == 0) ptx::bulk_wait_read(); // the previous tile's store has read the buffer
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + slot) : "memory");
+                }
                 if (valid) {
 #pragma unroll
                     for (int m = 0; m < 4; ++m) {
                         if (m < p.d_L) {
                             float c_hi = __ldg(ly.cA + m), c_lo = 0.f;
                             if (PER_TOKEN) c_hi = __fmul_rn(c_hi, s_x);
-                            p.out[tok * p.d_L + m] = epilogue(EPI_LINEAR, (float)(int)u[m], c_hi, c_lo, __ldg(ly.cB + m));
+                            const float yv = epilogue(EPI_LINEAR, (float)(int)u[m], c_hi, c_lo, __ldg(ly.cB + m));
+                            if (by_bulk) asm volatile("st.shared.f32 [%0], %1;" ::"r"(ot + (uint32_t)((c.row * p.d_L + m) * 4)), "f"(yv) : "memory");
+                            else p.out[tok * p.d_L + m] = yv;
                         }
                     }
+                }
+                if (by_bulk) {
+                    ptx::fence_proxy_async();
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + slot) : "memory");
+                    if (c.row == 0) ptx::bulk_s2g(p.out + tile * kTile * p.d_L, ot, (uint32_t)(kTile * p.d_L * 4));
                 }
             }
             ptx::tc_fence_before();
         }
     }
+    if (!AHEAD && !C::BULK_XY && sub == 0 && c.row == 0) ptx::bulk_wait_all(); // the last tiles' stores
 }
 
 template <int W, bool SPREAD>
@@ -1079,6 +1100,7 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     p.coords = coords; p.out = out; p.n = n;
     p.n_tiles = (n + kTile - 1) / kTile;
     p.bulk_xy = (((uintptr_t)coords) & 15) == 0;
+    p.bulk_out = (((uintptr_t)out) & 15) == 0 && (smem_map(h->w, p.n_stages, p.const_words).out_tile & 15) == 0;
     const int slots = (h->w == 512) ? 1 : 2;
     const bool spread = slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
     cudaPointerAttributes at;
