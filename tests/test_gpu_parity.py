@@ -442,6 +442,39 @@ def test_sharded_calibration_equals_whole_set(name, parts):
             dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("name", ["C2", "C5"])
+def test_buffers_that_are_only_8_byte_aligned_take_the_plain_paths(name):
+    """Whole tiles travel by bulk copies only when the buffers are 16-byte aligned (coordinates at
+    width 512, results of the host-buffer variant at width <= 256).  Buffers offset by one
+    coordinate / one float are legal (8- and 4-byte aligned) and must give the same bits."""
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h, _ = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        n, d_L = 3 * 18944 + 77, w.dims[-1]
+        coords = np.ascontiguousarray(w.coords()[: n + 1])
+        dhq.dhq_calibrate(h, to_dev(w.coords()))
+        cd = to_dev(coords)
+        ref = torch.empty((n, d_L), device="cuda")
+        dhq.dhq_forward(h, cd[1:].contiguous(), ref)                       # aligned copy of the same coordinates
+        out = torch.empty((n, d_L), device="cuda")
+        shifted = cd[1:]                                                   # a view: starts 8 bytes into the allocation
+        assert shifted.data_ptr() % 16 == 8 and shifted.is_contiguous()
+        dhq.dhq_forward(h, shifted, out)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int32), ref.view(torch.int32))
+        ch = torch.from_numpy(coords).pin_memory()
+        flat = torch.zeros(n * d_L + 1).pin_memory()
+        oh = flat[1:].view(n, d_L)                                         # starts 4 bytes into the allocation
+        assert oh.data_ptr() % 16 == 4
+        dhq.dhq_forward_host(h, ch[1:], oh)
+        torch.cuda.synchronize()
+        assert torch.equal(oh.view(torch.int32), ref.cpu().view(torch.int32))
+        assert dhq.dhq_last_status(h) == 0
+    finally:
+        dhq.dhq_destroy(h)
+
+
 def test_pipe_micro_benchmarks_run():
     for pipe in ("ffma", "mufu_sin", "tensor_i8", "pass1", "pass2", "pass12"):
         ops, ms = dhq.dhq_measure_pipe(pipe, 200)
