@@ -132,6 +132,7 @@ struct SmemMap {
     uint32_t slot_sync;  // [2 slots][4 lane quadrants]
     uint32_t last_full, drain;
     uint32_t xy_full, xy_empty; // [2 slots] each: coordinates by bulk copy
+    uint32_t out_sync;   // [2 slots]: the 128 threads that fill a slot's result buffer (host-buffer variant)
     uint32_t w_full, w_empty; // [kMaxStages] each
     uint32_t tmem_holder, abort_flag;
     uint32_t total;
@@ -158,6 +159,7 @@ __host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words
     m.last_full = off; off += 8;
     m.xy_full = off; if (W == 512) off += 16;
     m.xy_empty = off; if (W == 512) off += 16;
+    m.out_sync = off; if (W != 512) off += 16;
     m.drain = off; off += 8;
     m.w_full = off; off += 8 * kMaxStages;
     m.w_empty = off; off += 8 * kMaxStages;
@@ -580,6 +582,7 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
     const uint32_t xy_addr = smem_base + sm.xy + (uint32_t)(((slot * 4 + sub) * kTile + c.row) * 8);
     uint32_t acc_parity = 0, last_parity = 0;
     [[maybe_unused]] uint32_t xy_k = 0; // tiles taken from the bulk-copy buffer so far
+    [[maybe_unused]] uint32_t out_parity = 0;
     const FusedLayer &l1 = p.layer[0];
     const float qmaxf = p.qmaxf;
 
@@ -706,13 +709,16 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
                 ptx::tmem_wait_ld();
                 // Host-buffer variant: a whole tile's results (128 x d_L floats, contiguous in `out`) are
                 // collected in shared memory and leave by one bulk store: over the host link one large
-                // write instead of 128 x d_L four-byte ones.  The slot's 128 sub-0 threads meet on a named
-                // barrier before and after filling the buffer; its first thread issues the store.
+                // write instead of 128 x d_L four-byte ones.  The slot's 128 sub-0 threads meet on an
+                // mbarrier (bounded wait, like every other) before and after filling the buffer; its
+                // first thread issues the store.
                 const bool by_bulk = !AHEAD && !C::BULK_XY && p.bulk_out && (tile + 1) * kTile <= p.n;
                 const uint32_t ot = smem_base + sm.out_tile + (uint32_t)(slot * kTile * 16);
                 if (by_bulk) {
                     if (c.row == 0) ptx::bulk_wait_read(); // the previous tile's store has read the buffer
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + slot) : "memory");
+                    ptx::mbar_arrive(smem_base + sm.out_sync + 8 * slot);
+                    if (!wait_bar_warp<PER_TOKEN>(smem_base + sm.out_sync + 8 * slot, out_parity, abort_flag, p.status)) return;
+                    out_parity ^= 1;
                 }
                 if (valid) {
 #pragma unroll
@@ -728,7 +734,9 @@ __device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t 
                 }
                 if (by_bulk) {
                     ptx::fence_proxy_async();
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + slot) : "memory");
+                    ptx::mbar_arrive(smem_base + sm.out_sync + 8 * slot);
+                    if (!wait_bar_warp<PER_TOKEN>(smem_base + sm.out_sync + 8 * slot, out_parity, abort_flag, p.status)) return;
+                    out_parity ^= 1;
                     if (c.row == 0) ptx::bulk_s2g(p.out + tile * kTile * p.d_L, ot, (uint32_t)(kTile * p.d_L * 4));
                 }
             }
@@ -932,6 +940,9 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
             for (int q = 0; q < 4; ++q) ptx::mbar_init(smem_base + sm.slot_sync + 8 * (s * 4 + q), C::R * 32);
         }
         ptx::mbar_init(smem_base + sm.last_full, 1);
+        if constexpr (!C::BULK_XY) {
+            for (int s2 = 0; s2 < 2; ++s2) ptx::mbar_init(smem_base + sm.out_sync + 8 * s2, kTile);
+        }
         if constexpr (C::BULK_XY) {
             for (int s2 = 0; s2 < 2; ++s2) {
                 ptx::mbar_init(smem_base + sm.xy_full + 8 * s2, 1);
