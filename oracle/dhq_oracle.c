@@ -24,7 +24,10 @@
  * Parity pins (tests/test_oracle_*.py): Hadamard recursion vs closed form and H H^T = nI;
  * rotation vs an exact integer product and vs fp64; W x = (W H/K)(H x); Frobenius norm
  * preservation; quantizer error <= s/2; brute force on 4-wide layers; convergence of the whole
- * network to the unquantized fp64 SIREN as the bit-width grows.
+ * network to the unquantized fp64 SIREN as the bit-width grows; the per-output-channel branch of
+ * the weight quantizer by a hand-derived fixture and row-wise properties; every code of weights
+ * and activations against the same layer stated in fp64 with the orthonormal scaling (they may
+ * differ by one step only where the value to be rounded is within 1e-4 of a half-integer).
  * Parity unpinned by the paper: the order of the fp32 additions inside a rotation (pinned here
  * as a balanced pairwise sum in index order) and the rounding mode / granularity of the
  * quantizer (pinned as stated above).

@@ -2,7 +2,9 @@
 
 TEST INFRASTRUCTURE ONLY.  Used to pin the fp32 oracle (`dhq_oracle.c`): the Hadamard matrix of
 Eq. 3, the two-sided orthonormal transform of Eq. 4-5, and the unquantized SIREN forward that a
-quantized network must approach as the bit-width grows.
+quantized network must approach as the bit-width grows, and one DHQ layer with every step in
+fp64 and the orthonormal scaling (the tier the fp32 oracle's codes are compared with: they may
+differ only by one code step where the value to be rounded sits next to a half-integer).
 """
 from __future__ import annotations
 
@@ -40,3 +42,41 @@ def siren_forward(weights, biases, omega0: float, coords: np.ndarray) -> np.ndar
         z = x @ weights[l].astype(np.float64).T + biases[l].astype(np.float64)
         x = np.sin(omega0 * z) if l < L - 1 else z
     return x
+
+
+def quantize_def(v: np.ndarray, a, bits: int):
+    """The symmetric absmax quantizer of Section III-B in fp64: t = v * qmax / a, q = round half to
+    even of t, clipped to +-qmax; a = 0 gives zeros.  `a` broadcasts against v.  Returns (q, t)."""
+    qmax = float(2 ** (bits - 1) - 1)
+    a = np.broadcast_to(np.asarray(a, dtype=np.float64), v.shape)
+    t = np.divide(v * qmax, a, out=np.zeros_like(v, dtype=np.float64), where=a > 0)
+    return np.clip(np.rint(t), -qmax, qmax).astype(np.int64), t
+
+
+def dhq_layer_def(W, b, X, w_bits: int, a_bits: int, per_channel: bool, per_token: bool, omega0: float,
+                  sine: bool, a_frozen=None):
+    """One DHQ layer exactly as the formulas read, everything in fp64 with the orthonormal scaling
+    of Eq. 5 on the input dimension: W' = W H_K / sqrt(K), x' = H_K x / sqrt(K) (so W' x' = W x),
+    both quantized by the same absmax quantizer, integer product, dequantization, bias, sine.
+    W is the zero-padded [M][K] matrix, X the [n][K] layer inputs.  a_frozen is the per-tensor
+    activation absmax in the orthonormal scaling; None takes the maximum over X.
+    Returns a dict: qw, tw (pre-rounding weight values), codes, t (pre-rounding), acc, Y, a_x."""
+    W = np.asarray(W, dtype=np.float64)
+    X = np.asarray(X, dtype=np.float64)
+    M, K = W.shape
+    H = hadamard(K)
+    Wr = W @ H / np.sqrt(K)
+    Xr = X @ H.T / np.sqrt(K)
+    a_w = np.abs(Wr).max(axis=1, keepdims=True) if per_channel else np.full((M, 1), np.abs(Wr).max())
+    qw, tw = quantize_def(Wr, a_w, w_bits)
+    if per_token:
+        a_x = np.abs(Xr).max(axis=1, keepdims=True)
+    else:
+        a_x = np.full((X.shape[0], 1), np.abs(Xr).max() if a_frozen is None else float(a_frozen))
+    codes, t = quantize_def(Xr, a_x, a_bits)
+    acc = codes @ qw.T
+    s_w = a_w[:, 0] / float(2 ** (w_bits - 1) - 1)
+    s_x = a_x / float(2 ** (a_bits - 1) - 1)
+    z = s_w[None, :] * s_x * acc + np.asarray(b, dtype=np.float64)[None, :]
+    return {"qw": qw, "tw": tw, "codes": codes, "t": t, "acc": acc, "Y": np.sin(omega0 * z) if sine else z,
+            "a_x": a_x[:, 0]}
