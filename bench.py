@@ -6,9 +6,13 @@
     python bench.py --impl reference ...      # the CPU oracle on the host cores, same metric
 
 A step is one dhq_forward call over the workload's whole coordinate grid (one launch of the
-fused kernel).  Inputs are seeded and synthetic (SIREN-initialised network, pixel grid).  With
+fused kernel).  The default workload is the largest single-GPU configuration, C5 (width 512,
+2048 x 2048 grid); the other configurations are timed briefly in the same process and listed under
+"per_config".  Inputs are seeded and synthetic (SIREN-initialised network, pixel grid).  With
 N > 1 every rank runs the same grid on its own GPU (independent replicas, no collective on the
-data path), so the aggregate is N times the work: weak scaling.
+data path), so the aggregate is N times the work: weak scaling; with --shard the one grid is
+split over the ranks instead (per-tensor scales frozen with an all-reduce(max) per layer):
+strong scaling.
 
 Timing: CUDA events on the launching stream around each step, an L2 flush (a write of a buffer
 larger than L2) between steps and outside the events, the per-step times summed; the maximum
@@ -31,9 +35,12 @@ import numpy as np  # noqa: E402
 
 import dhq_inputs  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one fused-kernel launch, from the ncu capture
-# summarised in profiles/fused_kernel_w256_C2.md (full C2 grid, rotation on).
-NCU_DRAM_BYTES_PER_LAUNCH = {("C2", "input", 65536): 780032 + 0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one fused-kernel launch as ncu counted it, per
+# workload (rotation on): (bytes, coordinates of the captured launch).  Captures of the large grids
+# cover a few hundred thousand coordinates; a launch's traffic is the weights once plus a fixed
+# amount per coordinate, so it is scaled to the timed launch by the coordinate count.  An entry is
+# removed (traffic: null) when the kernel changes after its capture.
+NCU_DRAM_BYTES = {}
 METRIC = "coords/sec, fused W8A8 DHQ INR forward"
 UNIT = "coords/s"
 SM_COUNT = 148
@@ -126,41 +133,67 @@ def work_per_coord(dims, rotate=True):
     return macs, sines, fp32
 
 
-def time_oracle(workload, steps, warmup, sample_tokens, rotate=True, min_seconds=0.0):
-    """The CPU oracle, as it stands, on `sample_tokens` coordinates of the workload; with
-    min_seconds the passes repeat until that much CPU time has been measured."""
+SAMPLE_TOKENS = 16384   # coordinates per pass of the CPU oracle (cpu_baseline and --impl reference)
+
+
+def oracle_sample(workload, rotation="input"):
+    """The bounded sample both CPU legs run: a contiguous block of SAMPLE_TOKENS coordinates from
+    the middle of the workload's grid (the whole grid if it is smaller)."""
+    coords = workload.coords()
+    n = min(coords.shape[0], SAMPLE_TOKENS)
+    lo = (coords.shape[0] - n) // 2
+    desc = (f"{n} consecutive coordinates from the middle of the {workload.grid[0]}x{workload.grid[1]} grid "
+            f"(tokens {lo}..{lo + n - 1}) per pass")
+    return np.ascontiguousarray(coords[lo:lo + n]), desc
+
+
+def time_oracle(workload, steps, warmup, rotate=True, min_seconds=0.0, variant="definition"):
+    """The CPU oracle, as it stands, on the bounded sample of the workload; with min_seconds the
+    passes repeat until that much time has been measured.  variant "definition" is the parity
+    reference (O(n^2) rotation, as the paper's formula reads); "nlogn" the same layer with the
+    rotation as a butterfly.  Returns (coords/s, seconds per pass, threads, passes, sample text)."""
     from oracle import dhq_oracle as orc
+    from oracle import dhq_oracle_nlogn as orcn
     weights, biases = workload.network()
     net = orc.prepare(weights, biases, workload.dims, workload.omega0, workload.w_bits, workload.a_bits,
                       workload.w_gran, workload.a_gran, rotate=rotate)
-    coords = workload.coords()[:sample_tokens]
+    coords, desc = oracle_sample(workload)
     if workload.a_gran == 0:
         orc.calibrate(net, coords)
+    fwd = orc.forward if variant == "definition" else orcn.forward
     for _ in range(warmup):
-        orc.forward(net, coords[: max(1, sample_tokens // 8)])
+        fwd(net, coords[: max(1, coords.shape[0] // 8)])
     t0 = time.perf_counter()
     done = 0
     while done < steps or time.perf_counter() - t0 < min_seconds:
-        orc.forward(net, coords)
+        fwd(net, coords)
         done += 1
     dt = (time.perf_counter() - t0) / done
-    return coords.shape[0] / dt, dt, orc.threads(), done
+    return coords.shape[0] / dt, dt, orc.threads(), done, desc
+
+
+def config_of(workload, args, world):
+    """The `config` object of the JSON line, the same for both arms."""
+    mode = "one grid split over the ranks" if args.shard else "independent replica(s)"
+    return {"workload": workload.name, "dims": list(workload.dims), "coords_per_step": workload.n if args.limit_coords <= 0 else min(workload.n, args.limit_coords),
+            "bits": [workload.w_bits, workload.a_bits], "w_gran": workload.w_gran, "a_gran": workload.a_gran,
+            "rotation": args.rotation, "l2": "flushed between steps (256 MB write)",
+            "parallelism": f"{world} x {mode}"}
 
 
 def run_reference(args, workload):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample = min(workload.n, 16384)
     steps = max(1, min(args.steps, 5))
     warmup = min(args.warmup, 1)
-    value, dt, cores, _ = time_oracle(workload, steps, warmup, sample, rotations(args.rotation))
-    desc = f"first {sample} coordinates of the {workload.grid[0]}x{workload.grid[1]} grid per step"
+    value, dt, cores, _, desc = time_oracle(workload, steps, warmup, rotations(args.rotation))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "strong" if args.shard else "weak",
         "vs_baseline": None, "dtype": "int8 (int64 accumulate, f64 epilogue)", "data": "synthetic",
-        "config": {"workload": workload.name, "dims": list(workload.dims), "bits": [workload.w_bits, workload.a_bits]},
+        "config": config_of(workload, args, int(os.environ.get("WORLD_SIZE", "1"))),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -178,9 +211,107 @@ def max_over_ranks(values, world, device):
     return [float(v) for v in t]
 
 
-def aggregate_throughput(coords_per_rank, world, ms_per_step):
-    """Whole-job coordinates per second: every rank runs its own replica of the grid."""
-    return coords_per_rank * world / (ms_per_step * 1e-3)
+def aggregate_throughput(total_coords, ms_per_step):
+    """Whole-job coordinates per second: all coordinates all ranks processed in a step over the
+    slowest rank's step time."""
+    return total_coords / (ms_per_step * 1e-3)
+
+
+class Runner:
+    """One workload on this rank's GPU: handle, device and pinned host buffers, timed loops."""
+
+    def __init__(self, dhq, workload, rotation, limit_coords=0, shard=None, group=None):
+        import torch
+        self.dhq, self.torch, self.workload = dhq, torch, workload
+        weights, biases = workload.network()
+        coords_np = workload.coords()
+        if limit_coords > 0:
+            coords_np = coords_np[:limit_coords]
+        self.n_total = coords_np.shape[0]
+        if shard is not None:                      # (rank, world): this rank's contiguous block
+            lo, hi = dhq.shard_range(self.n_total, shard[0], shard[1])
+            coords_np = coords_np[lo:hi]
+        coords_np = np.ascontiguousarray(coords_np)
+        self.n, self.d_L = coords_np.shape[0], workload.dims[-1]
+        self.h = dhq.dhq_prepare(workload.dims, [torch.from_numpy(w).cuda() for w in weights],
+                                 [torch.from_numpy(b).cuda() for b in biases], workload.omega0, workload.w_bits,
+                                 workload.a_bits, workload.w_gran, workload.a_gran,
+                                 rotation={"input": 0, "both": 1, "none": 2}[rotation])
+        self.coords = torch.from_numpy(coords_np).cuda()
+        self.out = torch.empty((self.n, self.d_L), dtype=torch.float32, device="cuda")
+        self.coords_host = torch.from_numpy(coords_np).pin_memory()
+        self.out_host = torch.empty((self.n, self.d_L), dtype=torch.float32).pin_memory()
+        self.stream = torch.cuda.current_stream()
+        # per-tensor scales frozen on the workload's grid (all ranks' blocks together); no-op per token
+        if shard is not None:
+            dhq.calibrate_sharded(self.h, self.coords, len(workload.dims) - 1, group=group)
+        else:
+            dhq.dhq_calibrate(self.h, self.coords)
+
+    def warm(self, steps, e2e=True):
+        for _ in range(steps):
+            self.dhq.dhq_forward(self.h, self.coords, self.out)
+            if e2e:
+                self.dhq.dhq_forward_host(self.h, self.coords_host, self.out_host)
+        self.torch.cuda.synchronize()
+        if self.dhq.dhq_last_status(self.h) != 0:
+            raise SystemExit("device-side wait timed out during warm-up")
+
+    def timed(self, fn, steps, flush, barrier):
+        torch = self.torch
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        barrier()
+        for a, b in evs:
+            flush.fill_(1)
+            a.record(self.stream)
+            fn()
+            b.record(self.stream)
+        barrier()
+        return sum(a.elapsed_time(b) for a, b in evs)   # ms
+
+    def forward(self):
+        self.dhq.dhq_forward(self.h, self.coords, self.out)
+
+    def forward_host(self):
+        self.dhq.dhq_forward_host(self.h, self.coords_host, self.out_host)
+
+    def close(self):
+        self.dhq.dhq_destroy(self.h)
+
+
+def packed_weight_bytes(dims):
+    """Bytes of the prepared int8 weights a launch reads once (tensor-core images of the hidden and
+    last layers, one word per feature for the first)."""
+    w, hidden_matmuls = dims[1], len(dims) - 3
+    return 4 * w + hidden_matmuls * w * w + 16 * w
+
+
+def dram_traffic(workload, rotation, n):
+    """DRAM bytes of one launch over n coordinates from the kept ncu counters: the captured launch's
+    bytes beyond the weights grow with the coordinate count, the weights are read once."""
+    entry = NCU_DRAM_BYTES.get((workload.name, rotation))
+    if entry is None:
+        return None
+    captured, coords = entry
+    fixed = min(packed_weight_bytes(workload.dims), captured)
+    return fixed + (captured - fixed) * (n / coords)
+
+
+def roofline_of(workload, rotation, n, ms_per_step, sm_max_mhz, sampled_mhz, fma_peak):
+    """ALU roofline of one launch: algorithmic lane-ops over the CUDA-event duration, against (a) the
+    derived peak SMs x fp32 lanes x max SM clock, (b) the same at the SM clock sampled during the
+    timed steps, (c) the FMA loop's rate measured in this run."""
+    achieved = alu_laneops_per_coord(workload.dims, rotations(rotation)) * n / (ms_per_step * 1e-3) / 1e12
+    peak = SM_COUNT * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    r = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tlaneop/s", "frac": achieved / peak,
+         "peak_source": "148 SMs x 128 fp32 lanes x max SM clock (derived from unit counts and clock)"}
+    if sampled_mhz:
+        r["frac_at_sampled_clock"] = achieved / (SM_COUNT * FP32_LANES_PER_SM * sampled_mhz * 1e6 / 1e12)
+    if fma_peak:
+        r["peak_measured_fma"] = fma_peak / 1e12
+        r["frac_of_measured_fma"] = achieved / (fma_peak / 1e12)
+    r["traffic"] = dram_traffic(workload, rotation, n)
+    return r
 
 
 def run_ours(args, workload):
@@ -197,58 +328,29 @@ def run_ours(args, workload):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dhq.load_library()
-
-    weights, biases = workload.network()
-    coords_np = workload.coords()
-    if args.limit_coords > 0:
-        coords_np = np.ascontiguousarray(coords_np[: args.limit_coords])
-    n, d_L = coords_np.shape[0], workload.dims[-1]
-    W = [torch.from_numpy(w).cuda() for w in weights]
-    B = [torch.from_numpy(b).cuda() for b in biases]
-    h = dhq.dhq_prepare(workload.dims, W, B, workload.omega0, workload.w_bits, workload.a_bits,
-                        workload.w_gran, workload.a_gran, rotation={"input": 0, "both": 1, "none": 2}[args.rotation])
-    coords = torch.from_numpy(coords_np).cuda()
-    out = torch.empty((n, d_L), dtype=torch.float32, device="cuda")
-    coords_host = torch.from_numpy(coords_np).pin_memory()
-    out_host = torch.empty((n, d_L), dtype=torch.float32).pin_memory()
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # > 126 MB of L2
-    stream = torch.cuda.current_stream()
-
-    dhq.dhq_calibrate(h, coords)          # per-tensor scales frozen on the workload's grid; no-op per token
-    for _ in range(max(args.warmup, 3)):
-        dhq.dhq_forward(h, coords, out)
-        dhq.dhq_forward_host(h, coords_host, out_host)
-    torch.cuda.synchronize()
-    if dhq.dhq_last_status(h) != 0:
-        raise SystemExit("device-side wait timed out during warm-up")
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps):
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        barrier()
-        for a, b in evs:
-            flush.fill_(1)
-            a.record(stream)
-            fn()
-            b.record(stream)
-        barrier()
-        return sum(a.elapsed_time(b) for a, b in evs)   # ms
-
-    launches0 = dhq.dhq_launch_count(h)
+    run = Runner(dhq, workload, args.rotation, args.limit_coords, shard=(rank, world) if args.shard else None)
+    n = run.n
+    warmup = max(args.warmup, 3)
+    run.warm(warmup)
+    launches0 = dhq.dhq_launch_count(run.h)
     with ClockSampler(physical_gpu_index(local_rank)) as clocks:
-        total_ms = timed(lambda: dhq.dhq_forward(h, coords, out), args.steps)
-    launches = dhq.dhq_launch_count(h) - launches0
-    e2e_ms = timed(lambda: dhq.dhq_forward_host(h, coords_host, out_host), args.steps)
-    status = dhq.dhq_last_status(h)
+        total_ms = run.timed(run.forward, args.steps, flush, barrier)
+    launches = dhq.dhq_launch_count(run.h) - launches0
+    e2e_ms = run.timed(run.forward_host, args.steps, flush, barrier)
+    status = dhq.dhq_last_status(run.h)
 
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, "cuda")
     ms_per_step = total_ms / args.steps
-    value = aggregate_throughput(n, world, ms_per_step)
-    e2e_value = aggregate_throughput(n, world, e2e_ms / args.steps)
+    coords_per_step = run.n_total if args.shard else n * world
+    value = aggregate_throughput(coords_per_step, ms_per_step)
+    e2e_value = aggregate_throughput(coords_per_step, e2e_ms / args.steps)
 
     if rank == 0:
         peaks = {}
@@ -257,28 +359,25 @@ def run_ours(args, workload):
         except Exception:
             pass
         sm_max = float(peaks.get("sm_max_mhz", 1965.0))
-        alu_peak = SM_COUNT * FP32_LANES_PER_SM * sm_max * 1e6 / 1e12            # T lane-ops/s
-        achieved = alu_laneops_per_coord(workload.dims, rotations(args.rotation)) * n / (ms_per_step * 1e-3) / 1e12
+        csum = clocks.summary()
+        try:
+            fma_peak, _ = dhq.dhq_measure_pipe("ffma", 2000)
+        except Exception:
+            fma_peak = None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int8 (int32 accumulate, f32 epilogue)",
-            "data": "synthetic",
-            "config": {"workload": workload.name, "dims": list(workload.dims), "coords_per_step": n,
-                       "bits": [workload.w_bits, workload.a_bits], "w_gran": workload.w_gran,
-                       "a_gran": workload.a_gran, "rotation": args.rotation, "l2": "flushed between steps (256 MB write)",
-                       "parallelism": f"{world} independent replica(s)"},
-            "clocks": clocks.summary(),
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * 8, "d2h_bytes_per_step": n * d_L * 4,
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "strong" if args.shard else "weak", "vs_baseline": None,
+            "dtype": "int8 (int32 accumulate, f32 epilogue)", "data": "synthetic",
+            "config": config_of(workload, args, world),
+            "clocks": csum,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * 8, "d2h_bytes_per_step": n * run.d_L * 4,
                     "ms_per_step": e2e_ms / args.steps,
                     "route": "dhq_forward_host on pinned host buffers: the kernel reads the coordinates and writes "
                              "the result over the host link through the buffers' device mapping, every step "
                              "(whole tiles by bulk copy where the width's kernel has that variant)"},
             "gpu_launches": launches,
-            "roofline": {"bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "Tlaneop/s",
-                         "frac": achieved / alu_peak,
-                         "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((workload.name, args.rotation, n)),
-                         "peak_source": "148 SMs x 128 fp32 lanes x max SM clock (derived, not measured)"},
+            "roofline": roofline_of(workload, args.rotation, n, ms_per_step, sm_max, csum["sm_mhz"], fma_peak),
             "device_status": status,
         }
         # The same launch against the other pipes' ceilings, each measured now on this GPU by the
@@ -305,13 +404,40 @@ def run_ours(args, workload):
             except Exception as exc:
                 pipes["inner_loops_alone"] = {"error": str(exc)}
         line["pipes"] = pipes
+    run.close()
+
+    # The other configurations, briefly, in the same process (one GPU, the default invocation only).
+    if world == 1 and not args.no_per_config and args.limit_coords <= 0 and args.rotation == "input":
+        per = {}
+        for name in sorted(dhq_inputs.WORKLOADS):
+            if name == workload.name:
+                continue
+            other = dhq_inputs.WORKLOADS[name]
+            r = Runner(dhq, other, args.rotation)
+            steps = max(10, min(args.steps, 100))
+            r.warm(3, e2e=False)
+            with ClockSampler(physical_gpu_index(local_rank)) as ck:
+                ms = r.timed(r.forward, steps, flush, barrier) / steps
+            st = dhq.dhq_last_status(r.h)
+            roof = roofline_of(other, args.rotation, r.n, ms, sm_max, ck.summary()["sm_mhz"], fma_peak)
+            per[name] = {"coords_per_step": r.n, "steps": steps, "ms_per_step": ms, "value": r.n / (ms * 1e-3),
+                         "roofline_frac": roof["frac"], "frac_of_measured_fma": roof.get("frac_of_measured_fma"),
+                         "traffic": roof["traffic"], "device_status": st}
+            r.close()
+        line["per_config"] = per
+
+    if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            sample = min(n, 65536)
-            v, dt, cores, passes = time_oracle(workload, 1, 1, sample, rotations(args.rotation), min_seconds=10.0)
+            v, dt, cores, passes, desc = time_oracle(workload, 1, 1, rotations(args.rotation), min_seconds=10.0)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                    "sample": f"first {sample} coordinates of the grid, {passes} pass(es) of {dt:.1f} s"}
+                                    "sample": f"{desc}, {passes} pass(es) of {dt:.1f} s",
+                                    "rotation": "O(n^2) product with the explicit Hadamard matrix (the definition)"}
+            if args.rotation != "both":
+                v2, dt2, _, passes2, _ = time_oracle(workload, 1, 1, rotations(args.rotation), min_seconds=5.0, variant="nlogn")
+                line["cpu_baseline"]["nlogn_variant"] = {"value": v2, "unit": UNIT, "cores": cores,
+                                                         "sample": f"same sample, {passes2} pass(es) of {dt2:.1f} s",
+                                                         "rotation": "O(n log n) butterfly, bit-identical results"}
         print(json.dumps(line), flush=True)
-    dhq.dhq_destroy(h)
     if world > 1:
         dist.destroy_process_group()
 
@@ -362,14 +488,17 @@ def run_sweep(args, workload):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C2", choices=sorted(dhq_inputs.WORKLOADS))
+    ap.add_argument("--workload", default="C5", choices=sorted(dhq_inputs.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--shard", action="store_true",
+                    help="with N > 1 ranks: split the one grid over the ranks (strong scaling) instead of N replicas")
     ap.add_argument("--rotation", default="input", choices=["input", "none", "both"],
                     help="input = DHQ; none = the same path without the Hadamard rotation (uniform quantizer); "
-                         "both = the two-sided transform of Eq. 4-5, run layer by layer")
+                         "both = the two-sided transform of Eq. 4-5")
     ap.add_argument("--limit-coords", type=int, default=0,
                     help="use only the first N coordinates of the workload's grid (profiling captures)")
     ap.add_argument("--sweep", action="store_true", help="batch-size sweep 2^12..2^24 instead of the timed steps")

@@ -33,7 +33,7 @@
  *     the device (a bounded wait that ran out) are recorded in a status word read by
  *     dhq_last_status.  Nothing traps, aborts or throws.
  *   - One forward may be in flight per handle at a time.  Handles belong to the device that was
- *     current in dhq_prepare; that device must be current in later calls.
+ *     current in dhq_prepare; that device must be current in later calls (INVALID_ARG otherwise).
  */
 #ifndef DHQ_H_
 #define DHQ_H_
@@ -199,6 +199,45 @@ DHQ_API dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int6
                                        const dhq_debug_bufs_t *bufs, void *stream);
 
 /*
+ * The forward pass by the fused kernel itself, observed: the same kernel as dhq_forward (one
+ * launch, tensor-core products, activations staying on the SM; Section III-C's dataflow) compiled
+ * with stores added at the places where each per-layer value exists - the codes as they go into
+ * the tensor-core operand tile, the activation scale, the int32 accumulators as they are read
+ * from tensor memory, the layer output after the sine.  Same arithmetic, instruction for
+ * instruction, so `out` equals dhq_forward's bit for bit; it runs slower because of the stores.
+ *   bufs   as for dhq_forward_debug.  Inside the fused kernel the input of layer l+1 is the output
+ *          of layer l (one value): X[l] receives a copy of Y[l-1].  The first layer's accumulators
+ *          are never formed on the per-tensor route (its phase is built from the two distinct
+ *          input codes); acc[0] holds codes . weight codes computed for the dump.
+ *          X[0] must be 16-byte aligned, the other buffers 4-byte aligned.
+ * Requires frozen scales when a_gran = per tensor (NOT_CALIBRATED otherwise).  DHQ_ROT_BOTH runs
+ * layer by layer and is observed by dhq_forward_debug: UNSUPPORTED here.
+ * Errors: INVALID_ARG, UNSUPPORTED, NOT_CALIBRATED, CUDA.
+ */
+DHQ_API dhq_status_t dhq_forward_fused_debug(dhq_handle_t h, const float *coords, int64_t n, float *out,
+                                             const dhq_debug_bufs_t *bufs, void *stream);
+
+/*
+ * Bound of the waits inside the fused kernel.  Its warps hand tiles to each other through
+ * barriers in shared memory; every such wait gives up after this long, the kernel then records
+ * DHQ_ERR_TIMEOUT in the handle's status word (dhq_last_status), releases what it holds and
+ * returns, so that a stall never holds the GPU.  Default 2 s; at least 1000 ns.  Takes effect
+ * with the next launch.  (The paper's pipeline has no counterpart: an FPGA pipeline cannot
+ * stall this way.)
+ */
+DHQ_API dhq_status_t dhq_set_wait_limit(dhq_handle_t h, int64_t nanoseconds);
+
+/*
+ * Test hook for that bound: the next fused-kernel launch of this handle (dhq_forward or the
+ * pinned route of dhq_forward_host) leaves out the copy of the last layer's weights into shared
+ * memory.  Nothing is in flight for the missing piece; the warps that wait for it run into the
+ * wait limit, the kernel returns, `out` holds unspecified values and dhq_last_status reports
+ * DHQ_ERR_TIMEOUT.  Later launches are normal.  Set a short limit first (dhq_set_wait_limit).
+ * UNSUPPORTED for DHQ_ROT_BOTH (no fused kernel).
+ */
+DHQ_API dhq_status_t dhq_debug_stall_next_forward(dhq_handle_t h);
+
+/*
  * Read back one prepared layer (1-based).  Synchronizes the handle's preparation work.
  *   codes       host [M][K] int8, row-major, unswizzled (M, K as in dhq_debug_bufs_t), or NULL.
  *   w_scales    host [M] fp32 (per-tensor: the same value M times), or NULL.
@@ -240,6 +279,23 @@ DHQ_API dhq_status_t dhq_get_layer(dhq_handle_t h, int layer, int8_t *codes, flo
 #define DHQ_STATIC_MAX_TOKENS 4096
 DHQ_API dhq_status_t dhq_forward_static_scratch(dhq_handle_t h, const float *coords, int64_t n,
                                                 float *out, void *stream);
+
+/*
+ * A prepared (and, if it was, calibrated) handle as a block of host memory, and back: so that the
+ * weight-side work of Eq. 4-5 and the calibration run once and every GPU or process that serves
+ * the same network (coordinates are independent, Section II-A, so the work splits over GPUs by
+ * coordinate blocks) starts from the same bytes.
+ *   dhq_export  host_buf NULL: only *needed is written (size query).  Otherwise capacity must be
+ *               >= *needed (TOO_LARGE if not); synchronizes the device and fills host_buf.
+ *   dhq_import  builds a new handle on the current device from such a block; the block is
+ *               checked (magic, version, sizes against the configuration it states, checksum of
+ *               the arrays): INVALID_ARG if anything is off.  The caller may release host_buf when
+ *               the call returns.  Results of the new handle equal the exported one's bit for bit.
+ * The block is the library's own format, valid for this library version and sm_100a layouts.
+ * Errors: INVALID_ARG, UNSUPPORTED, TOO_LARGE, ALLOC, CUDA.
+ */
+DHQ_API dhq_status_t dhq_export(dhq_handle_t h, void *host_buf, int64_t capacity, int64_t *needed);
+DHQ_API dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_handle_t *out);
 
 /* Layer sizes as the library pads them: K, M of layer `layer` (1-based).  Either may be NULL. */
 DHQ_API dhq_status_t dhq_layer_dims(dhq_handle_t h, int layer, int *K, int *M);

@@ -49,6 +49,19 @@ typedef enum {
  */
 DHQ_PEAKS_API int dhq_measure_pipe(int pipe, int iters, void *stream, double *ops_per_s, double *ms);
 
+/*
+ * Accuracy of the sine the epilogue uses (the activation of Section III-C's input and linear
+ * layers), measured on the current device: the largest |f(x) - sin(x)| over `count` fp32
+ * arguments spread evenly over [lo, hi], against the fp64 sine of the same argument.
+ *   mode 0: the hardware approximation sin.approx.f32 alone (what the fast epilogue applies to
+ *           phases below its limit); mode 1: with the explicit two-part 2 pi reduction in front
+ *           (the wide epilogue).
+ * The fast epilogue's phase limit follows from this curve and the 1e-5 output tolerance.
+ * Synchronizes `stream`.  Returns 0, or a negative value on bad arguments or a CUDA error.
+ */
+DHQ_PEAKS_API int dhq_measure_sine_error(float lo, float hi, long long count, int mode, void *stream,
+                                         double *max_abs_err);
+
 #ifdef __cplusplus
 }
 #endif

@@ -135,16 +135,21 @@ ORC_API float dhq_orc_absmax(const float *v, int64_t count)
     return a;
 }
 
-/* Symmetric absmax quantizer scales: s = a/qmax, inv = qmax/a (fp32 divisions); a = 0 -> 0, 0. */
+/* Symmetric absmax quantizer scales: s = a/qmax, inv = qmax/a (fp32 divisions); a = 0 -> 0, 0.
+ * Reading of the "standard quantizer" (Section III-B) at its degenerate end: an absmax so small
+ * that qmax/a overflows fp32 (a below about 3.7e-37 at 8 bits) has no finite scale to round
+ * with; it is treated like a = 0 (all codes zero, s = 0). */
 ORC_API void dhq_orc_scales(float a, int bits, float *s, float *inv)
 {
     float qmax = (float)((1 << (bits - 1)) - 1);
+    *s = 0.0f;
+    *inv = 0.0f;
     if (a > 0.0f) {
-        *s = a / qmax;
-        *inv = qmax / a;
-    } else {
-        *s = 0.0f;
-        *inv = 0.0f;
+        float i = qmax / a;
+        if (!isinf(i)) {
+            *s = a / qmax;
+            *inv = i;
+        }
     }
 }
 

@@ -64,7 +64,7 @@ ORC_API int dhq_orcn_layer(const float *X, int64_t n, int K_pad, int M_pad, cons
                 }
             }
             float s = 0.0f, inv = 0.0f;
-            if (a > 0.0f) {
+            if (a > 0.0f && !isinf(qmaxf / a)) { /* no finite scale: treated like a = 0 */
                 s = a / qmaxf;
                 inv = qmaxf / a;
             }

@@ -69,6 +69,12 @@ def load_library():
     L.dhq_forward_static_scratch.argtypes = [vp, vp, c_i64, vp, vp]
     L.dhq_forward_static_scratch.restype = c_i
     L.dhq_forward_debug.argtypes = [vp, vp, c_i64, vp, ctypes.POINTER(_DebugBufs), vp]
+    L.dhq_forward_fused_debug.argtypes = [vp, vp, c_i64, vp, ctypes.POINTER(_DebugBufs), vp]
+    L.dhq_set_wait_limit.argtypes = [vp, c_i64]
+    L.dhq_export.argtypes = [vp, vp, c_i64, ctypes.POINTER(c_i64)]
+    L.dhq_import.argtypes = [ctypes.c_char_p, c_i64, vp, ctypes.POINTER(vp)]
+    L.dhq_debug_stall_next_forward.argtypes = [vp]
+    L.dhq_measure_sine_error.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_longlong, c_i, vp, ctypes.POINTER(ctypes.c_double)]
     L.dhq_get_layer.argtypes = [vp, c_i, vp, vp, vp]
     L.dhq_layer_dims.argtypes = [vp, c_i, ctypes.POINTER(c_i), ctypes.POINTER(c_i)]
     L.dhq_last_status.argtypes = [vp]
@@ -79,7 +85,8 @@ def load_library():
     L.dhq_status_string.argtypes = [c_i]
     L.dhq_status_string.restype = ctypes.c_char_p
     L.dhq_measure_pipe.argtypes = [c_i, c_i, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
-    for name in ("dhq_calibrate_layer", "dhq_get_act_absmax", "dhq_set_act_absmax"):
+    for name in ("dhq_calibrate_layer", "dhq_get_act_absmax", "dhq_set_act_absmax", "dhq_forward_fused_debug",
+                 "dhq_set_wait_limit", "dhq_debug_stall_next_forward", "dhq_measure_sine_error", "dhq_export", "dhq_import"):
         getattr(L, name).restype = c_i
     for name in ("dhq_prepare", "dhq_calibrate", "dhq_forward", "dhq_forward_host", "dhq_forward_debug",
                  "dhq_get_layer", "dhq_layer_dims", "dhq_last_status", "dhq_measure_pipe"):
@@ -94,6 +101,8 @@ def dhq_status_string(code: int) -> str:
 
 def _stream_ptr(stream):
     if stream is None:
+        if not torch.cuda.is_available():      # argument checks of the library can still be exercised
+            return ctypes.c_void_p(None)
         stream = torch.cuda.current_stream()
     return ctypes.c_void_p(stream.cuda_stream)
 
@@ -183,9 +192,10 @@ def dhq_layer_dims(handle, layer):
     return K.value, M.value
 
 
-def dhq_forward_debug(handle, coords, out=None, bufs=None, stream=None):
+def dhq_forward_debug(handle, coords, out=None, bufs=None, stream=None, fused=False):
     """bufs: dict with any of 'X', 'codes', 's_x', 'acc', 'Y', each a list of L CUDA tensors or
-    None entries (dtypes fp32, int8, fp32, int32, fp32)."""
+    None entries (dtypes fp32, int8, fp32, int32, fp32).  fused=True calls dhq_forward_fused_debug:
+    the same dumps written from inside the fused kernel."""
     n = coords.shape[0]
     dtypes = {"X": torch.float32, "codes": torch.int8, "s_x": torch.float32, "acc": torch.int32, "Y": torch.float32}
     st = _DebugBufs()
@@ -203,10 +213,31 @@ def dhq_forward_debug(handle, coords, out=None, bufs=None, stream=None):
             arr = (ctypes.c_void_p * len(lst))(*[_dev_ptr(t, dt, key) for t in lst])
             keep.append(arr)
             setattr(st, key, arr)
-    _check(load_library().dhq_forward_debug(handle, _dev_ptr(coords, torch.float32, "coords"), n,
-                                            _dev_ptr(out, torch.float32, "out"),
-                                            ctypes.byref(st) if bufs else None, _stream_ptr(stream)),
-           "dhq_forward_debug")
+    fn = load_library().dhq_forward_fused_debug if fused else load_library().dhq_forward_debug
+    _check(fn(handle, _dev_ptr(coords, torch.float32, "coords"), n, _dev_ptr(out, torch.float32, "out"),
+              ctypes.byref(st) if bufs else None, _stream_ptr(stream)),
+           "dhq_forward_fused_debug" if fused else "dhq_forward_debug")
+
+
+def dhq_forward_fused_debug(handle, coords, out, bufs=None, stream=None):
+    dhq_forward_debug(handle, coords, out, bufs, stream, fused=True)
+
+
+def dhq_set_wait_limit(handle, nanoseconds: int):
+    _check(load_library().dhq_set_wait_limit(handle, int(nanoseconds)), "dhq_set_wait_limit")
+
+
+def dhq_debug_stall_next_forward(handle):
+    _check(load_library().dhq_debug_stall_next_forward(handle), "dhq_debug_stall_next_forward")
+
+
+def dhq_measure_sine_error(lo, hi, count=1 << 22, mode=0, stream=None) -> float:
+    """Largest |f(x) - sin(x)| over `count` fp32 arguments in [lo, hi] (see dhq_peaks.h)."""
+    err = ctypes.c_double()
+    rc = load_library().dhq_measure_sine_error(float(lo), float(hi), int(count), int(mode), _stream_ptr(stream), ctypes.byref(err))
+    if rc != 0:
+        raise RuntimeError(f"dhq_measure_sine_error failed with {rc}")
+    return err.value
 
 
 def dhq_get_layer(handle, layer):
@@ -218,6 +249,23 @@ def dhq_get_layer(handle, layer):
     _check(load_library().dhq_get_layer(handle, int(layer), codes.ctypes.data_as(ctypes.c_void_p),
                                         scales.ctypes.data_as(ctypes.c_void_p), ctypes.byref(a)), "dhq_get_layer")
     return codes, scales, float(a.value)
+
+
+def dhq_export(handle) -> bytes:
+    """The prepared handle as a block of bytes (see dhq.h)."""
+    L = load_library()
+    need = ctypes.c_int64()
+    _check(L.dhq_export(handle, None, 0, ctypes.byref(need)), "dhq_export")
+    buf = ctypes.create_string_buffer(need.value)
+    _check(L.dhq_export(handle, buf, need.value, ctypes.byref(need)), "dhq_export")
+    return buf.raw
+
+
+def dhq_import(blob: bytes, stream=None):
+    """A new handle on the current device from an exported block."""
+    out = ctypes.c_void_p()
+    _check(load_library().dhq_import(blob, len(blob), _stream_ptr(stream), ctypes.byref(out)), "dhq_import")
+    return out.value
 
 
 def dhq_last_status(handle) -> int:

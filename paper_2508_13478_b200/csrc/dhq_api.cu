@@ -21,16 +21,100 @@ template <typename T> bool dev_alloc(T **p, size_t count)
     return cudaMalloc((void **)p, count * sizeof(T) < 16 ? 16 : count * sizeof(T)) == cudaSuccess;
 }
 
+// Every device array of a prepared layer with its size in bytes, in a fixed order (allocation,
+// release, export and import all walk this table).  Needs d.K, d.M, d.Mt.
+struct ArrayRef { void **ptr; size_t bytes; };
+constexpr int kLayerArrays = 16;
+void layer_arrays(LayerDev &d, ArrayRef (&t)[kLayerArrays])
+{
+    const size_t MK = (size_t)d.M * d.K, M = (size_t)d.M;
+    int i = 0;
+    t[i++] = {(void **)&d.w_rot, MK * 4};
+    t[i++] = {(void **)&d.row_absmax, M * 4};
+    t[i++] = {(void **)&d.row_l1, M * 4};
+    t[i++] = {(void **)&d.qw, MK};
+    t[i++] = {(void **)&d.qw_k4m, MK};
+    t[i++] = {(void **)&d.qw_umma, (size_t)d.Mt * (d.K < 16 ? 16 : d.K)};
+    t[i++] = {(void **)&d.s_w, M * 4};
+    t[i++] = {(void **)&d.inv_w, M * 4};
+    t[i++] = {(void **)&d.bias, M * 4};
+    t[i++] = {(void **)&d.cA, M * 4};
+    t[i++] = {(void **)&d.cA_lo, M * 4};
+    t[i++] = {(void **)&d.cB, M * 4};
+    t[i++] = {(void **)&d.fxP, M * 4};
+    t[i++] = {(void **)&d.fxQ, M * 4};
+    t[i++] = {(void **)&d.fxB, M * 4};
+    t[i++] = {(void **)&d.act, 16};
+}
+
+bool alloc_layer(LayerDev &d)
+{
+    ArrayRef t[kLayerArrays];
+    layer_arrays(d, t);
+    for (const ArrayRef &a : t)
+        if (cudaMalloc(a.ptr, a.bytes < 16 ? 16 : a.bytes) != cudaSuccess) return false;
+    return true;
+}
+
 void free_layer(LayerDev &d)
 {
-    cudaFree(d.w_rot); cudaFree(d.row_absmax); cudaFree(d.qw); cudaFree(d.qw_k4m); cudaFree(d.qw_umma);
-    cudaFree(d.s_w); cudaFree(d.inv_w); cudaFree(d.bias); cudaFree(d.cA); cudaFree(d.cA_lo); cudaFree(d.cB);
-    cudaFree(d.fxP); cudaFree(d.fxQ); cudaFree(d.fxB);
-    cudaFree(d.act);
+    ArrayRef t[kLayerArrays];
+    layer_arrays(d, t);
+    for (const ArrayRef &a : t) cudaFree(*a.ptr);
     d = LayerDev();
 }
 
-bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+// Padded sizes of layer l (1-based) of a network of hidden width w.
+void set_layer_dims(LayerDev &d, int l, int L, int w, const int *dims)
+{
+    d.K = (l == 1) ? 4 : w;
+    d.M = (l == L) ? 4 : w;
+    d.Mt = d.M < 16 ? 16 : d.M;
+    d.slab_k = fused_slab_k(d.K, d.Mt);
+    d.d_in = dims[l - 1];
+    d.d_out = dims[l];
+}
+
+dhq_status_t check_config(const dhq_config_t *cfg)
+{
+    const int L = cfg->n_layers;
+    if (L < 2 || L > kMaxLayers) return DHQ_ERR_INVALID_ARG;
+    const int w = cfg->dims[1], d_L = cfg->dims[L];
+    if (cfg->dims[0] != 2 || w <= 0 || (w & (w - 1)) != 0 || w < 64 || w > 512 || d_L < 1 || d_L > 4) return DHQ_ERR_UNSUPPORTED;
+    for (int l = 1; l < L; ++l)
+        if (cfg->dims[l] != w) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits < 2 || cfg->a_bits > 8) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->rotation != DHQ_ROT_INPUT && cfg->rotation != DHQ_ROT_NONE && cfg->rotation != DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
+    if ((cfg->w_gran != DHQ_GRAN_TENSOR && cfg->w_gran != DHQ_GRAN_CHANNEL_OR_TOKEN) ||
+        (cfg->a_gran != DHQ_GRAN_TENSOR && cfg->a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN))
+        return DHQ_ERR_INVALID_ARG;
+    if (!(cfg->omega0 == cfg->omega0) || std::isinf(cfg->omega0)) return DHQ_ERR_INVALID_ARG;
+    return DHQ_OK;
+}
+
+// Serialized handle (dhq_export / dhq_import): this header, then every array of every layer in
+// the order of layer_arrays.
+struct BlobHeader {
+    char magic[8];            // "DHQB200\0"
+    uint32_t version, header_bytes;
+    int32_t n_layers, dims[kMaxLayers + 1];
+    int32_t w_bits, a_bits, w_gran, a_gran, rotation;
+    float omega0;
+    int32_t calibrated, calib_layers_done;
+    int32_t epi_mode[kMaxLayers];
+    float phase_bound[kMaxLayers];
+    uint64_t payload_bytes, payload_fnv1a;
+};
+constexpr uint32_t kBlobVersion = 1;
+const char kBlobMagic[8] = {'D', 'H', 'Q', 'B', '2', '0', '0', 0};
+
+uint64_t fnv1a(const uint8_t *p, size_t n)
+{
+    uint64_t hsh = 1469598103934665603ull;
+    for (size_t i = 0; i < n; ++i) hsh = (hsh ^ p[i]) * 1099511628211ull;
+    return hsh;
+}
+
 
 dhq_status_t ensure_scratch(dhq_handle_s *h, int64_t tokens)
 {
@@ -122,10 +206,10 @@ dhq_status_t layerwise_forward(dhq_handle_s *h, const float *coords, int64_t n, 
 
 // The forward pass of a calibrated handle: the fused kernel, or, for the two-sided transform, the
 // layer-by-layer kernels.
-dhq_status_t run_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st)
+dhq_status_t run_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, bool on_host, cudaStream_t st)
 {
     if (h->cfg.rotation == DHQ_ROT_BOTH) return layerwise_forward(h, coords, n, out, st);
-    return fused_forward(h, coords, n, out, st);
+    return fused_forward(h, coords, n, out, on_host, st);
 }
 
 } // namespace
@@ -176,16 +260,11 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     if (L < 2 || L > kMaxLayers) return DHQ_ERR_INVALID_ARG;
     for (int l = 0; l < L; ++l)
         if (!W[l] || !b[l]) return DHQ_ERR_INVALID_ARG;
+    {
+        dhq_status_t cs = check_config(cfg);
+        if (cs != DHQ_OK) return cs;
+    }
     const int w = cfg->dims[1], d_L = cfg->dims[L];
-    if (cfg->dims[0] != 2 || !is_pow2(w) || w < 64 || w > 512 || d_L < 1 || d_L > 4) return DHQ_ERR_UNSUPPORTED;
-    for (int l = 1; l < L; ++l)
-        if (cfg->dims[l] != w) return DHQ_ERR_UNSUPPORTED;
-    if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits < 2 || cfg->a_bits > 8) return DHQ_ERR_UNSUPPORTED;
-    if (cfg->rotation != DHQ_ROT_INPUT && cfg->rotation != DHQ_ROT_NONE && cfg->rotation != DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
-    if ((cfg->w_gran != DHQ_GRAN_TENSOR && cfg->w_gran != DHQ_GRAN_CHANNEL_OR_TOKEN) ||
-        (cfg->a_gran != DHQ_GRAN_TENSOR && cfg->a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN))
-        return DHQ_ERR_INVALID_ARG;
-    if (!(cfg->omega0 == cfg->omega0) || std::isinf(cfg->omega0)) return DHQ_ERR_INVALID_ARG;
 
     dhq_handle_s *h = new (std::nothrow) dhq_handle_s();
     if (!h) return DHQ_ERR_ALLOC;
@@ -205,28 +284,17 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             cudaMemsetAsync(d_bounds, 0, kMaxLayers * sizeof(float), st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
         for (int l = 1; l <= L && rc == DHQ_OK; ++l) {
             LayerDev &d = h->layer[l - 1];
-            d.K = (l == 1) ? 4 : w;
-            d.M = (l == L) ? 4 : w;
-            d.Mt = d.M < 16 ? 16 : d.M;
-            d.slab_k = fused_slab_k(d.K, d.Mt);
-            d.d_in = cfg->dims[l - 1];
-            d.d_out = cfg->dims[l];
+            set_layer_dims(d, l, L, w, cfg->dims);
             if (l == 1) d.epi_mode = per_token ? EPI_SINE_WIDE : EPI_SINE_FIXED; // coordinates are not bounded by the weights
             if (both) d.epi_mode = EPI_BOTH;
-            const size_t MK = (size_t)d.M * d.K;
-            bool ok = dev_alloc(&d.w_rot, MK) && dev_alloc(&d.row_absmax, d.M) && dev_alloc(&d.qw, MK) &&
-                      dev_alloc(&d.qw_k4m, MK / 4) && dev_alloc(&d.qw_umma, (size_t)d.Mt * (d.K < 16 ? 16 : d.K)) &&
-                      dev_alloc(&d.s_w, d.M) && dev_alloc(&d.inv_w, d.M) && dev_alloc(&d.bias, d.M) &&
-                      dev_alloc(&d.cA, d.M) && dev_alloc(&d.cA_lo, d.M) && dev_alloc(&d.cB, d.M) &&
-                      dev_alloc(&d.fxP, d.M) && dev_alloc(&d.fxQ, d.M) && dev_alloc(&d.fxB, d.M) &&
-                      dev_alloc(&d.act, 4);
-            if (!ok) { rc = DHQ_ERR_ALLOC; break; }
+            if (!alloc_layer(d)) { rc = DHQ_ERR_ALLOC; break; }
             if (cudaMemsetAsync(d.act, 0, 16, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
             PrepArgs a;
             memset(&a, 0, sizeof(a));
             a.W = W[l - 1]; a.b = b[l - 1];
             a.d_out = d.d_out; a.d_in = d.d_in; a.K = d.K; a.M = d.M; a.Mt = d.Mt;
             a.bits = cfg->w_bits;
+            a.a_bits = cfg->a_bits;
             a.per_channel = cfg->w_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
             a.sine = l < L; a.first = l == 1;
             a.permute_rows = (l > 1 && l < L) ? 1 : 0;
@@ -267,6 +335,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
 dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void *stream)
 {
     if (!h || !coords || n < 1) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
     return calibrate_impl(h, coords, n, (cudaStream_t)stream);
 }
@@ -274,6 +343,7 @@ dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void 
 dhq_status_t dhq_calibrate_layer(dhq_handle_t h, int layer, const float *coords, int64_t n, void *stream)
 {
     if (!h || layer < 1 || layer > h->L || n < 0 || (n > 0 && !coords)) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
     if (layer > h->calib_layers_done + 1) return DHQ_ERR_NOT_CALIBRATED; // layers before it are not frozen yet
     h->calibrated = false;
@@ -288,6 +358,7 @@ dhq_status_t dhq_calibrate_layer(dhq_handle_t h, int layer, const float *coords,
 dhq_status_t dhq_get_act_absmax(dhq_handle_t h, int layer, float *absmax, void *stream)
 {
     if (!h || layer < 1 || layer > h->L || !absmax) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     CK(cudaMemcpyAsync(absmax, h->layer[layer - 1].act, sizeof(float), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
@@ -297,6 +368,7 @@ dhq_status_t dhq_get_act_absmax(dhq_handle_t h, int layer, float *absmax, void *
 dhq_status_t dhq_set_act_absmax(dhq_handle_t h, int layer, float absmax, void *stream)
 {
     if (!h || layer < 1 || layer > h->L || !(absmax >= 0.0f) || std::isinf(absmax)) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
     if (layer > h->calib_layers_done + 1) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
@@ -312,6 +384,7 @@ dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int64_t n, f
                                const dhq_debug_bufs_t *bufs, void *stream)
 {
     if (!h || n < 0 || (n > 0 && !coords)) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
@@ -341,9 +414,63 @@ dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int64_t n, f
     return DHQ_OK;
 }
 
+dhq_status_t dhq_forward_fused_debug(dhq_handle_t h, const float *coords, int64_t n, float *out,
+                                     const dhq_debug_bufs_t *bufs, void *stream)
+{
+    if (!h || n < 0 || (n > 0 && (!coords || !out))) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
+    if (n == 0) return DHQ_OK;
+    if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
+    if (h->cfg.rotation == DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED; // runs layer by layer: dhq_forward_debug observes it
+    if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
+    cudaStream_t st = (cudaStream_t)stream;
+    DumpPtrs d;
+    memset(&d, 0, sizeof(d));
+    if (bufs) {
+        for (int l = 1; l <= h->L; ++l) {
+            if (bufs->codes && bufs->codes[l - 1]) d.codes[l - 1] = bufs->codes[l - 1];
+            if (bufs->s_x && bufs->s_x[l - 1]) d.s_x[l - 1] = bufs->s_x[l - 1];
+            if (bufs->acc && bufs->acc[l - 1]) d.acc[l - 1] = bufs->acc[l - 1];
+            if (bufs->Y && bufs->Y[l - 1]) d.Y[l - 1] = bufs->Y[l - 1];
+        }
+        if (bufs->X && bufs->X[0]) d.X[0] = bufs->X[0];
+        // inside the fused kernel the input of layer l+1 IS the output of layer l (one value, in
+        // registers): it is written once, to Y[l-1] if given, else straight to X[l]
+        for (int l = 1; l < h->L; ++l)
+            if (!d.Y[l - 1] && bufs->X && bufs->X[l]) d.Y[l - 1] = bufs->X[l];
+        if (((uintptr_t)d.X[0] & 15)) return DHQ_ERR_INVALID_ARG;
+        for (int l = 0; l < h->L; ++l)
+            if (((uintptr_t)d.codes[l] & 3) || ((uintptr_t)d.s_x[l] & 3) || ((uintptr_t)d.acc[l] & 3) || ((uintptr_t)d.Y[l] & 3))
+                return DHQ_ERR_INVALID_ARG;
+    }
+    dhq_status_t s = fused_forward_dump(h, coords, n, out, d, st);
+    if (s != DHQ_OK) return s;
+    if (bufs && bufs->X)
+        for (int l = 1; l < h->L; ++l)
+            if (bufs->X[l] && d.Y[l - 1] != bufs->X[l])
+                CK(cudaMemcpyAsync(bufs->X[l], d.Y[l - 1], (size_t)n * h->w * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_set_wait_limit(dhq_handle_t h, int64_t nanoseconds)
+{
+    if (!h || nanoseconds < 1000) return DHQ_ERR_INVALID_ARG;
+    h->wait_limit_ns = (unsigned long long)nanoseconds;
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_debug_stall_next_forward(dhq_handle_t h)
+{
+    if (!h) return DHQ_ERR_INVALID_ARG;
+    if (h->cfg.rotation == DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
+    h->stall_next_forward = true;
+    return DHQ_OK;
+}
+
 dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *out, void *stream)
 {
     if (!h || n < 0 || (n > 0 && (!coords || !out))) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
@@ -351,13 +478,14 @@ dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *
         dhq_status_t s = calibrate_impl(h, coords, n, st);
         if (s != DHQ_OK) return s;
     }
-    return run_forward(h, coords, n, out, st);
+    return run_forward(h, coords, n, out, false, st);
 }
 
 dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t n, float *out_host,
                               void *stream)
 {
     if (!h || n < 0 || (n > 0 && (!coords_host || !out_host))) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     cudaStream_t st = (cudaStream_t)stream;
     // Pinned (page-locked, device-mapped) host buffers need no staging: the fused kernel reads the
@@ -365,14 +493,15 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     // inside the kernel, tile by tile, beside the arithmetic.  (Calibration reads the coordinates
     // once per layer: it goes through the staged path below.)
     if (h->calibrated && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
+        // one query per buffer: for page-locked memory it also gives the device alias (asked on every
+        // call on purpose: an answer remembered per address could outlive the buffer it was given for)
         cudaPointerAttributes ai, ao;
-        void *di = nullptr, *dout = nullptr;
         const bool mapped = cudaPointerGetAttributes(&ai, coords_host) == cudaSuccess && ai.type == cudaMemoryTypeHost &&
                             cudaPointerGetAttributes(&ao, out_host) == cudaSuccess && ao.type == cudaMemoryTypeHost &&
-                            cudaHostGetDevicePointer(&di, const_cast<float *>(coords_host), 0) == cudaSuccess &&
-                            cudaHostGetDevicePointer(&dout, out_host, 0) == cudaSuccess && di && dout;
+                            ai.devicePointer && ao.devicePointer;
+        void *di = mapped ? ai.devicePointer : nullptr, *dout = mapped ? ao.devicePointer : nullptr;
         (void)cudaGetLastError(); // a failed query of pageable memory is not an error of this call
-        if (mapped) return run_forward(h, static_cast<const float *>(di), n, static_cast<float *>(dout), st);
+        if (mapped) return run_forward(h, static_cast<const float *>(di), n, static_cast<float *>(dout), true, st);
     }
     if (n > h->stage_tokens) {
         CK(cudaDeviceSynchronize());
@@ -422,7 +551,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
                            cudaMemcpyHostToDevice, h->copy_in));
         CK(cudaEventRecord(h->ev_in[i], h->copy_in));
         CK(cudaStreamWaitEvent(st, h->ev_in[i], 0));
-        dhq_status_t s = run_forward(h, h->stage_in + t0 * 2, cnt, h->stage_out + t0 * h->d_L, st);
+        dhq_status_t s = run_forward(h, h->stage_in + t0 * 2, cnt, h->stage_out + t0 * h->d_L, false, st);
         if (s != DHQ_OK) return s;
         CK(cudaEventRecord(h->ev_k[i], st));
         CK(cudaStreamWaitEvent(h->copy_out, h->ev_k[i], 0));
@@ -432,6 +561,121 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     }
     CK(cudaEventRecord(h->ev_done, h->copy_out));
     CK(cudaStreamWaitEvent(st, h->ev_done, 0));
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_export(dhq_handle_t h, void *host_buf, int64_t capacity, int64_t *needed)
+{
+    if (!h || !needed || capacity < 0) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
+    size_t payload = 0;
+    for (int l = 0; l < h->L; ++l) {
+        ArrayRef t[kLayerArrays];
+        layer_arrays(h->layer[l], t);
+        for (const ArrayRef &a : t) payload += a.bytes;
+    }
+    *needed = (int64_t)(sizeof(BlobHeader) + payload);
+    if (!host_buf) return DHQ_OK;                       // size query
+    if (capacity < *needed) return DHQ_ERR_TOO_LARGE;
+    CK(cudaDeviceSynchronize());
+    uint8_t *dst = static_cast<uint8_t *>(host_buf) + sizeof(BlobHeader);
+    for (int l = 0; l < h->L; ++l) {
+        ArrayRef t[kLayerArrays];
+        layer_arrays(h->layer[l], t);
+        for (const ArrayRef &a : t) {
+            CK(cudaMemcpy(dst, *a.ptr, a.bytes, cudaMemcpyDeviceToHost));
+            dst += a.bytes;
+        }
+    }
+    BlobHeader hd;
+    memset(&hd, 0, sizeof(hd));
+    memcpy(hd.magic, kBlobMagic, 8);
+    hd.version = kBlobVersion;
+    hd.header_bytes = (uint32_t)sizeof(BlobHeader);
+    hd.n_layers = h->L;
+    for (int i = 0; i <= h->L; ++i) hd.dims[i] = h->dims[i];
+    hd.w_bits = h->cfg.w_bits; hd.a_bits = h->cfg.a_bits;
+    hd.w_gran = (int)h->cfg.w_gran; hd.a_gran = (int)h->cfg.a_gran; hd.rotation = (int)h->cfg.rotation;
+    hd.omega0 = h->cfg.omega0;
+    hd.calibrated = h->calibrated ? 1 : 0;
+    hd.calib_layers_done = h->calib_layers_done;
+    for (int l = 0; l < h->L; ++l) {
+        hd.epi_mode[l] = h->layer[l].epi_mode;
+        hd.phase_bound[l] = h->layer[l].phase_bound;
+    }
+    hd.payload_bytes = payload;
+    hd.payload_fnv1a = fnv1a(static_cast<uint8_t *>(host_buf) + sizeof(BlobHeader), payload);
+    memcpy(host_buf, &hd, sizeof(hd));
+    return DHQ_OK;
+}
+
+dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_handle_t *out)
+{
+    if (!host_buf || !out || bytes < (int64_t)sizeof(BlobHeader)) return DHQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    BlobHeader hd;
+    memcpy(&hd, host_buf, sizeof(hd));
+    if (memcmp(hd.magic, kBlobMagic, 8) != 0 || hd.version != kBlobVersion || hd.header_bytes != sizeof(BlobHeader))
+        return DHQ_ERR_INVALID_ARG;
+    if (hd.n_layers < 2 || hd.n_layers > kMaxLayers) return DHQ_ERR_INVALID_ARG;
+    dhq_config_t cfg;
+    int dims[kMaxLayers + 1];
+    for (int i = 0; i <= hd.n_layers; ++i) dims[i] = hd.dims[i];
+    cfg.n_layers = hd.n_layers; cfg.dims = dims;
+    cfg.w_bits = hd.w_bits; cfg.a_bits = hd.a_bits; cfg.omega0 = hd.omega0;
+    cfg.w_gran = (dhq_gran_t)hd.w_gran; cfg.a_gran = (dhq_gran_t)hd.a_gran; cfg.rotation = (dhq_rot_t)hd.rotation;
+    dhq_status_t cs = check_config(&cfg);
+    if (cs != DHQ_OK) return cs == DHQ_ERR_UNSUPPORTED ? DHQ_ERR_UNSUPPORTED : DHQ_ERR_INVALID_ARG;
+    dhq_handle_s *h = new (std::nothrow) dhq_handle_s();
+    if (!h) return DHQ_ERR_ALLOC;
+    h->cfg = cfg;
+    for (int i = 0; i <= hd.n_layers; ++i) h->dims[i] = dims[i];
+    h->cfg.dims = h->dims;
+    h->L = hd.n_layers; h->w = dims[1]; h->d_L = dims[hd.n_layers];
+    size_t payload = 0;
+    for (int l = 1; l <= h->L; ++l) {
+        LayerDev &d = h->layer[l - 1];
+        set_layer_dims(d, l, h->L, h->w, dims);
+        ArrayRef t[kLayerArrays];
+        layer_arrays(d, t);
+        for (const ArrayRef &a : t) payload += a.bytes;
+        const int e = hd.epi_mode[l - 1];
+        if (e < EPI_LINEAR || e > EPI_BOTH) { delete h; return DHQ_ERR_INVALID_ARG; }
+        d.epi_mode = e;
+        d.phase_bound = hd.phase_bound[l - 1];
+    }
+    const uint8_t *src = static_cast<const uint8_t *>(host_buf) + sizeof(BlobHeader);
+    if (hd.payload_bytes != payload || bytes < (int64_t)(sizeof(BlobHeader) + payload) || fnv1a(src, payload) != hd.payload_fnv1a) {
+        delete h;
+        return DHQ_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    dhq_status_t rc = DHQ_OK;
+    do {
+        if (cudaGetDevice(&h->device) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+        if (!dev_alloc(&h->d_status, 4)) { rc = DHQ_ERR_ALLOC; break; }
+        if (cudaMemsetAsync(h->d_status, 0, 16, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+        for (int l = 0; l < h->L && rc == DHQ_OK; ++l) {
+            LayerDev &d = h->layer[l];
+            if (!alloc_layer(d)) { rc = DHQ_ERR_ALLOC; break; }
+            ArrayRef t[kLayerArrays];
+            layer_arrays(d, t);
+            for (const ArrayRef &a : t) {
+                if (cudaMemcpyAsync(*a.ptr, src, a.bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+                src += a.bytes;
+            }
+        }
+        if (rc != DHQ_OK) break;
+        if (cudaStreamSynchronize(st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; } // host_buf may go after the call
+        h->calibrated = hd.calibrated != 0;
+        h->calib_layers_done = hd.calib_layers_done;
+        if (cfg.rotation != DHQ_ROT_BOTH) rc = fused_create(h);
+    } while (0);
+    if (rc != DHQ_OK) {
+        dhq_destroy(h);
+        return rc;
+    }
+    *out = h;
     return DHQ_OK;
 }
 
@@ -446,6 +690,7 @@ dhq_status_t dhq_layer_dims(dhq_handle_t h, int layer, int *K, int *M)
 dhq_status_t dhq_get_layer(dhq_handle_t h, int layer, int8_t *codes, float *w_scales, float *act_absmax)
 {
     if (!h || layer < 1 || layer > h->L) return DHQ_ERR_INVALID_ARG;
+    if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     const LayerDev &d = h->layer[layer - 1];
     CK(cudaDeviceSynchronize());
     if (codes) CK(cudaMemcpy(codes, d.qw, (size_t)d.M * d.K, cudaMemcpyDeviceToHost));
@@ -460,7 +705,7 @@ dhq_status_t dhq_get_layer(dhq_handle_t h, int layer, int8_t *codes, float *w_sc
 
 dhq_status_t dhq_last_status(dhq_handle_t h)
 {
-    if (!h) return DHQ_ERR_INVALID_ARG;
+    if (!h || !on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     int v = 0;
     CK(cudaDeviceSynchronize());
     CK(cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));

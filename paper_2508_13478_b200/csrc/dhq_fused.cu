@@ -1,1033 +1,31 @@
-// Fused forward kernel: the whole quantized INR (Sections III-B and III-C of the paper) for
-// tiles of 128 coordinates without activations leaving the SM between layers.
-//
-// One persistent CTA per SM, 18 warps (19 at width 512):
-//   warps 0-15  epilogue warps.  Width <= 256: two "slots" of 8 warps, each slot has one tile of
-//               128 tokens in flight (its own A operand tile and 256 tensor-memory columns), so
-//               that one slot's CUDA-core work overlaps the other slot's MMA; the second slot
-//               starts half a layer period late.  Width 512: one slot of 16 warps; a layer's
-//               weights arrive as eight pieces (256 output columns x 128 k, the first half of the
-//               columns first), each feeding N = 256 MMAs; a thread has one chunk in each half
-//               and starts on the first while the second half's weights and MMAs are under way.
-//               A token (row) is a tensor-memory lane; R = 2 (or 4) threads from different warps
-//               share a row and split its columns.
-//   warp 16     issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in tensor memory).
-//   warp 18     (width 512) brings each tile's coordinates into shared memory with one bulk copy,
-//               a tile ahead.
-//   warp 17     brings the packed weight codes into shared memory with bulk async copies: once,
-//               if every hidden layer fits (they then stay resident), else through a ring that
-//               is refilled slab by slab from L2.
-//
-// Per layer and tile:
-//   pass 1  each thread takes its chunks of 64 columns: acc (TMEM, int32) -> dequantize, bias,
-//           sine (dhq_math.cuh) -> butterfly stages with stride < 64 in registers -> fp32 back to
-//           the same TMEM columns.          [mbarrier of the R warps that share the 32 rows]
-//   pass 2  each thread takes its groups: one value from every chunk at G consecutive positions
-//           -> the remaining butterfly stages (stride 64, 128, ...) -> quantize, pack, st.shared
-//           into the next layer's A operand tile -> mbarrier -> next MMA.
-//           Per-token scales: the rotated values go back to TMEM once more while the row's
-//           absmax is combined through shared memory, then pass 3 quantizes.
-// Layer 1 (K = 4) runs on the CUDA cores; the last layer is an MMA with N = 16 whose first d_L
-// columns are the result.
-//
-// Every wait on an mbarrier is bounded: when it runs out the kernel records an error in the
-// handle's status word, all roles leave their loops, tensor memory is released and the kernel
-// returns.
-#include <cstring>
-#include <new>
-#include "dhq_internal.cuh"
-#include "dhq_tmem.cuh"
+// Host side of the fused forward (kernels: dhq_fused.cuh, instantiated per width in
+// dhq_fused_w*.cu): the parameter block of a handle, the choice of the instantiation and the
+// launch; and the kernel's per-element loops run in isolation (micro-benchmark).
+#include "dhq_fused.cuh"
 
 namespace dhq {
 
-constexpr int kTile = 128;
-constexpr int kEpiWarps = 16;
-constexpr int kMmaWarp = 16, kLoadWarp = 17, kXyWarp = 18;
-constexpr int kThreads = 18 * 32; // width 512 runs one more warp (Cfg::THREADS)
-constexpr int kMaxStages = 32;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull; // 2 s per wait
-constexpr uint32_t kCopyBytes = 8192; // bytes per bulk copy of a weight slab
-constexpr int kMinSmem = 120 * 1024; // more than half an SM's shared memory: one CTA per SM
-
-// Work split for a hidden width W.
-template <int W> struct Cfg {
-    static constexpr int SLOTS = (W == 512) ? 1 : 2;
-    static constexpr int R = kEpiWarps / (4 * SLOTS);          // threads per row: 2 or 4
-    static constexpr int CH = (W == 64) ? 32 : 64;             // columns per register chunk (= fused_chunk(W))
-    static constexpr int NCH = W / CH;                         // chunks per row
-    static constexpr int CPT = NCH / R;                        // chunks per thread
-    static constexpr int G = (64 / NCH < CH / R) ? 64 / NCH : CH / R; // positions per pass-2 group
-    static constexpr int GPT = CH / (G * R);                   // groups per thread
-    static constexpr int KSLABS = (W == 512) ? 4 : 1;          // weight slabs per layer along K
-    static constexpr int SLABK = W / KSLABS;                   // k per slab (= fused_slab_k)
-    static constexpr int NHALF = (W == 512) ? 2 : 1;           // MMAs along N (an MMA has N <= 256)
-    static constexpr int NW = W / NHALF;                       // N of one MMA
-    static constexpr int PIECES = KSLABS * NHALF;              // weight pieces per layer (ring units)
-    static constexpr int PIECE_BYTES = SLABK * NW;             // 64 KB (width 256), 32 KB (width 512)
-    static constexpr int SLOT_THREADS = R * kTile;
-    // Width 512: the coordinates of a whole tile arrive by one bulk copy issued by a 19th warp (measured:
-    // 2.6 % faster, 6.7 % from mapped host memory; narrower networks lost 4-7 % to the extra barrier).
-    static constexpr bool BULK_XY = (W == 512);
-    static constexpr int THREADS = kThreads + (BULK_XY ? 32 : 0);
-    static constexpr int TMEM_COLS_PER_SLOT = 512 / SLOTS;
-};
-
-// Tile of slot `slot` of this CTA in its round r.  Normally the slots of a CTA take adjacent tiles.
-// A launch with fewer tiles than CTAs x slots is spread instead: the tiles go round-robin first
-// over the CTAs, then over the slots, so that it covers as many SMs as it has tiles (one busy slot
-// each) before any SM gets a second tile.
-template <bool SPREAD> __device__ __forceinline__ long long tile_index(long long r, int slot, int slots)
-{
-    return SPREAD ? (r * slots + slot) * (long long)gridDim.x + blockIdx.x
-                  : ((long long)blockIdx.x + r * gridDim.x) * slots + slot;
-}
-
-// Chunk cc of the thread with index `sub` among the R threads of a row.  Width 512 gives every
-// thread one chunk in each half of the columns (the halves' accumulators complete one after the
-// other); otherwise a thread's chunks are adjacent.
-template <int W> __device__ __forceinline__ int chunk_of(int sub, int cc)
-{
-    return (W == 512) ? cc * Cfg<W>::R + sub : sub * Cfg<W>::CPT + cc;
-}
-
-struct FusedLayer {
-    const uint8_t *qw_umma;
-    const uint32_t *qw_k4m;
-    const float *cA, *cA_lo, *cB;
-    const uint32_t *fxP, *fxQ, *fxB;
-    const float *act;
-    int epi_mode;
-    int c_off; // word offset of this layer's constants in the shared-memory constant area
-};
-
-struct FusedParams {
-    const float *coords;
-    float *out;
-    long long n, n_tiles;
-    int L, W, d_L, per_token;
-    float qmaxf;
-    int n_stages, resident;
-    int bulk_xy;         // coords 16-byte aligned: whole tiles may arrive by bulk copy (width 512)
-    int bulk_out;        // out 16-byte aligned: whole tiles may leave by bulk store (host-buffer variant)
-    int const_words;
-    int *status;
-    FusedLayer layer[kMaxLayers];
-};
-
-struct FusedState {
-    FusedParams p;
-    size_t smem_bytes;
-    int sm_count;
-};
-
-// Shared-memory map (byte offsets from a 1024-byte aligned base).
-struct SmemMap {
-    uint32_t a_tile[2];
-    uint32_t ring, last_w, consts, amax;
-    uint32_t xy;         // [2 slots][4 threads of a row][128 rows] float2: coordinates fetched ahead
-    uint32_t out_tile;   // [2 slots][128 rows][4] fp32: a tile's results before their bulk store (width <= 256)
-    uint32_t acc_full;   // [2 slots][4 pieces]
-    uint32_t acc_last;   // [2]
-    uint32_t codes_full; // [2]
-    uint32_t slot_sync;  // [2 slots][4 lane quadrants]
-    uint32_t last_full, drain;
-    uint32_t xy_full, xy_empty; // [2 slots] each: coordinates by bulk copy
-    uint32_t out_sync;   // [2 slots]: the 128 threads that fill a slot's result buffer (host-buffer variant)
-    uint32_t w_full, w_empty; // [kMaxStages] each
-    uint32_t tmem_holder, abort_flag;
-    uint32_t total;
-};
-
-__host__ __device__ inline SmemMap smem_map(int W, int n_stages, int const_words)
-{
-    const int slots = (W == 512) ? 1 : 2;
-    const uint32_t piece_bytes = (W == 512) ? 128u * 256u : (uint32_t)W * W;
-    SmemMap m;
-    uint32_t off = 0;
-    m.a_tile[0] = off; off += kTile * W;
-    m.a_tile[1] = off; if (slots == 2) off += kTile * W;
-    m.ring = off; off += (uint32_t)n_stages * piece_bytes;
-    m.last_w = off; off += 16 * W;
-    m.consts = off; off += (uint32_t)const_words * 4;
-    m.amax = off; off += 2 * 4 * kTile * 4;
-    m.xy = off; off += (W != 512) ? 2 * 4 * kTile * 8 : kTile * 8; // per-thread entries, or one tile for the bulk copy
-    m.out_tile = off; if (W != 512) off += 2 * kTile * 4 * 4; // placed here, among the 16-byte aligned areas: a bulk store reads it
-    m.acc_full = off; off += 8 * 8;
-    m.acc_last = off; off += 8 * 2;
-    m.codes_full = off; off += 8 * 2;
-    m.slot_sync = off; off += 8 * 8;
-    m.last_full = off; off += 8;
-    m.xy_full = off; if (W == 512) off += 16;
-    m.xy_empty = off; if (W == 512) off += 16;
-    m.out_sync = off; if (W != 512) off += 16;
-    m.drain = off; off += 8;
-    m.w_full = off; off += 8 * kMaxStages;
-    m.w_empty = off; off += 8 * kMaxStages;
-    m.tmem_holder = off; off += 8;
-    m.abort_flag = off; off += 8;
-    m.total = off;
-    return m;
-}
-
-// Bounded wait.  Returns false when the wait ran out or another role already gave up.  Between
-// tries the thread either sleeps (SLEEP_NS), so that a waiting warp leaves the issue slots to the
-// working ones, or, with HINT_NS > 0, stays suspended inside the try itself for up to that long;
-// the time limit and the abort flag are looked at every 64 tries.  Which form is faster was
-// measured per role: the single-thread MMA and copy roles and the epilogue warps of the
-// per-token kernels (two more barriers per layer) do better suspended, the epilogue warps of the
-// per-tensor kernels sleeping.
-constexpr int kHintNs = 2000;
-template <int SLEEP_NS, int HINT_NS = 0>
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
-{
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    unsigned long long t0 = 0;
-    for (uint32_t tries = 1;; ++tries) {
-        if (HINT_NS > 0) {
-            if (ptx::mbar_try_wait_hint(bar, parity, HINT_NS)) return true;
-        } else {
-            __nanosleep(SLEEP_NS);
-            if (ptx::mbar_try_wait(bar, parity)) return true;
-        }
-        if ((tries & 63) == 0) {
-            if (*abort_flag) return false;
-            const unsigned long long now = ptx::globaltimer();
-            if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicExch(status, 1);
-                return false;
-            }
-        }
-    }
-}
-// The same for a whole warp: every lane takes the same decision.
-template <bool SUSPEND>
-__device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
-{
-    return __all_sync(0xffffffffu, wait_bar<32, SUSPEND ? kHintNs : 0>(bar, parity, abort_flag, status));
-}
-
-// Two fp32 values in one 64-bit register pair, and the packed sm_100 arithmetic on them: one
-// instruction, two IEEE round-to-nearest results (the same bits as two scalar operations).
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi)
-{
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ f32x2 pack2u(uint32_t lo, uint32_t hi)
-{
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ void unpack2u(f32x2 v, uint32_t &lo, uint32_t &hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
-// One butterfly on two independent pairs at once: (a, b) -> (a + b, a - b).
-__device__ __forceinline__ void bfly2(f32x2 &a, f32x2 &b)
-{
-    const f32x2 x = a, y = b;
-    a = add2(x, y);
-    b = sub2(x, y);
-}
-
-// Round-half-even of two values to integer codes held in the low bytes: multiply by inv,
-// (clamp,) add 1.5 * 2^23 - the sum rounds to the integer grid, ties to even, and its low
-// mantissa bits are the two's complement code.  Same integers as
-// __float2int_rn(clamp(v * inv, -qmax, qmax)).  With a per-token scale |v * inv| <= qmax
-// (1 + 2^-23) already, so the clamp is skipped.  The clamp is sign(t) * min(|t|, qmax).
-template <bool CLAMP> __device__ __forceinline__ void code_bits2(f32x2 v, f32x2 inv2, float qmaxf, uint32_t &b0, uint32_t &b1)
-{
-    f32x2 t = mul2(v, inv2);
-    float lo, hi;
-    unpack2(t, lo, hi);
-    if (CLAMP) {
-        asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(lo) : "f"(qmaxf));
-        asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(hi) : "f"(qmaxf));
-        unpack2u(add2(pack2(lo, hi), pack2(12582912.0f, 12582912.0f)), b0, b1);
-    } else {
-        // Scalar adds here: a packed multiply directly followed by a packed add was observed to be
-        // merged into one fused multiply-add by the assembler, which rounds v * inv only once and
-        // turns exact ties (x.5) the wrong way.  The product must be rounded to fp32 first.
-        b0 = __float_as_uint(__fadd_rn(lo, 12582912.0f));
-        b1 = __float_as_uint(__fadd_rn(hi, 12582912.0f));
-    }
-}
-template <bool CLAMP> __device__ __forceinline__ uint32_t code_bits(float v, float inv, float qmaxf)
-{
-    float t = __fmul_rn(v, inv);
-    if (CLAMP) asm("min.xorsign.abs.f32 %0, %0, %1;" : "+f"(t) : "f"(qmaxf));
-    return __float_as_uint(__fadd_rn(t, 12582912.0f));
-}
-__device__ __forceinline__ uint32_t pack4(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3)
-{
-    uint32_t lo = __byte_perm(b0, b1, 0x0040);
-    uint32_t hi = __byte_perm(b2, b3, 0x0040);
-    return __byte_perm(lo, hi, 0x5410);
-}
-// Store N (4, 8 or 16) consecutive-k codes of this thread's token, k0 a multiple of N, into the A
-// operand tile: byte offset (k/16) * 2048 + row * 16 + k % 16.  w holds N/4 packed words.
-template <int N> __device__ __forceinline__ void store_code_words(uint32_t a_tile, int row, int k0, const uint32_t *w)
-{
-    const uint32_t addr = a_tile + (k0 >> 4) * 2048 + row * 16 + (k0 & 15);
-    if constexpr (N == 16)
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-    else if constexpr (N == 8)
-        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(w[0]), "r"(w[1]) : "memory");
-    else
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(w[0]) : "memory");
-}
-// Quantize G consecutive tensor-memory columns of chunk `ch` starting at column position p0 (even
-// positions hold features p0/2 + k, odd positions features CH/2 + p0/2 + k) and store the codes.
-template <int G, int CH, bool CLAMP>
-__device__ __forceinline__ void quantize_store(uint32_t a_tile, int row, int ch, int p0, const uint32_t *u, float inv, float qmaxf)
-{
-    const f32x2 inv2 = pack2(inv, inv);
-    uint32_t even[G / 2], odd[G / 2];
-#pragma unroll
-    for (int k = 0; k < G / 2; ++k) code_bits2<CLAMP>(pack2u(u[2 * k], u[2 * k + 1]), inv2, qmaxf, even[k], odd[k]);
-    uint32_t we[G / 8], wo[G / 8];
-#pragma unroll
-    for (int j = 0; j < G / 8; ++j) {
-        we[j] = pack4(even[4 * j], even[4 * j + 1], even[4 * j + 2], even[4 * j + 3]);
-        wo[j] = pack4(odd[4 * j], odd[4 * j + 1], odd[4 * j + 2], odd[4 * j + 3]);
-    }
-    store_code_words<G / 2>(a_tile, row, ch * CH + p0 / 2, we);
-    store_code_words<G / 2>(a_tile, row, ch * CH + CH / 2 + p0 / 2, wo);
-}
-
-template <int N> __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[N])
-{
-    if constexpr (N == 8) ptx::tmem_ld8(taddr, v);
-    else if constexpr (N == 16) ptx::tmem_ld16(taddr, v);
-    else if constexpr (N == 32) ptx::tmem_ld32(taddr, v);
-    else ptx::tmem_ld64(taddr, v);
-}
-template <int N> __device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&v)[N])
-{
-    if constexpr (N == 8) ptx::tmem_st8(taddr, v);
-    else if constexpr (N == 16) ptx::tmem_st16(taddr, v);
-    else if constexpr (N == 32) ptx::tmem_st32(taddr, v);
-    else ptx::tmem_st64(taddr, v);
-}
-
-__device__ __forceinline__ float4 lds128(uint32_t addr)
-{
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-    return v;
-}
-
-// Pass 1 of one chunk, in place: v holds CH int32 accumulators (or nothing, for layer 1) on entry
-// and, on exit, the fp32 activations after the butterfly stages with strides 1 .. CH/2.
-// Tensor-memory column 2i of the chunk is feature i, column 2i+1 feature i + CH/2, so the
-// register pair (v[2i], v[2i+1]) goes through the stages with strides 1 .. CH/4 as one packed
-// value; the stride-CH/2 stage is the butterfly between its two halves.
-// `sine8(j, out)` produces the four pairs 4j .. 4j+3.  The work is ordered as a software pipeline -
-// the sines of group j+1 are issued before the stride-1/2 butterflies of group j, the stride-4/8
-// butterflies follow every fourth group - so that the special-function unit (one sine per 8 issue
-// cycles and scheduler) is fed evenly instead of in one burst per chunk.  Each element still goes
-// through the stages in the order 1, 2, 4, ...: the sums are unchanged.
-template <int CH, bool ROT, class Sine8> __device__ __forceinline__ void chunk_pipeline(uint32_t (&v)[CH], Sine8 sine8)
-{
-    constexpr int NP = CH / 2;
-    f32x2 P[NP];
-    if constexpr (!ROT) { // no rotation (plain uniform quantization): activations only
-#pragma unroll
-        for (int j = 0; j < NP / 4; ++j) sine8(j, &P[4 * j]);
-#pragma unroll
-        for (int i = 0; i < NP; ++i) unpack2u(P[i], v[2 * i], v[2 * i + 1]);
-        return;
-    }
-    sine8(0, &P[0]);
-#pragma unroll
-    for (int j = 0; j < NP / 4; ++j) {
-        if (j + 1 < NP / 4) sine8(j + 1, &P[4 * (j + 1)]);
-        bfly2(P[4 * j], P[4 * j + 1]);
-        bfly2(P[4 * j + 2], P[4 * j + 3]);
-        bfly2(P[4 * j], P[4 * j + 2]);
-        bfly2(P[4 * j + 1], P[4 * j + 3]);
-        if ((j & 3) == 3) {
-            const int base = 4 * (j - 3);
-#pragma unroll
-            for (int h = 4; h <= 8; h <<= 1) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if ((i & h) == 0) bfly2(P[base + i], P[base + i + h]);
-            }
-        }
-    }
-#pragma unroll
-    for (int h = 16; h < NP; h <<= 1) {
-#pragma unroll
-        for (int i = 0; i < NP; ++i)
-            if ((i & h) == 0) bfly2(P[i], P[i + h]);
-    }
-#pragma unroll
-    for (int i = 0; i < NP; ++i) {
-        float a, b;
-        unpack2(P[i], a, b);
-        v[2 * i] = __float_as_uint(__fadd_rn(a, b));
-        v[2 * i + 1] = __float_as_uint(__fsub_rn(a, b));
-    }
-}
-
-// Hidden layer: dequantize + bias + sine of the CH columns starting at column m0.  Constants come
-// from shared memory in column order: area A = cA, B = cB, C = cA_lo, each W words.
-template <int W, int CH, bool PER_TOKEN, bool ROT, int MODE>
-__device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH])
-{
-    chunk_pipeline<CH, ROT>(v, [&](int j, f32x2 *out) {
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int i = 8 * j + 4 * q; // four columns = two pairs
-            const float4 a = lds128(cbase + (m0 + i) * 4);
-            const float4 b = lds128(cbase + (W + m0 + i) * 4);
-            if (MODE == EPI_SINE_FAST && !PER_TOKEN) {
-                // x = fma(acc, cA, cB) for two columns at once, then the sine of each
-                float x0, x1, x2, x3;
-                unpack2(fma2(pack2((float)(int)v[i], (float)(int)v[i + 1]), pack2(a.x, a.y), pack2(b.x, b.y)), x0, x1);
-                unpack2(fma2(pack2((float)(int)v[i + 2], (float)(int)v[i + 3]), pack2(a.z, a.w), pack2(b.z, b.w)), x2, x3);
-                out[2 * q] = pack2(sin_approx(x0), sin_approx(x1));
-                out[2 * q + 1] = pack2(sin_approx(x2), sin_approx(x3));
-            } else {
-                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (MODE == EPI_SINE_WIDE) lo = lds128(cbase + (2 * W + m0 + i) * 4);
-                const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w}, lv[4] = {lo.x, lo.y, lo.z, lo.w};
-                float y[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float c_hi = av[e], c_lo = lv[e];
-                    if (PER_TOKEN) token_const(av[e], lv[e], s_x, c_hi, c_lo);
-                    y[e] = epilogue(MODE, (float)(int)v[i + e], c_hi, c_lo, bv[e]);
-                }
-                out[2 * q] = pack2(y[0], y[1]);
-                out[2 * q + 1] = pack2(y[2], y[3]);
-            }
-        }
-    });
-}
-
-// Layer 1 for the CH columns starting at column m0.  Fixed-point mode: areas A = P, B = B, C = Q.
-// Float mode (per-token scales): A = cA, B = cB, C = cA_lo, D = the weight codes, one word per
-// column, and acc = dp4a(codes of the token, codes of the column's feature).
-template <int W, int CH, bool PER_TOKEN, bool ROT>
-__device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int qd, uint32_t qx, float s_x, uint32_t (&v)[CH])
-{
-    chunk_pipeline<CH, ROT>(v, [&](int j, f32x2 *out) {
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int i = 8 * j + 4 * q;
-            const float4 A = lds128(cbase + (m0 + i) * 4);
-            const float4 B = lds128(cbase + (W + m0 + i) * 4);
-            const float4 Cc = lds128(cbase + (2 * W + m0 + i) * 4);
-            const float Av[4] = {A.x, A.y, A.z, A.w}, Bv[4] = {B.x, B.y, B.z, B.w}, Cv[4] = {Cc.x, Cc.y, Cc.z, Cc.w};
-            float y[4];
-            if constexpr (!PER_TOKEN) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    y[e] = sine_fixed(qs, qd, __float_as_uint(Av[e]), __float_as_uint(Cv[e]), __float_as_uint(Bv[e]));
-            } else {
-                const float4 wq = lds128(cbase + (3 * W + m0 + i) * 4);
-                const float wv[4] = {wq.x, wq.y, wq.z, wq.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float c_hi, c_lo;
-                    token_const(Av[e], Cv[e], s_x, c_hi, c_lo);
-                    const int acc = __dp4a((int)qx, (int)__float_as_uint(wv[e]), 0);
-                    y[e] = epilogue(EPI_SINE_WIDE, (float)acc, c_hi, c_lo, Bv[e]);
-                }
-            }
-            out[2 * q] = pack2(y[0], y[1]);
-            out[2 * q + 1] = pack2(y[2], y[3]);
-        }
-    });
-}
-
-// Everything a slot's threads need to finish a layer once their chunks are back in tensor memory.
-struct SlotCtx {
-    uint32_t taddr;      // TMEM address of this thread's lane, column 0 of the slot
-    uint32_t a_tile;     // shared-memory address of the slot's A operand tile
-    uint32_t bar_sync;   // mbarrier of the R warps that share this thread's 32 rows
-    uint32_t bar_codes;  // "codes ready" mbarrier
-    uint32_t amax_addr;  // shared memory: [R][128] floats for this slot
-    uint32_t sync_parity;
-    int row, sub;
-    float qmaxf;
-    volatile int *abort_flag;
-    int *status;
-};
-
-template <bool SUSPEND> __device__ __forceinline__ bool slot_barrier(SlotCtx &c)
-{
-    ptx::mbar_arrive(c.bar_sync);
-    bool ok = wait_bar_warp<SUSPEND>(c.bar_sync, c.sync_parity, c.abort_flag, c.status);
-    c.sync_parity ^= 1;
-    return ok;
-}
-
-// Passes 2 and 3: remaining butterfly stages across chunks, quantizer, store of the codes, and the
-// arrival on the "codes ready" barrier.  Returns false if a wait ran out.  s_out receives the
-// token's activation scale of the next layer.
-template <int W, bool PER_TOKEN, bool ROT>
-__device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float static_inv, float &s_out)
-{
-    using C = Cfg<W>;
-    constexpr int NCH = C::NCH, G = C::G, CH = C::CH;
-    ptx::tmem_wait_st();
-    ptx::tc_fence_before();
-    if (!slot_barrier<PER_TOKEN>(c)) return false;
-    ptx::tc_fence_after();
-    float amax = 0.f;
-#pragma unroll 1
-    for (int gg = 0; gg < C::GPT; ++gg) {
-        const int g = c.sub * C::GPT + gg;
-        uint32_t u[NCH][G];
-#pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
-        ptx::tmem_wait_ld();
-        // strides CH, 2 CH, ...: the chunk index is the butterfly index; two columns per instruction
-#pragma unroll
-        for (int h = 1; h < (ROT ? NCH : 1); h <<= 1) {
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-                if ((ch & h) == 0) {
-#pragma unroll
-                    for (int i = 0; i < G; i += 2) {
-                        f32x2 a = pack2u(u[ch][i], u[ch][i + 1]), b = pack2u(u[ch + h][i], u[ch + h][i + 1]);
-                        bfly2(a, b);
-                        unpack2u(a, u[ch][i], u[ch][i + 1]);
-                        unpack2u(b, u[ch + h][i], u[ch + h][i + 1]);
-                    }
-                }
-            }
-        }
-        if (PER_TOKEN) {
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-#pragma unroll
-                for (int i = 0; i < G; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(u[ch][i])));
-                tmem_st<G>(c.taddr + ch * CH + g * G, u[ch]);
-            }
-        } else {
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) quantize_store<G, CH, true>(c.a_tile, c.row, ch, g * G, u[ch], static_inv, c.qmaxf);
-        }
-    }
-    if (!PER_TOKEN) {
-        s_out = static_s;
-    } else {
-        // combine the row's absmax over the R threads that share it
-        asm volatile("st.shared.f32 [%0], %1;" ::"r"(c.amax_addr + (c.sub * kTile + c.row) * 4), "f"(amax) : "memory");
-        ptx::tmem_wait_st();
-        ptx::tc_fence_before();
-        if (!slot_barrier<PER_TOKEN>(c)) return false;
-        ptx::tc_fence_after();
-#pragma unroll
-        for (int r = 0; r < C::R; ++r) {
-            float o;
-            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(o) : "r"(c.amax_addr + (r * kTile + c.row) * 4));
-            amax = fmaxf(amax, o);
-        }
-        float s, inv;
-        scales_of(amax, c.qmaxf, s, inv);
-        s_out = s;
-#pragma unroll 1
-        for (int gg = 0; gg < C::GPT; ++gg) {
-            const int g = c.sub * C::GPT + gg;
-            uint32_t u[NCH][G];
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
-            ptx::tmem_wait_ld();
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) quantize_store<G, CH, false>(c.a_tile, c.row, ch, g * G, u[ch], inv, c.qmaxf);
-        }
-    }
-    ptx::fence_proxy_async();
-    ptx::tc_fence_before();
-    ptx::mbar_arrive(c.bar_codes);
-    return true;
-}
-
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD>
-__device__ void epilogue_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
-                              uint32_t tmem_base, volatile int *abort_flag)
-{
-    using C = Cfg<W>;
-    constexpr int CH = C::CH;
-    const int slot = warp / (4 * C::R);
-    const int quad = warp & 3;
-    const int sub = (warp % (4 * C::R)) >> 2;
-    SlotCtx c;
-    c.row = quad * 32 + lane;
-    c.sub = sub;
-    c.taddr = tmem_base + (uint32_t)(slot * C::TMEM_COLS_PER_SLOT) + ((uint32_t)(quad * 32) << 16);
-    c.a_tile = smem_base + sm.a_tile[slot];
-    c.bar_sync = smem_base + sm.slot_sync + 8 * (slot * 4 + quad);
-    c.bar_codes = smem_base + sm.codes_full + 8 * slot;
-    c.amax_addr = smem_base + sm.amax + slot * (4 * kTile * 4);
-    c.sync_parity = 0;
-    c.qmaxf = p.qmaxf;
-    c.abort_flag = abort_flag;
-    c.status = p.status;
-    const uint32_t bar_acc = smem_base + sm.acc_full + 8 * (slot * 4);
-    const uint32_t bar_last = smem_base + sm.acc_last + 8 * slot;
-    const uint32_t consts = smem_base + sm.consts;
-    const uint32_t xy_addr = smem_base + sm.xy + (uint32_t)(((slot * 4 + sub) * kTile + c.row) * 8);
-    uint32_t acc_parity = 0, last_parity = 0;
-    [[maybe_unused]] uint32_t xy_k = 0; // tiles taken from the bulk-copy buffer so far
-    [[maybe_unused]] uint32_t out_parity = 0;
-    const FusedLayer &l1 = p.layer[0];
-    const float qmaxf = p.qmaxf;
-
-    if (C::SLOTS == 2 && slot == 1 && tile_index<SPREAD>(0, 1, 2) < p.n_tiles && p.resident) {
-        // Start the second slot about half a layer period after the first, so that one slot's
-        // sine-heavy pass 1 and MMA wait fall on the other slot's pass 2 instead of both slots
-        // asking for the same pipe at the same time.  The offset then keeps itself.  Not when the
-        // weights are streamed: there both slots should consume a slab while it is in the ring.
-        const unsigned long long t0 = ptx::globaltimer(), delay = (3500ull * W * W) / (256 * 256);
-        while (ptx::globaltimer() - t0 < delay) __nanosleep(64);
-    }
-    for (long long r = 0;; ++r) {
-        const long long tile = tile_index<SPREAD>(r, slot, C::SLOTS);
-        if (tile >= p.n_tiles) break;
-        const long long tok = tile * kTile + c.row;
-        const bool valid = tok < p.n;
-
-        // ---------------- layer 1 on the CUDA cores: x~ = H_4 [x, y, 0, 0]
-        float x = 0.f, y = 0.f;
-        if constexpr (C::BULK_XY) {
-            if (p.bulk_xy && (tile + 1) * kTile <= p.n) {
-                // the whole tile was brought to shared memory by one bulk copy, a tile ahead
-                if (!wait_bar_warp<PER_TOKEN>(smem_base + sm.xy_full + 8 * slot, xy_k & 1u, abort_flag, p.status)) return;
-                ++xy_k;
-                asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x), "=f"(y) : "r"(smem_base + sm.xy + (uint32_t)((slot * kTile + c.row) * 8)));
-                ptx::mbar_arrive(smem_base + sm.xy_empty + 8 * slot);
-            } else if (valid) { // ragged last tile, or coordinates not 16-byte aligned
-                float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
-                x = xy.x; y = xy.y;
-            }
-        } else
-        if (!AHEAD || r == 0) {
-            if (valid) {
-                float2 xy = __ldg(reinterpret_cast<const float2 *>(p.coords) + tok);
-                x = xy.x; y = xy.y;
-            }
-        } else {
-            // copied into shared memory by this thread while the previous tile was in its hidden layers
-            asm volatile("cp.async.wait_all;" ::: "memory");
-            if (valid) asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x), "=f"(y) : "r"(xy_addr));
-        }
-        float e0 = x, e1 = y, e2 = 0.f, e3 = 0.f;
-        if (ROT) {
-            float r0 = __fadd_rn(x, y), r1 = __fsub_rn(x, y), r2 = __fadd_rn(0.f, 0.f), r3 = __fsub_rn(0.f, 0.f);
-            e0 = __fadd_rn(r0, r2); e2 = __fsub_rn(r0, r2); e1 = __fadd_rn(r1, r3); e3 = __fsub_rn(r1, r3);
-        }
-        float s_x, inv_x;
-        if (PER_TOKEN) {
-            float a = fmaxf(fmaxf(fabsf(e0), fabsf(e1)), fmaxf(fabsf(e2), fabsf(e3)));
-            scales_of(a, qmaxf, s_x, inv_x);
-        } else {
-            s_x = __ldg(l1.act + 1);
-            inv_x = __ldg(l1.act + 2);
-        }
-        const uint32_t b0 = code_bits<true>(e0, inv_x, qmaxf), b1 = code_bits<true>(e1, inv_x, qmaxf);
-        const uint32_t qx = pack4(b0, b1, code_bits<true>(e2, inv_x, qmaxf), code_bits<true>(e3, inv_x, qmaxf));
-        const int qs = (int)b0 - 0x4B400000, qd = (int)b1 - 0x4B400000;
-        float next_s = 1.f, next_inv = 0.f;
-        if (!PER_TOKEN) {
-            next_s = __ldg(p.layer[1].act + 1);
-            next_inv = __ldg(p.layer[1].act + 2);
-        }
-#pragma unroll
-        for (int cc = 0; cc < C::CPT; ++cc) {
-            const int ch = chunk_of<W>(sub, cc);
-            uint32_t v[CH];
-            layer1_chunk<W, CH, PER_TOKEN, ROT>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v);
-            tmem_st<CH>(c.taddr + ch * CH, v);
-        }
-        if (!finish_layer<W, PER_TOKEN, ROT>(c, next_s, next_inv, s_x)) return;
-        if constexpr (AHEAD) {
-            // The next tile's coordinates start their way into shared memory now.  An asynchronous
-            // copy holds neither a register nor one of the warp's dependency barriers while it is in
-            // flight (a plain load issued this early slowed the layers down: they wait on the barrier
-            // it occupies).  Not earlier than this: at the start of a launch every tile's first fetch
-            // is under way.  Only for coordinates in device memory: from mapped host memory the
-            // 8-byte asynchronous copies were slower than the plain load at the tile's start.
-            const long long tok_next = tile_index<SPREAD>(r + 1, slot, C::SLOTS) * kTile + c.row;
-            if (tok_next < p.n)
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(xy_addr), "l"(reinterpret_cast<const float2 *>(p.coords) + tok_next) : "memory");
-        }
-
-        // ---------------- layers 2 .. L on the tensor core
-        for (int l = 2; l < p.L; ++l) {
-            const FusedLayer &ly = p.layer[l - 1];
-            if (!wait_bar_warp<PER_TOKEN>(bar_acc, acc_parity, abort_flag, p.status)) return;
-            if constexpr (C::NHALF == 1) acc_parity ^= 1;
-            ptx::tc_fence_after();
-            if (!PER_TOKEN) {
-                next_s = __ldg(p.layer[l].act + 1);
-                next_inv = __ldg(p.layer[l].act + 2);
-            }
-            const uint32_t cbase = consts + ly.c_off * 4;
-            const bool fast = ly.epi_mode == EPI_SINE_FAST;
-#pragma unroll
-            for (int cc = 0; cc < C::CPT; ++cc) {
-                const int ch = chunk_of<W>(sub, cc);
-                if constexpr (C::NHALF == 2) {
-                    // width 512: the thread's second chunk lies in the second half of the output columns,
-                    // whose MMAs run while the first chunk is worked on
-                    if (cc == 1) {
-                        if (!wait_bar_warp<PER_TOKEN>(bar_acc + 8, acc_parity, abort_flag, p.status)) return;
-                        acc_parity ^= 1;
-                        ptx::tc_fence_after();
-                    }
-                }
-                uint32_t v[CH];
-                tmem_ld<CH>(c.taddr + ch * CH, v);
-                ptx::tmem_wait_ld();
-                if (fast) hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_FAST>(cbase, ch * CH, s_x, v);
-                else hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_WIDE>(cbase, ch * CH, s_x, v);
-                tmem_st<CH>(c.taddr + ch * CH, v);
-            }
-            if (!finish_layer<W, PER_TOKEN, ROT>(c, next_s, next_inv, s_x)) return;
-        }
-        {
-            const FusedLayer &ly = p.layer[p.L - 1];
-            if (!wait_bar_warp<PER_TOKEN>(bar_last, last_parity, abort_flag, p.status)) return;
-            last_parity ^= 1;
-            ptx::tc_fence_after();
-            if (sub == 0) {
-                uint32_t u[4];
-                ptx::tmem_ld4(c.taddr, u);
-                ptx::tmem_wait_ld();
-                // Host-buffer variant: a whole tile's results (128 x d_L floats, contiguous in `out`) are
-                // collected in shared memory and leave by one bulk store: over the host link one large
-                // write instead of 128 x d_L four-byte ones.  The slot's 128 sub-0 threads meet on an
-                // mbarrier (bounded wait, like every other) before and after filling the buffer; its
-                // first thread issues the store.
-                const bool by_bulk = !AHEAD && !C::BULK_XY && p.bulk_out && (tile + 1) * kTile <= p.n;
-                const uint32_t ot = smem_base + sm.out_tile + (uint32_t)(slot * kTile * 16);
-                if (by_bulk) {
-                    if (c.row == 0) ptx::bulk_wait_read(); // the previous tile's store has read the buffer
-                    ptx::mbar_arrive(smem_base + sm.out_sync + 8 * slot);
-                    if (!wait_bar_warp<PER_TOKEN>(smem_base + sm.out_sync + 8 * slot, out_parity, abort_flag, p.status)) return;
-                    out_parity ^= 1;
-                }
-                if (valid) {
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        if (m < p.d_L) {
-                            float c_hi = __ldg(ly.cA + m), c_lo = 0.f;
-                            if (PER_TOKEN) c_hi = __fmul_rn(c_hi, s_x);
-                            const float yv = epilogue(EPI_LINEAR, (float)(int)u[m], c_hi, c_lo, __ldg(ly.cB + m));
-                            if (by_bulk) asm volatile("st.shared.f32 [%0], %1;" ::"r"(ot + (uint32_t)((c.row * p.d_L + m) * 4)), "f"(yv) : "memory");
-                            else p.out[tok * p.d_L + m] = yv;
-                        }
-                    }
-                }
-                if (by_bulk) {
-                    ptx::fence_proxy_async();
-                    ptx::mbar_arrive(smem_base + sm.out_sync + 8 * slot);
-                    if (!wait_bar_warp<PER_TOKEN>(smem_base + sm.out_sync + 8 * slot, out_parity, abort_flag, p.status)) return;
-                    out_parity ^= 1;
-                    if (c.row == 0) ptx::bulk_s2g(p.out + tile * kTile * p.d_L, ot, (uint32_t)(kTile * p.d_L * 4));
-                }
-            }
-            ptx::tc_fence_before();
-        }
-    }
-    if (!AHEAD && !C::BULK_XY && sub == 0 && c.row == 0) ptx::bulk_wait_all(); // the last tiles' stores
-}
-
-template <int W, bool SPREAD>
-__device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, uint32_t tmem_base,
-                         volatile int *abort_flag)
-{
-    using C = Cfg<W>;
-    uint32_t codes_parity[2] = {0, 0};
-    const uint32_t idesc_hidden = ptx::idesc_i8(kTile, C::NW), idesc_last = ptx::idesc_i8(kTile, 16);
-    const uint32_t slab = C::PIECE_BYTES;
-    // each K step of 32 advances a descriptor's start-address field (bits 0-13, 16-byte units) by
-    // two core-matrix columns
-    const uint64_t a_step = (uint64_t)((2 * kTile * 16) >> 4);
-    long long use = 0; // ring uses so far (streaming mode)
-    bool ok = true;
-    for (long long r = 0; ok; ++r) {
-        if (tile_index<SPREAD>(r, 0, C::SLOTS) >= p.n_tiles) break;
-        const int active = (C::SLOTS == 2 && tile_index<SPREAD>(r, 1, C::SLOTS) < p.n_tiles) ? 2 : 1;
-        for (int l = 2; l < p.L && ok; ++l) {
-            if constexpr (C::NHALF == 2) {
-                // width 512: eight pieces per layer, the four k-pieces of output columns 0..255 first;
-                // each half of the accumulator is committed on its own barrier as soon as it is complete
-                for (int pc = 0; pc < C::PIECES && ok; ++pc) {
-                    const int half = pc / C::KSLABS, ksl = pc % C::KSLABS;
-                    const int stage = (int)(use % p.n_stages);
-                    const uint32_t par = (uint32_t)((use / p.n_stages) & 1);
-                    if (!wait_bar<0, kHintNs>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
-                    if (pc == 0) {
-                        if (!wait_bar<0, kHintNs>(smem_base + sm.codes_full, codes_parity[0], abort_flag, p.status)) { ok = false; break; }
-                        codes_parity[0] ^= 1;
-                        ptx::tc_fence_after();
-                    }
-                    const uint32_t b_addr = smem_base + sm.ring + (uint32_t)stage * C::PIECE_BYTES;
-                    const uint64_t ad0 = ptx::smem_desc(smem_base + sm.a_tile[0] + ksl * (C::SLABK / 16) * (kTile * 16), kTile * 16, 128);
-                    const uint32_t d = tmem_base + (uint32_t)(half * C::NW);
-                    const uint64_t bd0 = ptx::smem_desc(b_addr, C::NW * 16, 128);
-                    const uint64_t b_step = (uint64_t)((2 * C::NW * 16) >> 4);
-#pragma unroll
-                    for (int ks = 0; ks < C::SLABK / 32; ++ks)
-                        ptx::mma_i8(d, ad0 + ks * a_step, bd0 + ks * b_step, idesc_hidden, (ksl > 0 || ks > 0) ? 1u : 0u);
-                    if (ksl == C::KSLABS - 1) ptx::mma_commit(smem_base + sm.acc_full + 8 * half);
-                    ptx::mma_commit(smem_base + sm.w_empty + 8 * stage);
-                    ++use;
-                }
-                continue;
-            }
-            for (int ksl = 0; ksl < C::KSLABS && ok; ++ksl) {
-                const int slab_id = (l - 2) * C::KSLABS + ksl;
-                const int stage = p.resident ? slab_id : (int)(use % p.n_stages);
-                const uint32_t par = p.resident ? 0u : (uint32_t)((use / p.n_stages) & 1);
-                if (!wait_bar<0, kHintNs>(smem_base + sm.w_full + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
-                const uint32_t b_addr = smem_base + sm.ring + (uint32_t)stage * slab;
-                for (int s = 0; s < active; ++s) {
-                    if (ksl == 0) {
-                        if (!wait_bar<0, kHintNs>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
-                        codes_parity[s] ^= 1;
-                        ptx::tc_fence_after();
-                    }
-                    const uint64_t ad0 = ptx::smem_desc(smem_base + sm.a_tile[s] + ksl * (C::SLABK / 16) * (kTile * 16), kTile * 16, 128);
-#pragma unroll
-                    for (int half = 0; half < C::NHALF; ++half) {
-                        const uint32_t d = tmem_base + (uint32_t)(s * C::TMEM_COLS_PER_SLOT + half * C::NW);
-                        const uint64_t bd0 = ptx::smem_desc(b_addr + half * C::NW * 16, W * 16, 128);
-                        const uint64_t b_step = (uint64_t)((2 * W * 16) >> 4);
-#pragma unroll
-                        for (int ks = 0; ks < C::SLABK / 32; ++ks)
-                            ptx::mma_i8(d, ad0 + ks * a_step, bd0 + ks * b_step, idesc_hidden, (ksl > 0 || ks > 0) ? 1u : 0u);
-                    }
-                    if (ksl == C::KSLABS - 1) ptx::mma_commit(smem_base + sm.acc_full + 8 * (s * 4));
-                }
-                if (!ok) break;
-                if (!p.resident) {
-                    ptx::mma_commit(smem_base + sm.w_empty + 8 * stage);
-                    ++use;
-                }
-            }
-        }
-        if (!ok) break;
-        // last layer: N = 16, its weights stay in shared memory
-        if (!wait_bar<0, kHintNs>(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
-        for (int s = 0; s < active; ++s) {
-            if (!wait_bar<0, kHintNs>(smem_base + sm.codes_full + 8 * s, codes_parity[s], abort_flag, p.status)) { ok = false; break; }
-            codes_parity[s] ^= 1;
-            ptx::tc_fence_after();
-            const uint32_t d = tmem_base + (uint32_t)(s * C::TMEM_COLS_PER_SLOT);
-            const uint64_t ad0 = ptx::smem_desc(smem_base + sm.a_tile[s], kTile * 16, 128);
-            const uint64_t bd0 = ptx::smem_desc(smem_base + sm.last_w, 16 * 16, 128);
-            const uint64_t b_step = (uint64_t)((2 * 16 * 16) >> 4);
-#pragma unroll
-            for (int ks = 0; ks < W / 32; ++ks)
-                ptx::mma_i8(d, ad0 + ks * a_step, bd0 + ks * b_step, idesc_last, ks > 0 ? 1u : 0u);
-            ptx::mma_commit(smem_base + sm.acc_last + 8 * s);
-        }
-    }
-    if (!ok) { // give the MMAs already issued a bounded time to finish before TMEM is released
-        ptx::mma_commit(smem_base + sm.drain);
-        const unsigned long long t0 = ptx::globaltimer();
-        while (!ptx::mbar_try_wait(smem_base + sm.drain, 0) && ptx::globaltimer() - t0 < kWaitLimitNs) {}
-    }
-}
-
-template <int W, bool SPREAD>
-__device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
-{
-    using C = Cfg<W>;
-    const uint32_t slab = C::PIECE_BYTES;
-    ptx::mbar_expect_tx(smem_base + sm.last_full, 16 * W);
-    ptx::bulk_g2s(smem_base + sm.last_w, p.layer[p.L - 1].qw_umma, 16 * W, smem_base + sm.last_full);
-    const int slabs = (p.L - 2) * C::PIECES; // per tile round
-    if (slabs <= 0) return;
-    long long rounds = 0;
-    for (long long r = 0;; ++r) {
-        if (tile_index<SPREAD>(r, 0, C::SLOTS) >= p.n_tiles) break;
-        ++rounds;
-    }
-    const long long total = p.resident ? slabs : rounds * slabs;
-    long long issued = 0;
-    bool ok = true;
-    for (long long i = 0; i < total; ++i) {
-        const int stage = (int)(i % p.n_stages);
-        if (i >= p.n_stages) {
-            uint32_t par = (uint32_t)(((i / p.n_stages) - 1) & 1);
-            if (!wait_bar<0, kHintNs>(smem_base + sm.w_empty + 8 * stage, par, abort_flag, p.status)) { ok = false; break; }
-        }
-        const int id = (int)(i % slabs);
-        const int l = 2 + id / C::PIECES, pc = id % C::PIECES;
-        ptx::mbar_expect_tx(smem_base + sm.w_full + 8 * stage, slab);
-        // several copies in flight per slab: one large bulk copy did not reach the L2 bandwidth
-        for (uint32_t off = 0; off < slab; off += kCopyBytes) {
-            const uint32_t bytes = slab - off < kCopyBytes ? slab - off : kCopyBytes;
-            ptx::bulk_g2s(smem_base + sm.ring + (uint32_t)stage * slab + off,
-                          p.layer[l - 1].qw_umma + (size_t)pc * slab + off, bytes, smem_base + sm.w_full + 8 * stage);
-        }
-        ++issued;
-    }
-    if (!ok || *abort_flag) { // let copies in flight land before the CTA may exit
-        const unsigned long long t0 = ptx::globaltimer();
-        for (long long i = issued > p.n_stages ? issued - p.n_stages : 0; i < issued; ++i) {
-            const int stage = (int)(i % p.n_stages);
-            const uint32_t par = (uint32_t)((i / p.n_stages) & 1);
-            while (!ptx::mbar_try_wait(smem_base + sm.w_full + 8 * stage, par) &&
-                   ptx::globaltimer() - t0 < kWaitLimitNs) {}
-        }
-    }
-}
-
-// Width 512.  Coordinates: one bulk copy per whole tile (1 KB) into the slot's buffer, issued as
-// soon as the slot's threads have taken the previous tile's coordinates out of it.
-template <int W, bool SPREAD>
-__device__ void xy_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
-{
-    using C = Cfg<W>;
-    if (!p.bulk_xy) return;
-    uint32_t k[2] = {0, 0};
-    bool ok = true;
-    for (long long r = 0; ok; ++r) {
-        if (tile_index<SPREAD>(r, 0, C::SLOTS) >= p.n_tiles) break;
-        for (int s = 0; s < C::SLOTS && ok; ++s) {
-            const long long tile = tile_index<SPREAD>(r, s, C::SLOTS);
-            if (tile >= p.n_tiles || (tile + 1) * kTile > p.n) continue; // none, or ragged: the threads load it themselves
-            if (k[s] > 0 && !wait_bar<0, kHintNs>(smem_base + sm.xy_empty + 8 * s, (k[s] - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-            ptx::mbar_expect_tx(smem_base + sm.xy_full + 8 * s, kTile * 8);
-            ptx::bulk_g2s(smem_base + sm.xy + (uint32_t)(s * kTile * 8), p.coords + tile * kTile * 2, kTile * 8, smem_base + sm.xy_full + 8 * s);
-            ++k[s];
-        }
-    }
-    if (!ok || *abort_flag) { // let a copy in flight land before the CTA may exit
-        const unsigned long long t0 = ptx::globaltimer();
-        for (int s = 0; s < C::SLOTS; ++s)
-            if (k[s] > 0)
-                while (!ptx::mbar_try_wait(smem_base + sm.xy_full + 8 * s, (k[s] - 1) & 1u) && ptx::globaltimer() - t0 < kWaitLimitNs) {}
-    }
-}
-
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD>
-__global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_constant__ FusedParams p)
-{
-    using C = Cfg<W>;
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = ptx::smem_u32(smem_raw);
-    const uint32_t smem_base = (raw + 1023u) & ~1023u;
-    uint8_t *smem_gen = smem_raw + (smem_base - raw);
-    const SmemMap sm = smem_map(W, p.n_stages, p.const_words);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_gen + sm.abort_flag);
-    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(smem_gen + sm.tmem_holder);
-
-    if (threadIdx.x == 0) {
-        *abort_flag = 0;
-        for (int i = 0; i < 8; ++i) ptx::mbar_init(smem_base + sm.acc_full + 8 * i, 1);
-        for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(smem_base + sm.acc_last + 8 * s, 1);
-            ptx::mbar_init(smem_base + sm.codes_full + 8 * s, C::SLOT_THREADS);
-            for (int q = 0; q < 4; ++q) ptx::mbar_init(smem_base + sm.slot_sync + 8 * (s * 4 + q), C::R * 32);
-        }
-        ptx::mbar_init(smem_base + sm.last_full, 1);
-        if constexpr (!C::BULK_XY) {
-            for (int s2 = 0; s2 < 2; ++s2) ptx::mbar_init(smem_base + sm.out_sync + 8 * s2, kTile);
-        }
-        if constexpr (C::BULK_XY) {
-            for (int s2 = 0; s2 < 2; ++s2) {
-                ptx::mbar_init(smem_base + sm.xy_full + 8 * s2, 1);
-                ptx::mbar_init(smem_base + sm.xy_empty + 8 * s2, C::SLOT_THREADS);
-            }
-        }
-        ptx::mbar_init(smem_base + sm.drain, 1);
-        for (int i = 0; i < kMaxStages; ++i) {
-            ptx::mbar_init(smem_base + sm.w_full + 8 * i, 1);
-            ptx::mbar_init(smem_base + sm.w_empty + 8 * i, 1);
-        }
-        ptx::fence_mbar_init();
-    }
-    if (warp == kMmaWarp) {
-        ptx::tmem_alloc(smem_base + sm.tmem_holder, 512);
-        ptx::tmem_relinquish();
-    }
-    // per-layer epilogue constants -> shared memory
-    {
-        uint32_t *dst = reinterpret_cast<uint32_t *>(smem_gen + sm.consts);
-        for (int l = 0; l < p.L - 1; ++l) {
-            const FusedLayer &ly = p.layer[l];
-            uint32_t *d = dst + ly.c_off;
-            const bool fixed = ly.epi_mode == EPI_SINE_FIXED;
-            const uint32_t *srcA = fixed ? ly.fxP : reinterpret_cast<const uint32_t *>(ly.cA);
-            const uint32_t *srcB = fixed ? ly.fxB : reinterpret_cast<const uint32_t *>(ly.cB);
-            const uint32_t *srcC = fixed ? ly.fxQ : reinterpret_cast<const uint32_t *>(ly.cA_lo);
-            const int areas = (l == 0) ? (fixed ? 3 : 4) : (ly.epi_mode == EPI_SINE_WIDE ? 3 : 2);
-            for (int i = threadIdx.x; i < W; i += C::THREADS) { // i: tensor-memory column, m: its feature
-                const int m = fused_feature(i, W);
-                d[i] = __ldg(srcA + m);
-                d[W + i] = __ldg(srcB + m);
-                if (areas >= 3) d[2 * W + i] = __ldg(srcC + m);
-                if (areas >= 4) d[3 * W + i] = __ldg(ly.qw_k4m + m);
-            }
-        }
-    }
-    ptx::tc_fence_before();
-    __syncthreads();
-    ptx::tc_fence_after();
-    const uint32_t tmem_base = *tmem_holder;
-
-    if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
-    } else if (warp == kMmaWarp) {
-        if (lane == 0) mma_role<W, SPREAD>(p, sm, smem_base, tmem_base, abort_flag);
-    } else if (warp == kLoadWarp) {
-        if (lane == 0) load_role<W, SPREAD>(p, sm, smem_base, abort_flag);
-    } else {
-        if constexpr (C::BULK_XY) {
-            if (lane == 0) xy_role<W, SPREAD>(p, sm, smem_base, abort_flag);
-        }
-    }
-    ptx::tc_fence_before();
-    __syncthreads();
-    if (warp == kMmaWarp) {
-        __syncwarp();
-        ptx::tmem_dealloc(tmem_base, 512);
-    }
-}
-
-// ------------------------------------------------------------------------------------------ host
-
-typedef void (*fused_fn)(const FusedParams);
-
-template <int W, bool SPREAD, bool AHEAD> static fused_fn pick_flags(bool per_token, bool rot)
-{
-    if (rot) return per_token ? fused_kernel<W, true, true, SPREAD, AHEAD> : fused_kernel<W, false, true, SPREAD, AHEAD>;
-    return per_token ? fused_kernel<W, true, false, SPREAD, AHEAD> : fused_kernel<W, false, false, SPREAD, AHEAD>;
-}
-template <int W, bool AHEAD_OK> static fused_fn pick_width(bool per_token, bool rot, bool spread, bool ahead)
-{
-    if (AHEAD_OK && ahead) return spread ? pick_flags<W, true, AHEAD_OK>(per_token, rot) : pick_flags<W, false, AHEAD_OK>(per_token, rot);
-    return spread ? pick_flags<W, true, false>(per_token, rot) : pick_flags<W, false, false>(per_token, rot);
-}
 // spread: the tile-to-CTA mapping for launches smaller than one tile per slot of every SM (tile_index);
 // ahead: coordinates of the next tile copied to shared memory early (device memory only; width 512
 // gained nothing from it and has no such variant)
 static fused_fn pick_kernel(int W, bool per_token, bool rot, bool spread, bool ahead)
 {
     switch (W) {
-    case 64: return pick_width<64, true>(per_token, rot, spread, ahead);
-    case 128: return pick_width<128, true>(per_token, rot, spread, ahead);
-    case 256: return pick_width<256, true>(per_token, rot, spread, ahead);
-    case 512: return pick_width<512, false>(per_token, rot, spread, ahead);
+    case 64: return fused_pick_64(per_token, rot, spread, ahead);
+    case 128: return fused_pick_128(per_token, rot, spread, ahead);
+    case 256: return fused_pick_256(per_token, rot, spread, ahead);
+    case 512: return fused_pick_512(per_token, rot, spread, ahead);
+    }
+    return nullptr;
+}
+
+static fused_dump_fn pick_dump_kernel(int W, bool per_token, bool rot)
+{
+    switch (W) {
+    case 64: return fused_pick_dump_64(per_token, rot);
+    case 128: return fused_pick_dump_128(per_token, rot);
+    case 256: return fused_pick_dump_256(per_token, rot);
+    case 512: return fused_pick_dump_512(per_token, rot);
     }
     return nullptr;
 }
@@ -1087,6 +85,9 @@ dhq_status_t fused_create(dhq_handle_s *h)
         if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
+    fused_dump_fn fd = pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    if (!fd || cudaFuncSetAttribute(fd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+        return DHQ_ERR_CUDA;
     return DHQ_OK;
 }
 
@@ -1103,22 +104,50 @@ int64_t fused_round_tokens(const dhq_handle_s *h)
     return (int64_t)(fs ? fs->sm_count : 1) * slots * kTile;
 }
 
-dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st)
+// The per-call part of the parameter block.
+static void fill_call(const dhq_handle_s *h, FusedParams &p, const float *coords, int64_t n, float *out)
 {
-    FusedState *fs = static_cast<FusedState *>(h->fused);
-    if (!fs) return DHQ_ERR_INVALID_ARG;
-    FusedParams p = fs->p;
     p.coords = coords; p.out = out; p.n = n;
     p.n_tiles = (n + kTile - 1) / kTile;
     p.bulk_xy = (((uintptr_t)coords) & 15) == 0;
     p.bulk_out = (((uintptr_t)out) & 15) == 0 && (smem_map(h->w, p.n_stages, p.const_words).out_tile & 15) == 0;
+    p.wait_limit_ns = h->wait_limit_ns;
+    p.skip_last_weights = 0;
+}
+
+dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, bool on_host, cudaStream_t st)
+{
+    FusedState *fs = static_cast<FusedState *>(h->fused);
+    if (!fs) return DHQ_ERR_INVALID_ARG;
+    FusedParams p = fs->p;
+    fill_call(h, p, coords, n, out);
+    if (h->stall_next_forward) { // test hook, one launch only
+        p.skip_last_weights = 1;
+        h->stall_next_forward = false;
+    }
     const int slots = (h->w == 512) ? 1 : 2;
     const bool spread = slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
-    cudaPointerAttributes at;
-    const bool on_host = cudaPointerGetAttributes(&at, coords) == cudaSuccess && at.type == cudaMemoryTypeHost;
-    (void)cudaGetLastError();
     fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
+    int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
+    fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
+    h->launches++;
+    return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;
+}
+
+// The same forward by the observing instantiation of the kernel: every per-layer value the
+// caller asked for is written out from inside the fused kernel, where it is produced.
+dhq_status_t fused_forward_dump(dhq_handle_s *h, const float *coords, int64_t n, float *out, const DumpPtrs &d, cudaStream_t st)
+{
+    FusedState *fs = static_cast<FusedState *>(h->fused);
+    if (!fs) return DHQ_ERR_INVALID_ARG;
+    FusedParamsDump p;
+    static_cast<FusedParams &>(p) = fs->p;
+    fill_call(h, p, coords, n, out);
+    p.d = d;
+    const int slots = (h->w == 512) ? 1 : 2;
+    fused_dump_fn fn = pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    const long long ctas = (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
     h->launches++;

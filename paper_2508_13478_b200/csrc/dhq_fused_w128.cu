@@ -1,0 +1,10 @@
+// The fused forward kernels of hidden width 128 (see dhq_fused.cuh), compiled on their own so that
+// the widths build side by side.
+#include "dhq_fused.cuh"
+
+namespace dhq {
+
+fused_fn fused_pick_128(bool per_token, bool rot, bool spread, bool ahead) { return pick_width<128, true>(per_token, rot, spread, ahead); }
+fused_dump_fn fused_pick_dump_128(bool per_token, bool rot) { return pick_dump_width<128, true>(per_token, rot); }
+
+} // namespace dhq

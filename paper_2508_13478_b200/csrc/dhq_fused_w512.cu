@@ -1,0 +1,10 @@
+// The fused forward kernels of hidden width 512 (see dhq_fused.cuh), compiled on their own so that
+// the widths build side by side.
+#include "dhq_fused.cuh"
+
+namespace dhq {
+
+fused_fn fused_pick_512(bool per_token, bool rot, bool spread, bool ahead) { return pick_width<512, false>(per_token, rot, spread, ahead); }
+fused_dump_fn fused_pick_dump_512(bool per_token, bool rot) { return pick_dump_width<512, false>(per_token, rot); }
+
+} // namespace dhq

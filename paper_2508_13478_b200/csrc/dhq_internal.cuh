@@ -17,7 +17,8 @@ struct LayerDev {
     int slab_k = 0;            // k per contiguous slab of the tensor-core image
     int d_in = 0, d_out = 0;
     int epi_mode = EPI_LINEAR;
-    float phase_bound = 0.f;   // omega0 * max_m (sum_k |W_mk| + |b_m|), hidden layers
+    float phase_bound = 0.f;   // bound of |omega0 (s_w s_x acc + b)| over unsaturated inputs in [-1, 1] (prep_bound_kernel)
+    float *row_l1 = nullptr;   // [M] sum_k |W_mk| + |b_m| of the unquantized row
     float *w_rot = nullptr;    // [M][K] fp32 rotated weights (kept for inspection)
     float *row_absmax = nullptr; // [M]
     int8_t *qw = nullptr;      // [M][K] codes, row-major
@@ -53,9 +54,19 @@ struct dhq_handle_s {
     bool pipe_ready = false;
     int64_t launches = 0;
     void *fused = nullptr;          // state of the fused path (device parameter block)
+    unsigned long long wait_limit_ns = 2000000000ull; // bound of every wait inside the fused kernel (dhq_set_wait_limit)
+    bool stall_next_forward = false; // test hook: see dhq_debug_stall_next_forward
 };
 
 namespace dhq {
+
+// A handle's buffers live on the device that was current in dhq_prepare; a launch on another
+// device with them would fault instead of returning a status, so every entry point asks first.
+inline bool on_own_device(const dhq_handle_s *h)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
 
 // Arguments of one pass of the layer-by-layer kernel.
 struct LayerArgs {
@@ -88,6 +99,7 @@ struct PrepArgs {
     const float *W, *b;
     int d_out, d_in, K, M, Mt;
     int bits, per_channel;
+    int a_bits;            // activation bit-width (enters the phase bound)
     int rotate;            // 0: DHQ_ROT_NONE, weights are quantized as they are; 2: DHQ_ROT_BOTH, columns rotated too
     int permute_rows;      // 1: rows of the tensor-core image in fused_column order (layers 2 .. L-1)
     int sine;              // hidden or first layer
@@ -136,7 +148,20 @@ __host__ __device__ inline int fused_feature(int col, int W)
 // Fused tensor-core forward.
 dhq_status_t fused_create(dhq_handle_s *h);
 void fused_destroy(dhq_handle_s *h);
-dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, cudaStream_t st);
+// on_host: coords / out are device aliases of mapped host memory (the variants that fetch the next
+// tile's coordinates early are for device memory)
+dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, bool on_host, cudaStream_t st);
+// Per-layer dump targets of the observing instantiation of the fused kernel: device pointers
+// laid out as dhq_debug_bufs_t describes, entry l-1 for layer l, NULL entries skipped.  X is only
+// used for layer 1; the input of a later layer is the output of the one before it.
+struct DumpPtrs {
+    float *X[kMaxLayers];
+    int8_t *codes[kMaxLayers];
+    float *s_x[kMaxLayers];
+    int32_t *acc[kMaxLayers];
+    float *Y[kMaxLayers];
+};
+dhq_status_t fused_forward_dump(dhq_handle_s *h, const float *coords, int64_t n, float *out, const DumpPtrs &d, cudaStream_t st);
 // Coordinates one launch of the fused kernel works on at a time over the whole GPU (one tile per
 // slot of every SM): launches cut at multiples of this leave no SM idle.
 int64_t fused_round_tokens(const dhq_handle_s *h);

@@ -11,29 +11,34 @@ namespace dhq {
 // Epilogue variants, chosen per layer when the network is prepared.
 enum EpiMode : int {
     EPI_LINEAR = 0,    // last layer: z = c * acc + b
-    EPI_SINE_FAST = 1, // hidden layer whose phase is provably small: sin.approx(fma(acc, c, B))
+    EPI_SINE_FAST = 1, // hidden layer whose phase stays below kFastPhaseLimit (bound taken at prepare time over all
+                       // unsaturated inputs, quantization error of weights and activations included): sin.approx(fma(acc, c, B))
     EPI_SINE_WIDE = 2, // large phases: compensated phase and explicit 2*pi reduction
     EPI_SINE_FIXED = 3, // first layer with a per-tensor activation scale: phase in 32-bit fixed point
     EPI_BOTH = 4       // two-sided transform: the layer kernel undoes the output-side rotation in fp64
 };
 
-// Largest |omega0 z| for which EPI_SINE_FAST keeps the result within 1e-5 of an exact sine:
-// fma rounding (ulp(32)/2 = 1.9e-6) + constant rounding (32 * 2^-24 = 1.9e-6) + the multiply by
-// 1/(2 pi) inside sin.approx (1.5e-6) + the approximation itself (about 7e-7).
-constexpr float kFastPhaseLimit = 32.0f;
+// Largest |omega0 z| for which EPI_SINE_FAST keeps the result within 1e-5 of an exact sine.  Worst
+// case at the limit, term by term: rounding of the fma result (half an ulp of a value in [32, 64):
+// 1.9e-6), rounding of the constant c to fp32 (36 * 2^-24 = 2.1e-6) and of B (1e-7), and the
+// hardware approximation itself, measured on B200 against the fp64 sine over 2^24 arguments per
+// range (dhq_measure_sine_error): 6.2e-7 for |x| <= 3.2, 2.3e-6 to 16, 4.4e-6 to 32, 4.6e-6 to 40,
+// 5.0e-6 to 48, 8.3e-6 to 56 - its internal multiply by 1/(2 pi) loses absolute accuracy as the
+// argument grows.  Sum at 36: 8.7e-6.
+constexpr float kFastPhaseLimit = 36.0f;
 
 __device__ __forceinline__ float qmax_of(int bits) { return (float)((1 << (bits - 1)) - 1); }
 
 // Symmetric absmax scales: s = a / qmax, inv = qmax / a, both IEEE divisions; a = 0 -> 0, 0.
+// An absmax so small that qmax / a is not a finite fp32 number (a below about 3.7e-37 at 8 bits)
+// counts as zero: no code can be formed with an infinite scale, and values of that size
+// contribute nothing.
 __device__ __forceinline__ void scales_of(float a, float qmaxf, float &s, float &inv)
 {
-    if (a > 0.0f) {
-        s = __fdiv_rn(a, qmaxf);
-        inv = __fdiv_rn(qmaxf, a);
-    } else {
-        s = 0.0f;
-        inv = 0.0f;
-    }
+    const float s_ = __fdiv_rn(a, qmaxf), i_ = __fdiv_rn(qmaxf, a);
+    const bool ok = a > 0.0f && i_ <= 3.402823466e+38f; // false for a = 0 (i_ = inf), NaN, and the overflow case
+    s = ok ? s_ : 0.0f;
+    inv = ok ? i_ : 0.0f;
 }
 
 // q = clamp(round_half_even(fl32(v * inv)), -qmax, +qmax).  Clamping before rounding gives the

@@ -1,5 +1,6 @@
 // Micro-benchmarks of the pipes that bound the fused kernel (see include/dhq_peaks.h).
 #include <cuda_runtime.h>
+#include <cstring>
 #include "../../include/dhq_peaks.h"
 #include "dhq_internal.cuh"
 #include "dhq_tmem.cuh"
@@ -99,7 +100,42 @@ template <int PIPE> static cudaError_t run_scalar(int blocks, int iters, float *
     return cudaGetLastError();
 }
 
+// Largest |f(x) - sin(x)| over `count` fp32 arguments spread evenly over [lo, hi]; f is the
+// hardware approximation alone (mode 0) or with the explicit 2 pi reduction in front (mode 1); the
+// reference is the fp64 sine of the same fp32 argument.
+__global__ void sine_error_kernel(float lo, float hi, long long count, int mode, unsigned long long *worst_bits)
+{
+    double worst = 0.0;
+    const double step = count > 1 ? ((double)hi - (double)lo) / (double)(count - 1) : 0.0;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x) {
+        const float x = (float)((double)lo + step * (double)i);
+        const float y = mode == 1 ? sin_wide(x) : sin_approx(x);
+        const double e = fabs((double)y - sin((double)x));
+        if (e > worst) worst = e;
+    }
+    atomicMax(worst_bits, (unsigned long long)__double_as_longlong(worst)); // non-negative doubles order as integers
+}
+
 } // namespace dhq
+
+extern "C" int dhq_measure_sine_error(float lo, float hi, long long count, int mode, void *stream, double *max_abs_err)
+{
+    if (!max_abs_err || count < 1 || !(lo <= hi) || (mode != 0 && mode != 1)) return -1;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long *d = nullptr, bits = 0;
+    if (cudaMalloc(&d, sizeof(bits)) != cudaSuccess) return -3;
+    int rc = 0;
+    if (cudaMemsetAsync(d, 0, sizeof(bits), st) != cudaSuccess) rc = -5;
+    if (rc == 0) {
+        dhq::sine_error_kernel<<<1024, 256, 0, st>>>(lo, hi, count, mode, d);
+        if (cudaGetLastError() != cudaSuccess || cudaMemcpyAsync(&bits, d, sizeof(bits), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            rc = -6;
+    }
+    cudaFree(d);
+    if (rc == 0) memcpy(max_abs_err, &bits, sizeof(double));
+    return rc;
+}
 
 extern "C" int dhq_measure_pipe(int pipe, int iters, void *stream, double *ops_per_s, double *ms)
 {

@@ -25,8 +25,7 @@ __global__ void prep_rotate_kernel(PrepArgs a)
         float s = 0.f;
         for (int i = 0; i < (blockDim.x + 31) / 32; ++i) s += red[i];
         float bm = (m < a.d_out) ? fabsf(a.b[m]) : 0.f;
-        float bound = (float)a.omega0 * (s + bm) * 1.0001f;
-        atomicMax((unsigned int *)a.phase_bound, __float_as_uint(bound));
+        a.dev.row_l1[m] = s + bm; // |W_m . x + b_m| <= this for inputs in [-1, 1]
         a.dev.bias[m] = (m < a.d_out) ? a.b[m] : 0.0f;
     }
     for (int h = 1; h < (a.rotate ? K : 1); h <<= 1) {
@@ -132,6 +131,38 @@ __global__ void prep_quant_kernel(PrepArgs a)
     }
 }
 
+// Bound of the phase omega0 (s_w s_x acc + b) that the epilogue of a hidden layer sees, over all
+// inputs in [-1, 1]^K whose codes do not saturate: the unquantized bound sum_k |W_mk| + |b_m|
+// plus what the two quantizers can add.  With s_x q_x = x~ + e_x, |e_x| <= s_x / 2 and
+// s_w q_w = w~ + e_w, |e_w| <= s_w / 2:
+//   s_w s_x acc = W x + sum_k e_w x~_k + sum_k s_w q_w e_x
+//   |sum e_w x~|    <= (s_w / 2) * sum_k |x~_k|,  sum |x~_k| <= K sqrt(K) rotated (||x~||_2 = sqrt(K) ||x||_2), K unrotated
+//   |sum s_w q_w e_x| <= (s_x / 2) * s_w * sum_k |q_w[m][k]|,  s_x <= max |x~| / qmax <= K / qmax rotated, 1 / qmax unrotated.
+// The maximum over the rows goes to a.phase_bound; it decides between the fast and the wide sine.
+__global__ void prep_bound_kernel(PrepArgs a)
+{
+    __shared__ float red[32];
+    const int K = a.K;
+    const float xsum = a.rotate ? (float)K * sqrtf((float)K) : (float)K;
+    const float sx_max = (a.rotate ? (float)K : 1.0f) / qmax_of(a.a_bits);
+    float worst = 0.f;
+    for (int m = threadIdx.x; m < a.M; m += blockDim.x) {
+        float qsum = 0.f;
+        for (int k = 0; k < K; ++k) qsum += fabsf((float)a.dev.qw[(size_t)m * K + k]);
+        const float sw = a.dev.s_w[m];
+        const float slack = 0.5f * sw * xsum + 0.5f * sx_max * sw * qsum;
+        worst = fmaxf(worst, (float)a.omega0 * (a.dev.row_l1[m] + slack) * 1.0001f);
+    }
+    for (int o = 16; o; o >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = worst;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float r = 0.f;
+        for (int i = 0; i < (blockDim.x + 31) / 32; ++i) r = fmaxf(r, red[i]);
+        *a.phase_bound = r;
+    }
+}
+
 // Epilogue constants in fp64, rounded once: cA = fl32(A), cA_lo = fl32(A - cA) with
 // A = f * s_w[m] (* s_x when the activation scale is per tensor), cB = fl32(f * b[m]),
 // f = omega0 for sine layers and 1 for the last layer.  Also derives s_x and inv from the frozen
@@ -182,7 +213,8 @@ cudaError_t launch_prepare(const PrepArgs &a, cudaStream_t st, int64_t *launches
     prep_scales_kernel<<<1, 256, 0, st>>>(a);
     int total = a.Mt * a.K;
     prep_quant_kernel<<<(total + 255) / 256, 256, 0, st>>>(a);
-    *launches += 3;
+    prep_bound_kernel<<<1, 256, 0, st>>>(a);
+    *launches += 4;
     return cudaGetLastError();
 }
 

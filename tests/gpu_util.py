@@ -28,7 +28,9 @@ def check_weights(h, net):
         assert np.array_equal(scales.view(np.uint32), lay.s_w.view(np.uint32)), f"weight scales of layer {l}"
 
 
-def run_debug(h, net, coords_dev):
+def run_debug(h, net, coords_dev, fused=False):
+    """Per-layer dumps of the layer-by-layer path, or (fused=True) written by the fused tensor-core
+    kernel itself from where each value is produced."""
     n = coords_dev.shape[0]
     L = len(net.layers)
     bufs = {"X": [], "codes": [], "s_x": [], "acc": [], "Y": []}
@@ -39,8 +41,9 @@ def run_debug(h, net, coords_dev):
         bufs["acc"].append(torch.empty((n, lay.M_pad), dtype=torch.int32, device="cuda"))
         bufs["Y"].append(torch.empty((n, lay.M_pad), dtype=torch.float32, device="cuda"))
     out = torch.empty((n, net.dims[-1]), dtype=torch.float32, device="cuda")
-    dhq.dhq_forward_debug(h, coords_dev, out, bufs)
+    dhq.dhq_forward_debug(h, coords_dev, out, bufs, fused=fused)
     torch.cuda.synchronize()
+    assert dhq.dhq_last_status(h) == 0
     return out, bufs
 
 

@@ -1,0 +1,241 @@
+"""GPU parity of the fused tensor-core kernel itself, stage by stage.
+
+dhq_forward_fused_debug runs the kernel that dhq_forward runs, compiled with stores at the places
+where each per-layer value exists (codes on their way into the operand tile, activation scales,
+int32 accumulators as read from tensor memory, layer outputs after the sine).  The oracle, given
+the kernel's own input of each layer, must reproduce codes, scale bits and accumulators exactly and
+the fp32 outputs within 1e-5; the chain must close and dhq_forward must return the same bits.
+"""
+import numpy as np
+import pytest
+import torch
+
+import dhq_inputs
+from tests.gpu_util import TOL_Y, check_layers_against_oracle, check_weights, prepare_pair, run_debug, to_dev
+
+pytestmark = pytest.mark.gpu
+
+dhq = pytest.importorskip("paper_2508_13478_b200")
+from oracle import dhq_oracle as orc  # noqa: E402
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2508_13478_b200 import build
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _observe(h, net, coords_np, calib_is_this_set=True):
+    cd = to_dev(coords_np)
+    out_dump, bufs = run_debug(h, net, cd, fused=True)
+    worst = check_layers_against_oracle(h, net, coords_np, out_dump, bufs, calib_is_this_set=calib_is_this_set)
+    out = torch.full((coords_np.shape[0], net.dims[-1]), float("nan"), device="cuda")
+    dhq.dhq_forward(h, cd, out)
+    torch.cuda.synchronize()
+    assert dhq.dhq_last_status(h) == 0
+    assert torch.equal(out.view(torch.int32), out_dump.view(torch.int32)), "dhq_forward != observed fused kernel"
+    return worst
+
+
+@pytest.mark.parametrize("rotate", [True, False])
+@pytest.mark.parametrize("width,a_gran", [(64, 0), (64, 1), (128, 0), (128, 1), (256, 0), (256, 1), (512, 0), (512, 1)])
+def test_fused_kernel_stages_match_the_oracle(width, a_gran, rotate):
+    # more than one round of the persistent grid (148 SMs x slots x 128 tokens) plus a ragged tail
+    wl = dhq_inputs.Workload("obs", (2, width, width, width, 3), 30.0, 700 + width + a_gran, 8, 8, a_gran, a_gran, (8, 8))
+    n = 148 * (1 if width == 512 else 2) * 128 + 300
+    coords = dhq_inputs.grid_coords(251, 157)[:n]
+    weights, biases = wl.network()
+    h, net = prepare_pair(wl.dims, weights, biases, wl.omega0, 8, 8, a_gran, a_gran, rotate=rotate)
+    try:
+        check_weights(h, net)
+        if a_gran == 0:
+            dhq.dhq_calibrate(h, to_dev(coords))
+        _observe(h, net, coords)
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_all_of_c3_through_the_observed_fused_kernel():
+    # every coordinate of the 512 x 512 grid, 65,536 at a time
+    w = dhq_inputs.WORKLOADS["C3"]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        check_weights(h, net)
+        coords = w.coords()
+        worst = 0.0
+        for t0 in range(0, w.n, 65536):
+            worst = max(worst, _observe(h, net, np.ascontiguousarray(coords[t0:t0 + 65536])))
+        print(f"C3, all {w.n} coordinates: integer stages exact, outputs within {worst:.2e}")
+    finally:
+        dhq.dhq_destroy(h)
+
+
+@pytest.mark.parametrize("name", ["C4-W4A4", "C4-W6A6", "C5"])
+def test_contiguous_chunk_of_the_large_grids(name):
+    # 65,536 consecutive coordinates from the middle of the grid: 1.7 rounds of the persistent grid
+    # at width 256, 3.5 at width 512; per-tensor scales (C5) are frozen on the whole grid and the
+    # first layer's frozen absmax is checked against the oracle on the whole grid
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        check_weights(h, net)
+        coords = w.coords()
+        if w.a_gran == 0:
+            dhq.dhq_calibrate(h, to_dev(coords))
+            a1 = float(orc.rotated_absmax(net, 1, orc.pad_coords(coords)).max())
+            assert np.float32(dhq.dhq_get_layer(h, 1)[2]) == np.float32(a1)
+        t0 = w.n // 2 - 12345
+        _observe(h, net, np.ascontiguousarray(coords[t0:t0 + 65536]), calib_is_this_set=False)
+    finally:
+        dhq.dhq_destroy(h)
+
+
+@pytest.mark.parametrize("name", ["C3", "C4-W4A4", "C4-W6A6", "C5"])
+def test_full_grid_launch_equals_the_observed_kernel_on_samples(name):
+    # The launch bench.py times (whole grid, one dhq_forward call) against the observed kernel on
+    # 3,000 tokens sampled over the grid, the last tile included; those go through the oracle.
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        grid = to_dev(w.coords())
+        if w.a_gran == 0:
+            dhq.dhq_calibrate(h, grid)
+            a1 = float(orc.rotated_absmax(net, 1, orc.pad_coords(w.coords())).max())
+            assert np.float32(dhq.dhq_get_layer(h, 1)[2]) == np.float32(a1)
+        full = torch.empty((w.n, w.dims[-1]), device="cuda")
+        dhq.dhq_forward(h, grid, full)
+        torch.cuda.synchronize()
+        assert dhq.dhq_last_status(h) == 0
+        idx = np.unique(np.concatenate([np.linspace(0, w.n - 1, 2990).astype(np.int64), np.arange(w.n - 10, w.n)]))
+        sample = np.ascontiguousarray(w.coords()[idx])
+        out_dump, bufs = run_debug(h, net, to_dev(sample), fused=True)
+        check_layers_against_oracle(h, net, sample, out_dump, bufs, calib_is_this_set=False)
+        assert torch.equal(full[torch.from_numpy(idx).cuda()].view(torch.int32), out_dump.view(torch.int32))
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_observed_kernel_equals_the_layer_by_layer_dumps():
+    # two independent CUDA routes (tensor-core fused kernel, dp4a layer kernel) give the same dumps
+    w = dhq_inputs.WORKLOADS["C3"]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        cd = to_dev(w.coords()[:5000])
+        out_a, a = run_debug(h, net, cd, fused=True)
+        out_b, b = run_debug(h, net, cd, fused=False)
+        assert torch.equal(out_a.view(torch.int32), out_b.view(torch.int32))
+        for key in ("X", "codes", "s_x", "acc", "Y"):
+            for l in range(len(net.layers)):
+                ta, tb = a[key][l], b[key][l]
+                same = torch.equal(ta.view(torch.int32), tb.view(torch.int32)) if ta.dtype == torch.float32 else torch.equal(ta, tb)
+                assert same, f"{key} of layer {l + 1}"
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_absmax_without_a_finite_scale_counts_as_zero():
+    # coordinates so small that qmax / absmax overflows fp32: all codes zero, scale zero, and the
+    # first layer then returns sin(omega0 b); just above the threshold the quantizer works normally
+    w = dhq_inputs.WORKLOADS["C1"]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 0, 1)
+    try:
+        coords = np.array([[1e-39, 0.0], [1e-38, -1e-38], [1e-37, 0.0], [3e-37, 1e-37], [1e-36, 0.0], [0.25, -0.5]], np.float32)
+        cd = to_dev(coords)
+        for fused in (False, True):
+            out, bufs = run_debug(h, net, cd, fused=fused)
+            check_layers_against_oracle(h, net, coords, out, bufs)
+            codes = bufs["codes"][0].cpu().numpy()
+            s_x = bufs["s_x"][0].cpu().numpy()
+            assert not codes[:3].any() and not s_x[:3].any()
+            assert np.abs(codes[3:]).max(axis=1).tolist() == [127, 127, 127] and (s_x[3:] > 0).all()
+    finally:
+        dhq.dhq_destroy(h)
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C5"])
+def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable(name):
+    # The copy warp leaves out one piece (the last layer's weights); nothing is in flight for it.
+    # The warps that wait for it give up after the handle's wait limit, the kernel frees its tensor
+    # memory and returns, the status word says TIMEOUT, and the next launch is bit-correct again.
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        coords = np.ascontiguousarray(w.coords()[:100])            # one tile
+        cd = to_dev(coords)
+        if w.a_gran == 0:
+            dhq.dhq_calibrate(h, cd)
+        ref = torch.empty((100, w.dims[-1]), device="cuda")
+        dhq.dhq_forward(h, cd, ref)
+        torch.cuda.synchronize()
+        assert dhq.dhq_last_status(h) == 0
+        dhq.dhq_set_wait_limit(h, 5_000_000)                       # 5 ms
+        dhq.dhq_debug_stall_next_forward(h)
+        junk = torch.zeros_like(ref)
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        dhq.dhq_forward(h, cd, junk)
+        t1.record()
+        torch.cuda.synchronize()
+        assert t0.elapsed_time(t1) < 500.0                         # milliseconds: it gave up, it did not sit out 2 s
+        assert dhq.dhq_last_status(h) == 6                         # DHQ_ERR_TIMEOUT
+        assert dhq.dhq_last_status(h) == 0                         # reading clears it
+        out = torch.zeros_like(ref)
+        dhq.dhq_forward(h, cd, out)                                # the hook was for one launch only
+        torch.cuda.synchronize()
+        assert dhq.dhq_last_status(h) == 0
+        assert torch.equal(out.view(torch.int32), ref.view(torch.int32))
+        out_dump, bufs = run_debug(h, net, cd, fused=True)
+        check_layers_against_oracle(h, net, coords, out_dump, bufs)
+        with pytest.raises(dhq.DhqError):
+            dhq.dhq_set_wait_limit(h, 10)                          # below the minimum
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_free_running_chains_differ_only_through_code_flips_at_rounding_ties():
+    # Oracle on its own chain (fp64 sines rounded to fp32) against the kernel on its own chain (fp32
+    # sines).  Every coordinate whose outputs differ by more than 1e-5 must trace back to a first
+    # layer where an activation code differs, there by one step only, with the value to be rounded
+    # next to a half-integer (as close as the two chains' inputs of that layer allow).
+    w = dhq_inputs.WORKLOADS["C2"]
+    weights, biases = w.network()
+    coords = np.ascontiguousarray(w.coords()[::8])
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 0, 1)      # per-token scales: no calibration coupling
+    try:
+        out_dump, bufs = run_debug(h, net, to_dev(coords), fused=True)
+        ref, per = orc.forward(net, coords, return_layers=True)
+        got = out_dump.cpu().numpy().astype(np.float64)
+        far = np.abs(got - ref).max(axis=1) > TOL_Y
+        L = len(net.layers)
+        gpu_codes = [bufs["codes"][l].cpu().numpy().astype(np.int32) for l in range(L)]
+        gpu_X = [bufs["X"][l].cpu().numpy() for l in range(L)]
+        first = np.full(coords.shape[0], -1)
+        for l in range(L - 1, -1, -1):
+            differs = (gpu_codes[l] != per[l]["codes"]).any(axis=1)
+            first[differs] = l
+        assert np.all(first[far] >= 0), "outputs differ although every code agrees"
+        agree_everywhere = first < 0
+        assert np.abs(got - ref)[agree_everywhere].max() <= TOL_Y
+        flips = 0
+        for t in np.nonzero(first >= 0)[0]:
+            l = first[t]
+            diff = gpu_codes[l][t] - per[l]["codes"][t]
+            assert np.abs(diff).max() == 1
+            inv = orc.scales(float(np.abs(per[l]["Xrot"][t]).max()), 8)[1]
+            tq = per[l]["Xrot"][t].astype(np.float64) * float(inv)
+            room = float(inv) * np.abs(gpu_X[l][t].astype(np.float64) - per[l]["X"][t]).sum() * 1.5 + 127 * 2.0 ** -20
+            k = np.nonzero(diff)[0]
+            assert np.all(np.abs(np.abs(tq[k] - np.floor(tq[k])) - 0.5) <= room), "a code differs away from a rounding tie"
+            flips += 1
+        print(f"free-running: {coords.shape[0]} coordinates, {int(far.sum())} beyond 1e-5 ({100 * far.mean():.2f} %), "
+              f"{flips} with a first code flip (all by one step at a tie), max |d| = {np.abs(got - ref).max():.2e}")
+    finally:
+        dhq.dhq_destroy(h)

@@ -1,0 +1,59 @@
+"""dhq_export / dhq_import: a prepared, calibrated handle as bytes and back, bit-identical."""
+import numpy as np
+import pytest
+import torch
+
+import dhq_inputs
+from tests.gpu_util import to_dev
+
+dhq = pytest.importorskip("paper_2508_13478_b200")
+
+
+def test_import_rejects_blocks_that_are_not_an_export():
+    # header checks come before any CUDA call: runs without a GPU
+    from paper_2508_13478_b200 import build
+    build.build()
+    for blob in (b"", b"x" * 64, b"DHQB200\0" + b"\0" * 4000):
+        with pytest.raises(dhq.DhqError) as e:
+            dhq.dhq_import(blob)
+        assert e.value.code == 1
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", ["C1", "C3", "C5"])
+def test_export_import_round_trip_is_bit_identical(name):
+    from paper_2508_13478_b200 import build
+    build.build()
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h = dhq.dhq_prepare(w.dims, [to_dev(x) for x in weights], [to_dev(x) for x in biases], w.omega0,
+                        w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    h2 = None
+    try:
+        coords = to_dev(w.coords()[: 40000])
+        dhq.dhq_calibrate(h, coords)
+        blob = dhq.dhq_export(h)
+        h2 = dhq.dhq_import(blob)
+        for l in range(1, len(w.dims)):
+            a, b = dhq.dhq_get_layer(h, l), dhq.dhq_get_layer(h2, l)
+            assert np.array_equal(a[0], b[0]) and np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
+            assert np.float32(a[2]).view(np.uint32) == np.float32(b[2]).view(np.uint32)
+        out1 = torch.empty((coords.shape[0], w.dims[-1]), device="cuda")
+        out2 = torch.full_like(out1, float("nan"))
+        dhq.dhq_forward(h, coords, out1)
+        dhq.dhq_forward(h2, coords, out2)        # no calibration happens here: the frozen scales came with the block
+        torch.cuda.synchronize()
+        assert dhq.dhq_last_status(h2) == 0
+        assert torch.equal(out1.view(torch.int32), out2.view(torch.int32))
+        assert dhq.dhq_export(h2) == blob         # exporting the import gives the same bytes
+        bad = bytearray(blob)
+        bad[len(bad) // 2] ^= 0x40                # one flipped bit in the arrays: checksum
+        with pytest.raises(dhq.DhqError) as e:
+            dhq.dhq_import(bytes(bad))
+        assert e.value.code == 1
+        with pytest.raises(dhq.DhqError):
+            dhq.dhq_import(blob[: len(blob) - 100])   # truncated
+    finally:
+        dhq.dhq_destroy(h)
+        if h2:
+            dhq.dhq_destroy(h2)

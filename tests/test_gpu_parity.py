@@ -75,7 +75,7 @@ def test_c3_c4_c5_sampled_tokens(name, count):
     _p1(w, np.ascontiguousarray(coords[idx]))
 
 
-@pytest.mark.parametrize("name", ["C3", "C4-W4A4", "C5"])
+@pytest.mark.parametrize("name", ["C3", "C4-W4A4", "C4-W6A6", "C5"])
 def test_full_size_launch_on_sampled_outputs(name):
     # The launch bench.py times: the whole grid of the workload in one dhq_forward call.  The
     # oracle cannot run millions of tokens, so 3,000 tokens sampled over the grid are checked: the
@@ -250,28 +250,6 @@ def test_forward_auto_calibrates_and_is_deterministic_and_batch_independent():
         for l in range(1, 5):
             a = dhq.dhq_get_layer(h, l)[2]
             assert abs(a - frozen[l - 1]) <= 2e-5 * max(1.0, abs(frozen[l - 1]))
-    finally:
-        dhq.dhq_destroy(h)
-
-
-def test_free_running_end_to_end_report():
-    # Reported, loosely gated: oracle on its own chain and calibration.  A code flipped at a
-    # near-tie moves one accumulator by one weight code, so a small fraction of coordinates may
-    # differ by more than 1e-5; all stay far below one quantization step of the output.
-    w = dhq_inputs.WORKLOADS["C2"]
-    weights, biases = w.network()
-    coords = w.coords()[:: 16]
-    h, net = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 0, 0)
-    try:
-        out = torch.empty((coords.shape[0], 3), device="cuda")
-        dhq.dhq_forward(h, to_dev(coords), out)
-        torch.cuda.synchronize()
-        orc.calibrate(net, coords)
-        ref = orc.forward(net, coords)
-        d = np.abs(out.cpu().numpy().astype(np.float64) - ref)
-        frac = float((d.max(axis=1) > TOL_Y).mean())
-        print(f"free-running: max |d| = {d.max():.3e}, fraction of coordinates beyond 1e-5 = {frac:.4f}")
-        assert frac < 0.25 and d.max() < 5e-2
     finally:
         dhq.dhq_destroy(h)
 

@@ -1,5 +1,7 @@
-"""The N > 1 bookkeeping of bench.py on CPU: two gloo ranks, replicas of the same grid, the
-slowest rank defines the step time and the aggregate is N times one replica's coordinates."""
+"""The N > 1 bookkeeping of bench.py on CPU: two gloo ranks.  Replicas of the same grid: the
+slowest rank defines the step time and the aggregate is N times one replica's coordinates.  One
+grid split over the ranks (--shard): the blocks are disjoint and complete, the aggregate is the one
+grid over the slowest rank's time, and the per-layer maxima are exchanged by all-reduce."""
 import os
 import socket
 import sys
@@ -30,11 +32,18 @@ def _rank_main(rank, world, port, out):
     coords = w.coords()                                   # every rank builds the same replica
     mine = [10.0 + 5.0 * rank, 20.0 - 3.0 * rank]          # per-rank timings (ms)
     total_ms, e2e_ms = bench.max_over_ranks(mine, world, "cpu")
-    value = bench.aggregate_throughput(coords.shape[0], world, total_ms / 4)
+    value = bench.aggregate_throughput(coords.shape[0] * world, total_ms / 4)
     checksum = torch.tensor([float(coords.sum())], dtype=torch.float64)
     both = [torch.zeros_like(checksum) for _ in range(world)]
     dist.all_gather(both, checksum)
-    out.put((rank, total_ms, e2e_ms, value, [float(b) for b in both]))
+    # the sharded mode: this rank's block of the one grid
+    from paper_2508_13478_b200.sharded import shard_range
+    lo, hi = shard_range(coords.shape[0], rank, world)
+    block = torch.tensor([float(hi - lo), float(coords[lo:hi].sum())], dtype=torch.float64)
+    dist.all_reduce(block)
+    sharded_value = bench.aggregate_throughput(coords.shape[0], total_ms / 4)
+    out.put((rank, total_ms, e2e_ms, value, [float(b) for b in both], (lo, hi), [float(v) for v in block], sharded_value,
+             float(coords.sum())))
     dist.destroy_process_group()
 
 
@@ -49,10 +58,13 @@ def test_two_gloo_ranks_take_the_slowest_time_and_sum_the_replicas():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    for rank, total_ms, e2e_ms, value, sums in results:
+    for rank, total_ms, e2e_ms, value, sums, block, reduced, sharded_value, whole_sum in results:
         assert total_ms == 15.0 and e2e_ms == 20.0            # max over ranks, element-wise
         assert value == 4096 * 2 / (15.0 / 4 * 1e-3)          # two replicas of 4,096 coordinates
         assert sums[0] == sums[1]                             # identical seeded inputs on both ranks
+        assert block == (rank * 2048, (rank + 1) * 2048)      # --shard: contiguous halves of the one grid
+        assert reduced[0] == 4096.0 and abs(reduced[1] - whole_sum) < 1e-6   # together they are the grid, once
+        assert sharded_value == 4096 / (15.0 / 4 * 1e-3)      # strong scaling: one grid over the slowest rank's time
 
 
 class _FakeApi:

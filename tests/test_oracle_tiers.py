@@ -160,3 +160,30 @@ def test_nlogn_forward_equals_definition_forward():
     net = orc.prepare(weights, biases, w.dims, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
     coords = w.coords()[1000:1200]
     assert np.array_equal(orc.forward(net, coords).view(np.uint64), orcn.forward(net, coords).view(np.uint64))
+
+
+# ---------------------------------------------------------------- absmax without a finite scale
+
+def test_absmax_whose_reciprocal_scale_overflows_counts_as_zero():
+    # Reading of the quantizer's degenerate end: qmax / a must be a finite fp32 number.  4-wide brute
+    # force: below the threshold every code is zero and the layer returns its bias term; above it
+    # the absmax element maps to +-qmax as usual.
+    for bits in (4, 8):
+        qmax = 2 ** (bits - 1) - 1
+        fmax = float(np.finfo(np.float32).max)
+        below = np.float32(qmax / fmax * 0.9)
+        above = np.float32(qmax / fmax * 1.2)
+        assert orc.scales(float(below), bits) == (0.0, 0.0)
+        s, inv = orc.scales(float(above), bits)
+        assert s > 0 and np.isfinite(inv) and inv == np.float32(qmax) / above
+        v = np.array([above, -above / 2, 0.0, above / 4], np.float32)
+        assert orc.quantize(v, inv, bits)[0] == qmax
+    W2 = np.eye(4, dtype=np.float32)
+    b2 = np.array([0.5, -0.25, 0.0, 1.0], np.float32)
+    net = orc.prepare([np.zeros((4, 2), np.float32), W2], [np.zeros(4, np.float32), b2], (2, 4, 4), 30.0, a_gran=1, rotate=False)
+    X = np.array([[1e-39, -1e-39, 0, 5e-40], [2e-38, 0, 0, 0], [1e-36, -5e-37, 0, 0]], np.float32)
+    r = orc.layer(net, 2, X)
+    assert not r["codes"][:2].any() and not r["s_x"][:2].any() and not r["acc"][:2].any()
+    assert np.array_equal(r["Y"][:2], np.tile(b2.astype(np.float64), (2, 1)))
+    assert r["codes"][2].tolist() == [127, -64, 0, 0] or r["codes"][2].tolist() == [127, -63, 0, 0]
+    assert np.array_equal(orcn.layer(net, 2, X)["codes"], r["codes"])

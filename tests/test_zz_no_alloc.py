@@ -24,7 +24,7 @@ def _dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-@pytest.mark.parametrize("name,a_gran", [("C2", 0), ("C3", 1)])
+@pytest.mark.parametrize("name,a_gran", [("C2", 0), ("C3", 1), ("C5", 0)])
 def test_static_scratch_forward_matches_forward_twice_in_a_row(name, a_gran):
     from paper_2508_13478_b200 import build
     build.build()
@@ -36,14 +36,24 @@ def test_static_scratch_forward_matches_forward_twice_in_a_row(name, a_gran):
     try:
         if a_gran == 0:
             dhq.dhq_calibrate(h, _dev(grid[::8]))          # the allocating part happens up front
-        batches = [grid[: dhq.DHQ_STATIC_MAX_TOKENS], grid[5000:5000 + 1237]]
-        for coords in batches:                              # two calls in a row, same scratch
+        # the largest batch the scratch holds (at width 512 this fills both halves of the array to
+        # their last float), then a ragged one, then a small one
+        batches = [grid[: dhq.DHQ_STATIC_MAX_TOKENS], grid[7000:7000 + dhq.DHQ_STATIC_MAX_TOKENS - 1], grid[5000:5000 + 1237]]
+        # The documented set-up: the first call on a device looks up the array's address, which is
+        # also when the driver brings the library image with its 16 MiB array onto the GPU.
+        warm = _dev(grid[:8])
+        dhq.dhq_forward_static_scratch(h, warm, torch.empty((8, w.dims[-1]), device="cuda"))
+        torch.cuda.synchronize()
+        for coords in batches:                              # calls in a row, same scratch
             cd = _dev(coords)
             want = torch.empty((coords.shape[0], w.dims[-1]), device="cuda")
             got = torch.full_like(want, float("nan"))
             dhq.dhq_forward(h, cd, want)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]      # the driver's own count of free device memory
             dhq.dhq_forward_static_scratch(h, cd, got)
             torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
             assert dhq.dhq_last_status(h) == 0
             assert torch.isfinite(got).all()
             assert (got - want).abs().max().item() <= TOL
