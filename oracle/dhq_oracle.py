@@ -257,3 +257,23 @@ def forward(net: OracleNet, coords, return_layers=False):
             X = r["Y"].astype(np.float32)
     out = r["Y"][:, : net.dims[-1]]
     return (out, per) if return_layers else out
+
+
+def forward_w8a32(net: OracleNet, coords, chain_fp32=True, return_layers=False):
+    """Weight-only quantized forward (W8A32): the weights of `net` (folded and quantized exactly as
+    for DHQ), activations not quantized.  Each layer is odef.w8a32_layer in fp64; between layers
+    the activation is rounded to fp32 (chain_fp32), as a datapath with fp32 activations holds it."""
+    from . import odef
+    X = odef.pad_first_input(coords)
+    if chain_fp32:
+        X = X.astype(np.float32).astype(np.float64)
+    per = []
+    L = len(net.layers)
+    for l, lay in enumerate(net.layers, start=1):
+        Y = odef.w8a32_layer(lay.qw, lay.s_w, lay.b_pad, X, net.rotate == 1, net.omega0, lay.sine)
+        per.append({"X": X.astype(np.float32), "Y": Y})
+        if l < L:
+            X = Y.astype(np.float32).astype(np.float64) if chain_fp32 else Y
+    out = Y[:, : net.dims[-1]]
+    return (out, per) if return_layers else out
+

@@ -80,3 +80,24 @@ def dhq_layer_def(W, b, X, w_bits: int, a_bits: int, per_channel: bool, per_toke
     z = s_w[None, :] * s_x * acc + np.asarray(b, dtype=np.float64)[None, :]
     return {"qw": qw, "tw": tw, "codes": codes, "t": t, "acc": acc, "Y": np.sin(omega0 * z) if sine else z,
             "a_x": a_x[:, 0]}
+
+
+def w8a32_layer(qw, s_w, b, X, rotate: bool, omega0: float, sine: bool) -> np.ndarray:
+    """One layer of the weight-only quantized network (the W8A32 datapath of Section I / Table 2):
+    quantized weights q_w with scales s_w (from the same weight-side fold and quantizer as DHQ),
+    activations left in floating point.  x~ = H_K x (or x itself without the rotation), exactly, in
+    fp64; z = s_w[m] * sum_k q_w[m][k] x~_k + b[m]; sin(omega0 z) for hidden layers.
+    qw [M][K] integers, s_w [M], b [M], X [n][K]."""
+    X = np.asarray(X, dtype=np.float64)
+    K = X.shape[1]
+    Xr = X @ hadamard(K).T if rotate else X
+    z = (Xr @ np.asarray(qw, dtype=np.float64).T) * np.asarray(s_w, dtype=np.float64)[None, :] + np.asarray(b, dtype=np.float64)[None, :]
+    return np.sin(omega0 * z) if sine else z
+
+
+def pad_first_input(coords: np.ndarray) -> np.ndarray:
+    """[x, y] -> [x, y, 0, 0]: the first layer's input padded to the Hadamard size 4."""
+    c = np.asarray(coords, dtype=np.float64)
+    X = np.zeros((c.shape[0], 4))
+    X[:, : c.shape[1]] = c
+    return X

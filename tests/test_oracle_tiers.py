@@ -187,3 +187,42 @@ def test_absmax_whose_reciprocal_scale_overflows_counts_as_zero():
     assert np.array_equal(r["Y"][:2], np.tile(b2.astype(np.float64), (2, 1)))
     assert r["codes"][2].tolist() == [127, -64, 0, 0] or r["codes"][2].tolist() == [127, -63, 0, 0]
     assert np.array_equal(orcn.layer(net, 2, X)["codes"], r["codes"])
+
+
+# ---------------------------------------------------------------- comparison datapaths: W8A32, W32A32
+
+def _w8a32_error(w_bits, rotate=True):
+    dims = (2, 64, 64, 3)
+    weights, biases = dhq_inputs.siren_init(dims, 30.0, 21)
+    coords = dhq_inputs.grid_coords(12, 12)
+    net = orc.prepare(weights, biases, dims, 30.0, w_bits=w_bits, a_bits=8, w_gran=1, a_gran=1, rotate=rotate)
+    got = orc.forward_w8a32(net, coords)
+    return np.abs(got - odef.siren_forward(weights, biases, 30.0, coords)).max(), got, net, coords
+
+
+def test_weight_only_quantized_network_converges_to_the_unquantized_siren():
+    # W8A32 (Section I, Fig. 1; Table 2's middle column): only the weights carry quantization error,
+    # so the distance to the fp64 SIREN shrinks with the weight bit-width alone
+    e8, g8, net8, coords = _w8a32_error(8)
+    e12, _, _, _ = _w8a32_error(12)
+    e16, g16, _, _ = _w8a32_error(16)
+    assert e12 < e8 / 4 and e16 < e12 / 4 and e16 < 1e-4
+    _, g16_plain, _, _ = _w8a32_error(16, rotate=False)
+    assert np.abs(g16 - g16_plain).max() < 1e-3                 # the rotation changes nothing in the limit
+    # and it is the a_bits -> infinity limit of the fully quantized network with the same weights
+    net_a16 = orc.prepare(*dhq_inputs.siren_init((2, 64, 64, 3), 30.0, 21), (2, 64, 64, 3), 30.0, w_bits=8, a_bits=16, w_gran=1, a_gran=1)
+    assert np.abs(orc.forward(net_a16, coords) - g8).max() < 2e-3
+    net_a8 = orc.prepare(*dhq_inputs.siren_init((2, 64, 64, 3), 30.0, 21), (2, 64, 64, 3), 30.0, w_bits=8, a_bits=8, w_gran=1, a_gran=1)
+    assert np.abs(orc.forward(net_a16, coords) - g8).max() < np.abs(orc.forward(net_a8, coords) - g8).max()
+
+
+def test_w8a32_layer_by_hand():
+    # 4-wide layer, rotation on: x = [1, 2, 3, 4] -> H_4 x = [10, -2, -4, 0]; q_w rows [1, 0, -1, 2] and
+    # [3, 3, 3, 3] with scales 0.5 and 0.25, biases 0.125 and -1:
+    #   z0 = 0.5 * (10 + 4 + 0) + 0.125 = 7.125 ;  z1 = 0.25 * 3 * (10 - 2 - 4 + 0) - 1 = 2.0
+    qw = np.array([[1, 0, -1, 2], [3, 3, 3, 3]])
+    z = odef.w8a32_layer(qw, [0.5, 0.25], [0.125, -1.0], np.array([[1.0, 2.0, 3.0, 4.0]]), True, 30.0, False)
+    assert z.tolist() == [[7.125, 2.0]]
+    y = odef.w8a32_layer(qw, [0.5, 0.25], [0.125, -1.0], np.array([[1.0, 2.0, 3.0, 4.0]]), False, 2.0, True)
+    # without the rotation: z0 = 0.5 * (1 - 3 + 8) + 0.125 = 3.125, z1 = 0.25 * 30 - 1 = 6.5
+    assert np.allclose(y, np.sin(2.0 * np.array([[3.125, 6.5]])), atol=1e-15)
