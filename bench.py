@@ -177,7 +177,7 @@ def config_of(workload, args, world):
     mode = "one grid split over the ranks" if args.shard else "independent replica(s)"
     return {"workload": workload.name, "dims": list(workload.dims), "coords_per_step": workload.n if args.limit_coords <= 0 else min(workload.n, args.limit_coords),
             "bits": [workload.w_bits, workload.a_bits], "w_gran": workload.w_gran, "a_gran": workload.a_gran,
-            "rotation": args.rotation, "l2": "flushed between steps (256 MB write)",
+            "rotation": args.rotation, "variant": args.variant, "l2": "flushed between steps (256 MB write)",
             "parallelism": f"{world} x {mode}"}
 
 
@@ -301,7 +301,10 @@ def roofline_of(workload, rotation, n, ms_per_step, sm_max_mhz, sampled_mhz, fma
     """ALU roofline of one launch: algorithmic lane-ops over the CUDA-event duration, against (a) the
     derived peak SMs x fp32 lanes x max SM clock, (b) the same at the SM clock sampled during the
     timed steps, (c) the FMA loop's rate measured in this run."""
-    achieved = alu_laneops_per_coord(workload.dims, rotations(rotation)) * n / (ms_per_step * 1e-3) / 1e12
+    laneops = alu_laneops_per_coord(workload.dims, rotations(rotation))
+    if workload.a_bits == 32:      # fp32 datapaths: one fused multiply-add per weight and coordinate on the CUDA cores
+        laneops = float(work_per_coord(workload.dims, rotations(rotation))[0])
+    achieved = laneops * n / (ms_per_step * 1e-3) / 1e12
     peak = SM_COUNT * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
     r = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tlaneop/s", "frac": achieved / peak,
          "peak_source": "148 SMs x 128 fp32 lanes x max SM clock (derived from unit counts and clock)"}
@@ -499,12 +502,20 @@ def main():
     ap.add_argument("--rotation", default="input", choices=["input", "none", "both"],
                     help="input = DHQ; none = the same path without the Hadamard rotation (uniform quantizer); "
                          "both = the two-sided transform of Eq. 4-5")
+    ap.add_argument("--variant", default="w8a8", choices=["w8a8", "w8a32", "w32a32"],
+                    help="datapath (Section I / Table 2 of the paper): the workload's fully quantized network, the same "
+                         "with fp32 activations, or the plain fp32 network")
     ap.add_argument("--limit-coords", type=int, default=0,
                     help="use only the first N coordinates of the workload's grid (profiling captures)")
     ap.add_argument("--sweep", action="store_true", help="batch-size sweep 2^12..2^24 instead of the timed steps")
     ap.add_argument("--sweep-reps", type=int, default=20)
     args = ap.parse_args()
     workload = dhq_inputs.WORKLOADS[args.workload]
+    if args.variant != "w8a8":
+        import dataclasses
+        workload = dataclasses.replace(workload, w_bits=32 if args.variant == "w32a32" else workload.w_bits, a_bits=32)
+        args.no_per_config = True
+        args.no_cpu_baseline = True
     if args.impl == "reference":
         run_reference(args, workload)
     elif args.sweep:

@@ -76,11 +76,26 @@ typedef enum { DHQ_GRAN_TENSOR = 0, DHQ_GRAN_CHANNEL_OR_TOKEN = 1 } dhq_gran_t;
  * memory between layers), not in the fused kernel; dhq_forward_static_scratch does not take it. */
 typedef enum { DHQ_ROT_INPUT = 0, DHQ_ROT_BOTH = 1, DHQ_ROT_NONE = 2 } dhq_rot_t;
 
+/* Bit-width value that means "not quantized, fp32": the comparison datapaths of the paper's
+ * motivation figure (Section I) and hardware table (Table 2).
+ *   w_bits 2..8, a_bits 2..8            the fully quantized network (W8A8 and the narrower sweeps)
+ *   w_bits 2..8, a_bits DHQ_BITS_FLOAT  W8A32: weights folded and quantized as above, activations
+ *                                       kept in fp32 (rotated in fp32 when rotation = DHQ_ROT_INPUT):
+ *                                       z = s_w sum_k q_w x~_k + b
+ *   both DHQ_BITS_FLOAT                 W32A32: the plain fp32 network, z = W x + b (rotation ignored)
+ * The two floating-point datapaths run one kernel pass per layer with fp32 multiply-adds on the
+ * CUDA cores (activations in device memory between layers).  They need no calibration; the
+ * calibration calls are no-ops for them.  dhq_forward_debug dumps only X and Y for them;
+ * dhq_forward_fused_debug, dhq_forward_static_scratch and DHQ_ROT_BOTH are UNSUPPORTED.
+ * Their layer outputs carry fp32 summation and phase rounding error: they are checked against the
+ * fp64 definition within 2e-5 per layer (measured: 5.6e-6), not 1e-5. */
+#define DHQ_BITS_FLOAT 32
+
 typedef struct {
     int n_layers;       /* L linear layers, 2..16                                          */
     const int *dims;    /* host, L+1 ints: 2, w, ..., w, d_L; w a power of two in 64..512, */
                         /* the same for all hidden layers; d_L in 1..4                     */
-    int w_bits, a_bits; /* 2..8                                                            */
+    int w_bits, a_bits; /* 2..8, or DHQ_BITS_FLOAT (see above)                             */
     float omega0;       /* sine frequency of layers 1..L-1                                 */
     dhq_gran_t w_gran;
     dhq_gran_t a_gran;

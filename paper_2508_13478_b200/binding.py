@@ -22,6 +22,7 @@ DHQ_ROT_INPUT = 0
 DHQ_ROT_BOTH = 1
 DHQ_ROT_NONE = 2
 DHQ_STATIC_MAX_TOKENS = 4096
+DHQ_BITS_FLOAT = 32
 
 PIPES = {"ffma": 0, "fadd": 1, "mufu_sin": 2, "i2f": 3, "f2i": 4, "prmt": 5, "fmnmx": 6, "tensor_i8": 7, "fadd2": 8, "ffma2": 9,
          "pass1": 10, "pass2": 11, "pass12": 12}

@@ -15,7 +15,8 @@ CSRC = os.path.join(_HERE, "csrc")
 OBJ_DIR = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libdhq_b200.so")
 SOURCES = ["dhq_api.cu", "dhq_prepare.cu", "dhq_layerwise.cu", "dhq_fused.cu", "dhq_fused_w64.cu",
-           "dhq_fused_w128.cu", "dhq_fused_w256.cu", "dhq_fused_w512.cu", "dhq_peaks.cu", "dhq_static.cu"]
+           "dhq_fused_w128.cu", "dhq_fused_w256.cu", "dhq_fused_w512.cu", "dhq_peaks.cu", "dhq_static.cu",
+           "dhq_float.cu"]
 ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]
 NVCC_FLAGS = [*ARCH_FLAGS, "-lineinfo", "-O3", "-std=c++17", "--fmad=false",
               "-Xcompiler", "-fPIC,-fvisibility=hidden"]

@@ -24,7 +24,7 @@ template <typename T> bool dev_alloc(T **p, size_t count)
 // Every device array of a prepared layer with its size in bytes, in a fixed order (allocation,
 // release, export and import all walk this table).  Needs d.K, d.M, d.Mt.
 struct ArrayRef { void **ptr; size_t bytes; };
-constexpr int kLayerArrays = 16;
+constexpr int kLayerArrays = 17;
 void layer_arrays(LayerDev &d, ArrayRef (&t)[kLayerArrays])
 {
     const size_t MK = (size_t)d.M * d.K, M = (size_t)d.M;
@@ -45,6 +45,7 @@ void layer_arrays(LayerDev &d, ArrayRef (&t)[kLayerArrays])
     t[i++] = {(void **)&d.fxQ, M * 4};
     t[i++] = {(void **)&d.fxB, M * 4};
     t[i++] = {(void **)&d.act, 16};
+    t[i++] = {(void **)&d.w_f32, d.has_f32 ? MK * 4 : 0};
 }
 
 bool alloc_layer(LayerDev &d)
@@ -83,13 +84,23 @@ dhq_status_t check_config(const dhq_config_t *cfg)
     if (cfg->dims[0] != 2 || w <= 0 || (w & (w - 1)) != 0 || w < 64 || w > 512 || d_L < 1 || d_L > 4) return DHQ_ERR_UNSUPPORTED;
     for (int l = 1; l < L; ++l)
         if (cfg->dims[l] != w) return DHQ_ERR_UNSUPPORTED;
-    if (cfg->w_bits < 2 || cfg->w_bits > 8 || cfg->a_bits < 2 || cfg->a_bits > 8) return DHQ_ERR_UNSUPPORTED;
+    const bool wq = cfg->w_bits >= 2 && cfg->w_bits <= 8, aq = cfg->a_bits >= 2 && cfg->a_bits <= 8;
+    const bool wf = cfg->w_bits == DHQ_BITS_FLOAT, af = cfg->a_bits == DHQ_BITS_FLOAT;
+    if (!((wq && aq) || (wq && af) || (wf && af))) return DHQ_ERR_UNSUPPORTED; // W8A8 family, W8A32 family, W32A32
     if (cfg->rotation != DHQ_ROT_INPUT && cfg->rotation != DHQ_ROT_NONE && cfg->rotation != DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
+    if (af && cfg->rotation == DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
     if ((cfg->w_gran != DHQ_GRAN_TENSOR && cfg->w_gran != DHQ_GRAN_CHANNEL_OR_TOKEN) ||
         (cfg->a_gran != DHQ_GRAN_TENSOR && cfg->a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN))
         return DHQ_ERR_INVALID_ARG;
     if (!(cfg->omega0 == cfg->omega0) || std::isinf(cfg->omega0)) return DHQ_ERR_INVALID_ARG;
     return DHQ_OK;
+}
+
+// Which datapath a configuration asks for: 0 fully quantized, 1 W8A32, 2 W32A32.
+int float_mode_of(const dhq_config_t &cfg)
+{
+    if (cfg.a_bits != DHQ_BITS_FLOAT) return 0;
+    return cfg.w_bits == DHQ_BITS_FLOAT ? 2 : 1;
 }
 
 // Serialized handle (dhq_export / dhq_import): this header, then every array of every layer in
@@ -204,10 +215,45 @@ dhq_status_t layerwise_forward(dhq_handle_s *h, const float *coords, int64_t n, 
     return DHQ_OK;
 }
 
+// W8A32 / W32A32: one pass of the floating-point layer kernel per layer, in chunks; X dumps optional.
+dhq_status_t float_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, const dhq_debug_bufs_t *bufs, cudaStream_t st)
+{
+    const int64_t chunk = n < kDebugChunk ? n : kDebugChunk;
+    dhq_status_t s = ensure_scratch(h, chunk);
+    if (s != DHQ_OK) return s;
+    for (int64_t t0 = 0; t0 < n; t0 += chunk) {
+        const int64_t cnt = n - t0 < chunk ? n - t0 : chunk;
+        const float *X = nullptr;
+        for (int l = 1; l <= h->L; ++l) {
+            const LayerDev &d = h->layer[l - 1];
+            FloatLayerArgs a;
+            memset(&a, 0, sizeof(a));
+            a.X = X; a.coords = coords + t0 * 2; a.n = cnt;
+            a.K = d.K; a.M = d.M; a.d_L = h->d_L;
+            a.w8 = h->float_mode == 1;
+            a.rotate = a.w8 && h->cfg.rotation == DHQ_ROT_INPUT;
+            a.qw_k4m = d.qw_k4m; a.w_f32 = reinterpret_cast<const float4 *>(d.w_f32);
+            a.s_w = d.s_w; a.bias = d.bias;
+            a.omega0 = h->cfg.omega0; a.sine = l < h->L;
+            a.Y = h->scratch[(l - 1) & 1];
+            if (l == h->L) a.out = out ? out + t0 * h->d_L : nullptr;
+            if (bufs) {
+                if (bufs->X && bufs->X[l - 1]) a.dX = bufs->X[l - 1] + t0 * d.K;
+                if (bufs->Y && bufs->Y[l - 1]) a.Y = bufs->Y[l - 1] + t0 * d.M;
+            }
+            CK(launch_float_layer(a, st));
+            h->launches++;
+            X = a.Y;
+        }
+    }
+    return DHQ_OK;
+}
+
 // The forward pass of a calibrated handle: the fused kernel, or, for the two-sided transform, the
 // layer-by-layer kernels.
 dhq_status_t run_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, bool on_host, cudaStream_t st)
 {
+    if (h->float_mode) return float_forward(h, coords, n, out, nullptr, st);
     if (h->cfg.rotation == DHQ_ROT_BOTH) return layerwise_forward(h, coords, n, out, st);
     return fused_forward(h, coords, n, out, on_host, st);
 }
@@ -275,8 +321,10 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     cudaStream_t st = (cudaStream_t)stream;
     dhq_status_t rc = DHQ_OK;
     float *d_bounds = nullptr;
-    const bool per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
     const bool both = cfg->rotation == DHQ_ROT_BOTH;
+    h->float_mode = float_mode_of(*cfg);
+    // the floating-point datapaths have no activation quantizer: nothing to calibrate
+    const bool per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN || h->float_mode != 0;
     do {
         if (cudaGetDevice(&h->device) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
         if (!dev_alloc(&h->d_status, 4) || !dev_alloc(&d_bounds, kMaxLayers)) { rc = DHQ_ERR_ALLOC; break; }
@@ -287,24 +335,29 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             set_layer_dims(d, l, L, w, cfg->dims);
             if (l == 1) d.epi_mode = per_token ? EPI_SINE_WIDE : EPI_SINE_FIXED; // coordinates are not bounded by the weights
             if (both) d.epi_mode = EPI_BOTH;
+            d.has_f32 = h->float_mode == 2;
             if (!alloc_layer(d)) { rc = DHQ_ERR_ALLOC; break; }
+            if (d.has_f32 && launch_prep_float_weights(W[l - 1], d.d_out, d.d_in, d.K, d.M, d.w_f32, st) != cudaSuccess) {
+                rc = DHQ_ERR_CUDA; break;
+            }
             if (cudaMemsetAsync(d.act, 0, 16, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
             PrepArgs a;
             memset(&a, 0, sizeof(a));
             a.W = W[l - 1]; a.b = b[l - 1];
             a.d_out = d.d_out; a.d_in = d.d_in; a.K = d.K; a.M = d.M; a.Mt = d.Mt;
-            a.bits = cfg->w_bits;
-            a.a_bits = cfg->a_bits;
+            // (a W32A32 handle still gets 8-bit codes of the unrotated weights; its forward does not read them)
+            a.bits = h->float_mode == 2 ? 8 : cfg->w_bits;
+            a.a_bits = h->float_mode ? 8 : cfg->a_bits;
             a.per_channel = cfg->w_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
             a.sine = l < L; a.first = l == 1;
             a.permute_rows = (l > 1 && l < L) ? 1 : 0;
-            a.rotate = cfg->rotation == DHQ_ROT_INPUT ? 1 : both ? 2 : 0;
+            a.rotate = h->float_mode == 2 ? 0 : cfg->rotation == DHQ_ROT_INPUT ? 1 : both ? 2 : 0;
             a.omega0 = (double)cfg->omega0;
             a.dev = d;
             a.phase_bound = d_bounds + (l - 1);
             if (launch_prepare(a, st, &h->launches) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
             if (per_token &&
-                launch_finalize(d, cfg->a_bits, 1, l < L, (double)cfg->omega0, st, &h->launches) != cudaSuccess) {
+                launch_finalize(d, h->float_mode ? 8 : cfg->a_bits, 1, l < L, (double)cfg->omega0, st, &h->launches) != cudaSuccess) {
                 rc = DHQ_ERR_CUDA; break;
             }
         }
@@ -321,7 +374,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit) ? EPI_SINE_FAST : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;
-        if (!both) rc = fused_create(h); // the two-sided transform runs layer by layer (no fused kernel yet)
+        if (!both && !h->float_mode) rc = fused_create(h); // the two-sided transform and the fp32 datapaths run layer by layer
     } while (0);
     cudaFree(d_bounds);
     if (rc != DHQ_OK) {
@@ -336,7 +389,7 @@ dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void 
 {
     if (!h || !coords || n < 1) return DHQ_ERR_INVALID_ARG;
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
+    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN || h->float_mode) return DHQ_OK;
     return calibrate_impl(h, coords, n, (cudaStream_t)stream);
 }
 
@@ -344,7 +397,7 @@ dhq_status_t dhq_calibrate_layer(dhq_handle_t h, int layer, const float *coords,
 {
     if (!h || layer < 1 || layer > h->L || n < 0 || (n > 0 && !coords)) return DHQ_ERR_INVALID_ARG;
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
+    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN || h->float_mode) return DHQ_OK;
     if (layer > h->calib_layers_done + 1) return DHQ_ERR_NOT_CALIBRATED; // layers before it are not frozen yet
     h->calibrated = false;
     h->calib_layers_done = layer - 1;
@@ -369,7 +422,7 @@ dhq_status_t dhq_set_act_absmax(dhq_handle_t h, int layer, float absmax, void *s
 {
     if (!h || layer < 1 || layer > h->L || !(absmax >= 0.0f) || std::isinf(absmax)) return DHQ_ERR_INVALID_ARG;
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN) return DHQ_OK;
+    if (h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN || h->float_mode) return DHQ_OK;
     if (layer > h->calib_layers_done + 1) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
     CK(cudaMemcpyAsync(h->layer[layer - 1].act, &absmax, sizeof(float), cudaMemcpyHostToDevice, st));
@@ -386,6 +439,7 @@ dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int64_t n, f
     if (!h || n < 0 || (n > 0 && !coords)) return DHQ_ERR_INVALID_ARG;
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
+    if (h->float_mode) return float_forward(h, coords, n, out, bufs, (cudaStream_t)stream); // X and Y dumps only
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t chunk = n < kDebugChunk ? n : kDebugChunk;
@@ -421,7 +475,7 @@ dhq_status_t dhq_forward_fused_debug(dhq_handle_t h, const float *coords, int64_
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.rotation == DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED; // runs layer by layer: dhq_forward_debug observes it
+    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode) return DHQ_ERR_UNSUPPORTED; // run layer by layer: dhq_forward_debug observes them
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
     DumpPtrs d;
@@ -462,7 +516,7 @@ dhq_status_t dhq_set_wait_limit(dhq_handle_t h, int64_t nanoseconds)
 dhq_status_t dhq_debug_stall_next_forward(dhq_handle_t h)
 {
     if (!h) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.rotation == DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
+    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode) return DHQ_ERR_UNSUPPORTED;
     h->stall_next_forward = true;
     return DHQ_OK;
 }
@@ -492,7 +546,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     // coordinates and writes the result through their device addresses, so the transfers happen
     // inside the kernel, tile by tile, beside the arithmetic.  (Calibration reads the coordinates
     // once per layer: it goes through the staged path below.)
-    if (h->calibrated && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
+    if (h->calibrated && !h->float_mode && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
         // one query per buffer: for page-locked memory it also gives the device alias (asked on every
         // call on purpose: an answer remembered per address could outlive the buffer it was given for)
         cudaPointerAttributes ai, ao;
@@ -517,7 +571,8 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     const int64_t round = fused_round_tokens(h);
     const int64_t rounds = (n + round - 1) / round;
     int chunks = (int)(rounds >= 16 ? 8 : rounds < 4 ? rounds : 4);
-    if (!h->calibrated) chunks = 1; // the first forward freezes the per-tensor scales on ALL of its coordinates
+    if (!h->calibrated || h->float_mode || h->cfg.rotation == DHQ_ROT_BOTH) chunks = 1; // the first forward freezes the per-tensor
+                                                                 // scales on ALL of its coordinates; the layer-by-layer paths are not cut
     if (chunks <= 1) {
         CK(cudaMemcpyAsync(h->stage_in, coords_host, (size_t)n * 2 * sizeof(float), cudaMemcpyHostToDevice, st));
         dhq_status_t s = dhq_forward(h, h->stage_in, n, h->stage_out, stream);
@@ -632,10 +687,12 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
     for (int i = 0; i <= hd.n_layers; ++i) h->dims[i] = dims[i];
     h->cfg.dims = h->dims;
     h->L = hd.n_layers; h->w = dims[1]; h->d_L = dims[hd.n_layers];
+    h->float_mode = float_mode_of(cfg);
     size_t payload = 0;
     for (int l = 1; l <= h->L; ++l) {
         LayerDev &d = h->layer[l - 1];
         set_layer_dims(d, l, h->L, h->w, dims);
+        d.has_f32 = h->float_mode == 2;
         ArrayRef t[kLayerArrays];
         layer_arrays(d, t);
         for (const ArrayRef &a : t) payload += a.bytes;
@@ -669,7 +726,7 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
         if (cudaStreamSynchronize(st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; } // host_buf may go after the call
         h->calibrated = hd.calibrated != 0;
         h->calib_layers_done = hd.calib_layers_done;
-        if (cfg.rotation != DHQ_ROT_BOTH) rc = fused_create(h);
+        if (cfg.rotation != DHQ_ROT_BOTH && !h->float_mode) rc = fused_create(h);
     } while (0);
     if (rc != DHQ_OK) {
         dhq_destroy(h);

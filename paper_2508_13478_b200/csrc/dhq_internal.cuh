@@ -30,6 +30,8 @@ struct LayerDev {
     float *cA = nullptr, *cA_lo = nullptr, *cB = nullptr; // [M] epilogue constants
     uint32_t *fxP = nullptr, *fxQ = nullptr, *fxB = nullptr; // [M] fixed-point phase constants (EPI_SINE_FIXED)
     float *act = nullptr;      // [4]: frozen absmax (max taken on the bit pattern), s_x, inv, unused
+    int has_f32 = 0;           // W32A32 handles keep the unquantized weights too
+    float *w_f32 = nullptr;    // [K/4][M] float4: fp32 weights, zero padded (has_f32 only)
 };
 
 } // namespace dhq
@@ -56,6 +58,7 @@ struct dhq_handle_s {
     void *fused = nullptr;          // state of the fused path (device parameter block)
     unsigned long long wait_limit_ns = 2000000000ull; // bound of every wait inside the fused kernel (dhq_set_wait_limit)
     bool stall_next_forward = false; // test hook: see dhq_debug_stall_next_forward
+    int float_mode = 0;             // 0: fully quantized (DHQ); 1: W8A32 (activations fp32); 2: W32A32 (plain fp32 network)
 };
 
 namespace dhq {
@@ -94,6 +97,26 @@ struct LayerArgs {
 };
 
 cudaError_t launch_layer(const LayerArgs &a, cudaStream_t st);
+
+// Arguments of one pass of the floating-point comparison datapaths (W8A32, W32A32).
+struct FloatLayerArgs {
+    const float *X;        // [n][K] layer input, or NULL for layer 1 (built from coords)
+    const float *coords;   // [n][2], layer 1 only
+    int64_t n;
+    int K, M, d_L;
+    int rotate;            // W8A32 with the Hadamard fold: rotate the layer input
+    int w8;                // 1: quantized weights (qw_k4m, s_w); 0: fp32 weights (w_f32)
+    const uint32_t *qw_k4m;
+    const float4 *w_f32;
+    const float *s_w, *bias;
+    float omega0;
+    int sine;
+    float *Y;              // [n][M] or NULL
+    float *out;            // [n][d_L] or NULL (last layer)
+    float *dX;             // dump of the layer input, or NULL
+};
+cudaError_t launch_float_layer(const FloatLayerArgs &a, cudaStream_t st);
+cudaError_t launch_prep_float_weights(const float *W, int d_out, int d_in, int K, int M, float *dst, cudaStream_t st);
 
 struct PrepArgs {
     const float *W, *b;
