@@ -15,6 +15,10 @@
  *     s = a/qmax and inv = qmax/a both as IEEE fp32 divisions, q = clamp(rint(fl32(v*inv))) with
  *     round-half-to-even, a = 0 giving s = inv = 0.
  *   - The output layer has no activation (Section III-C); hidden layers apply sin(omega0 * z).
+ *   - Section IV also evaluates WIRE, "featuring wavelet activation functions", without giving the
+ *     function.  Reading (gabor_s0 > 0): the real-valued Gabor wavelet of the WIRE paper,
+ *     psi(z) = sin(omega0 z) * exp(-(s0 z)^2); its complex form exp(j omega0 z - |s0 z|^2) is not
+ *     built.  gabor_s0 = 0 is the sine.
  *   - rotate = 2 is the two-sided transform of Eq. 4-5 taken literally: W~ = H_M W H_K / (K M)
  *     (rows rotated first, then columns, both as pinned fp32 pairwise sums, both scales exact
  *     powers of two), and since H_M H_M = M I the layer output is z = H_M d + b with
@@ -259,15 +263,23 @@ ORC_API void dhq_orc_rotated_absmax(const float *X, int64_t n, int K_pad, int ro
  *   a  = per-token absmax, or a_frozen     -> s_x   [n] fp32 (per-tensor: the same value)
  *   q  = quantize(x~)                      -> codes [n][K_pad]
  *   acc[m] = sum_k q[k] * qw[m][k]         -> acc   [n][M_pad] int64 (exact)
- *   z = s_w[m] * s_x * acc + b[m] in fp64; Y = sin(omega0 z) for hidden layers, z for the last
+ *   z = s_w[m] * s_x * acc + b[m] in fp64; Y = sin(omega0 z) (times exp(-(gabor_s0 z)^2) if gabor_s0 > 0)
+ *       for hidden layers, z for the last
  *                                          -> Y     [n][M_pad] fp64
  *   rotate = 2: z = H_M (s_w s_x acc) + b instead (fp64 matrix product)
  * Any output pointer may be NULL.  Returns 0, or -3 if an accumulator leaves the int32 range.
  */
+static double activation(double z, double omega0, double gabor_s0)
+{
+    double y = sin(omega0 * z);
+    if (gabor_s0 > 0.0) y *= exp(-(gabor_s0 * z) * (gabor_s0 * z));
+    return y;
+}
+
 ORC_API int dhq_orc_layer(const float *X, int64_t n, int K_pad, int M_pad, const int32_t *qw,
                           const float *s_w, const float *b_pad, int a_bits, int per_token,
                           float a_frozen, int apply_sine, double omega0, int rotate, float *Xrot,
-                          int32_t *codes, float *s_x, int64_t *acc, double *Y)
+                          int32_t *codes, float *s_x, int64_t *acc, double *Y, double gabor_s0)
 {
     int8_t *H = (int8_t *)malloc((size_t)K_pad * K_pad);
     int8_t *HM = (int8_t *)malloc((size_t)M_pad * M_pad);
@@ -308,7 +320,7 @@ ORC_API int dhq_orc_layer(const float *X, int64_t n, int K_pad, int M_pad, const
                     dq[m] = (double)s_w[m] * (double)s * (double)sum; /* still in the rotated output basis */
                 } else if (Y) {
                     double z = (double)s_w[m] * (double)s * (double)sum + (double)b_pad[m];
-                    Y[t * M_pad + m] = apply_sine ? sin(omega0 * z) : z;
+                    Y[t * M_pad + m] = apply_sine ? activation(z, omega0, gabor_s0) : z;
                 }
             }
             if (rotate == 2 && Y) {
@@ -318,7 +330,7 @@ ORC_API int dhq_orc_layer(const float *X, int64_t n, int K_pad, int M_pad, const
                     double z = 0.0;
                     for (int m = 0; m < M_pad; ++m) z += (hr[m] > 0) ? dq[m] : -dq[m];
                     z += (double)b_pad[j];
-                    Y[t * M_pad + j] = apply_sine ? sin(omega0 * z) : z;
+                    Y[t * M_pad + j] = apply_sine ? activation(z, omega0, gabor_s0) : z;
                 }
             }
         }

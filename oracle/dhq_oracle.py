@@ -52,7 +52,7 @@ def lib():
         L.dhq_orc_rotated_absmax.argtypes = [vp, c_i64, c_i, c_i, vp]
         L.dhq_orc_rotated_absmax.restype = None
         L.dhq_orc_layer.argtypes = [vp, c_i64, c_i, c_i, vp, vp, vp, c_i, c_i, c_f, c_i, c_d, c_i,
-                                    vp, vp, vp, vp, vp]
+                                    vp, vp, vp, vp, vp, c_d]
         L.dhq_orc_layer.restype = c_i
         _lib = L
     return _lib
@@ -144,6 +144,7 @@ class OracleNet:
     a_gran: int
     rotate: int           # 0: none, 1: input side (the hot path), 2: both sides (Eq. 4-5 literally)
     layers: list
+    gabor_s0: float = 0.0  # > 0: hidden layers use the real Gabor wavelet sin(omega0 z) exp(-(s0 z)^2) (WIRE reading)
 
 
 def _rot_mode(rotate) -> int:
@@ -155,7 +156,7 @@ def _rot_mode(rotate) -> int:
     return int(bool(rotate))
 
 
-def prepare(weights, biases, dims, omega0, w_bits=8, a_bits=8, w_gran=0, a_gran=0, rotate=True) -> OracleNet:
+def prepare(weights, biases, dims, omega0, w_bits=8, a_bits=8, w_gran=0, a_gran=0, rotate=True, gabor_s0=0.0) -> OracleNet:
     """Weight-side fold and quantizer for every layer (Eq. 4-5: rotate=True the input-side factor,
     rotate="both" the two-sided transform, rotate=False none)."""
     mode = _rot_mode(rotate)
@@ -175,7 +176,7 @@ def prepare(weights, biases, dims, omega0, w_bits=8, a_bits=8, w_gran=0, a_gran=
         b_pad = np.zeros(M_pad, dtype=np.float32)
         b_pad[:d_out] = _f32(biases[l - 1])
         layers.append(OracleLayer(K_pad, M_pad, Wrot, qw, s_w, b_pad, sine=(l < L)))
-    return OracleNet(tuple(dims), float(omega0), w_bits, a_bits, int(w_gran), int(a_gran), mode, layers)
+    return OracleNet(tuple(dims), float(omega0), w_bits, a_bits, int(w_gran), int(a_gran), mode, layers, float(gabor_s0))
 
 
 def pad_coords(coords) -> np.ndarray:
@@ -219,7 +220,7 @@ def layer(net: OracleNet, l: int, X, want=("Xrot", "codes", "s_x", "acc", "Y"), 
     rc = lib().dhq_orc_layer(_p(X), n, lay.K_pad, lay.M_pad, _p(lay.qw), _p(lay.s_w), _p(lay.b_pad),
                              net.a_bits, per_token, ctypes.c_float(float(af)), int(lay.sine),
                              ctypes.c_double(net.omega0), int(net.rotate), _p(out["Xrot"]),
-                             _p(out["codes"]), _p(out["s_x"]), _p(out["acc"]), _p(out["Y"]))
+                             _p(out["codes"]), _p(out["s_x"]), _p(out["acc"]), _p(out["Y"]), ctypes.c_double(net.gabor_s0))
     if rc == -3 and max(net.a_bits, net.w_bits) <= 8:
         raise OverflowError("accumulator left the int32 range")
     if rc not in (0, -3):

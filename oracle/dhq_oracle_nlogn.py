@@ -51,6 +51,8 @@ def layer(net, l: int, X, want=("Xrot", "codes", "s_x", "acc", "Y"), a_frozen=No
         "acc": np.empty((n, lay.M_pad), np.int64) if "acc" in want else None,
         "Y": np.empty((n, lay.M_pad), np.float64) if "Y" in want else None,
     }
+    if net.gabor_s0 > 0:
+        raise NotImplementedError("the O(n log n) baseline covers the sine network only")
     per_token = int(net.a_gran == 1)
     af = 0.0 if per_token else (lay.a_frozen if a_frozen is None else a_frozen)
     if not np.isfinite(af):

@@ -33,14 +33,19 @@ def input_side_fold(W: np.ndarray) -> np.ndarray:
     return W.astype(np.float64) @ hadamard(K) / K
 
 
-def siren_forward(weights, biases, omega0: float, coords: np.ndarray) -> np.ndarray:
-    """Unquantized fp64 SIREN: sin(omega0 (W x + b)) per hidden layer, affine last layer
-    (Section III-C: the output layer has no activation)."""
+def gabor(z: np.ndarray, omega0: float, s0: float) -> np.ndarray:
+    """Real Gabor wavelet (the reading of the WIRE activation): sin(omega0 z) exp(-(s0 z)^2)."""
+    return np.sin(omega0 * z) * np.exp(-(s0 * z) ** 2)
+
+
+def siren_forward(weights, biases, omega0: float, coords: np.ndarray, gabor_s0: float = 0.0) -> np.ndarray:
+    """Unquantized fp64 network: sin(omega0 (W x + b)) per hidden layer (or the Gabor wavelet with
+    gabor_s0 > 0), affine last layer (Section III-C: the output layer has no activation)."""
     x = coords.astype(np.float64)
     L = len(weights)
     for l in range(L):
         z = x @ weights[l].astype(np.float64).T + biases[l].astype(np.float64)
-        x = np.sin(omega0 * z) if l < L - 1 else z
+        x = (gabor(z, omega0, gabor_s0) if gabor_s0 > 0 else np.sin(omega0 * z)) if l < L - 1 else z
     return x
 
 

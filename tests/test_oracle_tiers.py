@@ -226,3 +226,40 @@ def test_w8a32_layer_by_hand():
     y = odef.w8a32_layer(qw, [0.5, 0.25], [0.125, -1.0], np.array([[1.0, 2.0, 3.0, 4.0]]), False, 2.0, True)
     # without the rotation: z0 = 0.5 * (1 - 3 + 8) + 0.125 = 3.125, z1 = 0.25 * 30 - 1 = 6.5
     assert np.allclose(y, np.sin(2.0 * np.array([[3.125, 6.5]])), atol=1e-15)
+
+
+# ---------------------------------------------------------------- wavelet activation (WIRE reading)
+
+def test_gabor_activation_by_hand_and_its_limits():
+    # psi(z) = sin(omega0 z) exp(-(s0 z)^2): z = 0.1, omega0 = 10, s0 = 5 -> sin(1) exp(-0.25)
+    import math
+    assert abs(float(odef.gabor(np.array([0.1]), 10.0, 5.0)[0]) - math.sin(1.0) * math.exp(-0.25)) < 1e-16
+    z = np.linspace(-2, 2, 1001)
+    assert np.abs(odef.gabor(z, 30.0, 10.0)).max() <= 1.0                       # bounded like the sine
+    assert np.array_equal(odef.gabor(z, 30.0, 0.0), np.sin(30.0 * z))           # s0 = 0 is the sine
+    # the layer routine applies it to z = s_w s_x acc + b of hidden layers only
+    W2 = np.eye(4, dtype=np.float32) * 0.5
+    b2 = np.array([0.05, -0.02, 0.0, 0.1], np.float32)
+    for sine_layer in (True, False):
+        dims = (2, 4, 4, 4) if sine_layer else (2, 4, 4)
+        weights = [np.zeros((4, 2), np.float32), W2] + ([np.zeros((4, 4), np.float32)] if sine_layer else [])
+        biases = [np.zeros(4, np.float32), b2] + ([np.zeros(4, np.float32)] if sine_layer else [])
+        net = orc.prepare(weights, biases, dims, 30.0, a_gran=1, rotate=False, gabor_s0=7.0)
+        X = np.array([[0.25, -0.5, 1.0, 0.125]], np.float32)
+        r = orc.layer(net, 2, X)
+        z = net.layers[1].s_w.astype(np.float64) * float(r["s_x"][0]) * r["acc"][0] + b2.astype(np.float64)
+        want = odef.gabor(z, 30.0, 7.0) if sine_layer else z
+        assert np.allclose(r["Y"][0], want, rtol=0, atol=1e-15)
+
+
+def test_quantized_gabor_network_converges_to_the_unquantized_one():
+    dims = (2, 64, 64, 3)
+    weights, biases = dhq_inputs.siren_init(dims, 30.0, 33)
+    coords = dhq_inputs.grid_coords(12, 12)
+    want = odef.siren_forward(weights, biases, 30.0, coords, gabor_s0=6.0)
+    errs = []
+    for bits in (8, 12, 16):
+        net = orc.prepare(weights, biases, dims, 30.0, w_bits=bits, a_bits=bits, w_gran=1, a_gran=1, gabor_s0=6.0)
+        errs.append(np.abs(orc.forward(net, coords) - want).max())
+    assert errs[1] < errs[0] / 4 and errs[2] < errs[1] / 4 and errs[2] < 2e-4
+    assert np.abs(want - odef.siren_forward(weights, biases, 30.0, coords)).max() > 1e-2   # and it is not the sine network
