@@ -111,6 +111,36 @@ def grid_coords(height: int, width: int) -> np.ndarray:
     return np.ascontiguousarray(out.reshape(height * width, 2))
 
 
+def procedural_image(height: int, width: int, channels: int, seed: int) -> np.ndarray:
+    """Seeded synthetic target image, fp32 [height][width][channels] in [0, 1], standing in for the
+    photographs of the paper's quality experiments (Section IV: cameraman, Kodak, CT), which are not
+    available: a smooth background gradient, soft blobs, a few hard-edged discs and boxes (object
+    outlines), and a patch of fine oriented texture whose frequency sweeps (detail that a
+    sinusoidal network has to work for)."""
+    st = Stream(seed + 0x1A6E)
+    yy, xx = np.meshgrid(np.linspace(-1, 1, height), np.linspace(-1, 1, width), indexing="ij")
+    img = np.zeros((height, width, channels), dtype=np.float64)
+    for c in range(channels):
+        g = st.uniform_sym(2, 0.15)
+        plane = 0.45 + g[0] * yy + g[1] * xx
+        for _ in range(6):                                   # soft blobs
+            cy, cx, r, a = st.uniform_sym(1, 0.8)[0], st.uniform_sym(1, 0.8)[0], 0.1 + 0.3 * st.uniform(1)[0], st.uniform_sym(1, 0.25)[0]
+            plane += a * np.exp(-((yy - cy) ** 2 + (xx - cx) ** 2) / (2 * r * r))
+        for _ in range(4):                                   # hard-edged discs
+            cy, cx, r, a = st.uniform_sym(1, 0.7)[0], st.uniform_sym(1, 0.7)[0], 0.05 + 0.2 * st.uniform(1)[0], st.uniform_sym(1, 0.3)[0]
+            plane += a * (((yy - cy) ** 2 + (xx - cx) ** 2) < r * r)
+        for _ in range(3):                                   # boxes
+            cy, cx, hh, ww, a = (st.uniform_sym(1, 0.7)[0], st.uniform_sym(1, 0.7)[0], 0.05 + 0.25 * st.uniform(1)[0],
+                                 0.05 + 0.25 * st.uniform(1)[0], st.uniform_sym(1, 0.25)[0])
+            plane += a * ((np.abs(yy - cy) < hh) & (np.abs(xx - cx) < ww))
+        ang, f0, f1, amp = st.uniform(1)[0] * np.pi, 6 + 10 * st.uniform(1)[0], 10 + 20 * st.uniform(1)[0], 0.08 + 0.08 * st.uniform(1)[0]
+        u = np.cos(ang) * xx + np.sin(ang) * yy
+        window = np.exp(-((yy - 0.35) ** 2 + (xx + 0.3) ** 2) / (2 * 0.35 ** 2))
+        plane += amp * window * np.sin(np.pi * (f0 * u + 0.5 * (f1 - f0) * u * u))
+        img[:, :, c] = plane
+    return np.clip(img, 0.0, 1.0).astype(np.float32)
+
+
 def sweep_grid(k: int) -> np.ndarray:
     """Grid with 2**k points, 2**ceil(k/2) rows by 2**floor(k/2) columns (batch-size sweep)."""
     return grid_coords(1 << ((k + 1) // 2), 1 << (k // 2))

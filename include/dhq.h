@@ -91,6 +91,14 @@ typedef enum { DHQ_ROT_INPUT = 0, DHQ_ROT_BOTH = 1, DHQ_ROT_NONE = 2 } dhq_rot_t
  * fp64 definition within 2e-5 per layer (measured: 5.6e-6), not 1e-5. */
 #define DHQ_BITS_FLOAT 32
 
+/* Activation of layers 1..L-1.  DHQ_ACT_SINE: sin(omega0 z), the SIREN of the paper's method
+ * sections.  DHQ_ACT_GABOR: the real Gabor wavelet sin(omega0 z) exp(-(act_s0 z)^2), this
+ * library's reading of the "wavelet activation" of the WIRE experiments (Section IV; the paper
+ * gives no formula, the complex form of the WIRE paper is not built).  The wavelet runs layer by
+ * layer (one kernel pass per layer), not in the fused kernel; it needs omega0 != 0, and the
+ * floating-point datapaths, dhq_forward_fused_debug and dhq_forward_static_scratch do not take it. */
+typedef enum { DHQ_ACT_SINE = 0, DHQ_ACT_GABOR = 1 } dhq_act_t;
+
 typedef struct {
     int n_layers;       /* L linear layers, 2..16                                          */
     const int *dims;    /* host, L+1 ints: 2, w, ..., w, d_L; w a power of two in 64..512, */
@@ -100,6 +108,8 @@ typedef struct {
     dhq_gran_t w_gran;
     dhq_gran_t a_gran;
     dhq_rot_t rotation; /* DHQ_ROT_INPUT, DHQ_ROT_NONE or DHQ_ROT_BOTH                     */
+    dhq_act_t activation; /* DHQ_ACT_SINE or DHQ_ACT_GABOR                                 */
+    float act_s0;       /* width parameter of the Gabor wavelet (> 0); ignored for the sine */
 } dhq_config_t;
 
 /*

@@ -23,6 +23,8 @@ DHQ_ROT_BOTH = 1
 DHQ_ROT_NONE = 2
 DHQ_STATIC_MAX_TOKENS = 4096
 DHQ_BITS_FLOAT = 32
+DHQ_ACT_SINE = 0
+DHQ_ACT_GABOR = 1
 
 PIPES = {"ffma": 0, "fadd": 1, "mufu_sin": 2, "i2f": 3, "f2i": 4, "prmt": 5, "fmnmx": 6, "tensor_i8": 7, "fadd2": 8, "ffma2": 9,
          "pass1": 10, "pass2": 11, "pass12": 12}
@@ -37,7 +39,8 @@ class DhqError(RuntimeError):
 class _Config(ctypes.Structure):
     _fields_ = [("n_layers", ctypes.c_int), ("dims", ctypes.POINTER(ctypes.c_int)),
                 ("w_bits", ctypes.c_int), ("a_bits", ctypes.c_int), ("omega0", ctypes.c_float),
-                ("w_gran", ctypes.c_int), ("a_gran", ctypes.c_int), ("rotation", ctypes.c_int)]
+                ("w_gran", ctypes.c_int), ("a_gran", ctypes.c_int), ("rotation", ctypes.c_int),
+                ("activation", ctypes.c_int), ("act_s0", ctypes.c_float)]
 
 
 class _DebugBufs(ctypes.Structure):
@@ -122,12 +125,13 @@ def _dev_ptr(t, dtype, what):
 
 
 def dhq_prepare(dims, weights, biases, omega0=30.0, w_bits=8, a_bits=8, w_gran=DHQ_GRAN_TENSOR,
-                a_gran=DHQ_GRAN_TENSOR, rotation=DHQ_ROT_INPUT, stream=None):
+                a_gran=DHQ_GRAN_TENSOR, rotation=DHQ_ROT_INPUT, stream=None, activation=DHQ_ACT_SINE, act_s0=0.0):
     """dims: L+1 ints; weights[l]: CUDA fp32 [dims[l+1]][dims[l]]; biases[l]: CUDA fp32 [dims[l+1]].
     Returns the opaque handle (an integer address)."""
     L = len(dims) - 1
     dims_arr = (ctypes.c_int * (L + 1))(*[int(d) for d in dims])
-    cfg = _Config(L, dims_arr, int(w_bits), int(a_bits), float(omega0), int(w_gran), int(a_gran), int(rotation))
+    cfg = _Config(L, dims_arr, int(w_bits), int(a_bits), float(omega0), int(w_gran), int(a_gran), int(rotation),
+                  int(activation), float(act_s0))
     W = (ctypes.c_void_p * L)(*[_dev_ptr(w, torch.float32, "weights") for w in weights])
     B = (ctypes.c_void_p * L)(*[_dev_ptr(b, torch.float32, "biases") for b in biases])
     out = ctypes.c_void_p()

@@ -89,6 +89,11 @@ dhq_status_t check_config(const dhq_config_t *cfg)
     if (!((wq && aq) || (wq && af) || (wf && af))) return DHQ_ERR_UNSUPPORTED; // W8A8 family, W8A32 family, W32A32
     if (cfg->rotation != DHQ_ROT_INPUT && cfg->rotation != DHQ_ROT_NONE && cfg->rotation != DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
     if (af && cfg->rotation == DHQ_ROT_BOTH) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->activation != DHQ_ACT_SINE && cfg->activation != DHQ_ACT_GABOR) return DHQ_ERR_UNSUPPORTED;
+    if (cfg->activation == DHQ_ACT_GABOR) {
+        if (af) return DHQ_ERR_UNSUPPORTED;
+        if (!(cfg->act_s0 > 0.0f) || std::isinf(cfg->act_s0) || cfg->omega0 == 0.0f) return DHQ_ERR_INVALID_ARG;
+    }
     if ((cfg->w_gran != DHQ_GRAN_TENSOR && cfg->w_gran != DHQ_GRAN_CHANNEL_OR_TOKEN) ||
         (cfg->a_gran != DHQ_GRAN_TENSOR && cfg->a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN))
         return DHQ_ERR_INVALID_ARG;
@@ -109,14 +114,14 @@ struct BlobHeader {
     char magic[8];            // "DHQB200\0"
     uint32_t version, header_bytes;
     int32_t n_layers, dims[kMaxLayers + 1];
-    int32_t w_bits, a_bits, w_gran, a_gran, rotation;
-    float omega0;
+    int32_t w_bits, a_bits, w_gran, a_gran, rotation, activation;
+    float omega0, act_s0;
     int32_t calibrated, calib_layers_done;
     int32_t epi_mode[kMaxLayers];
     float phase_bound[kMaxLayers];
     uint64_t payload_bytes, payload_fnv1a;
 };
-constexpr uint32_t kBlobVersion = 1;
+constexpr uint32_t kBlobVersion = 2;
 const char kBlobMagic[8] = {'D', 'H', 'Q', 'B', '2', '0', '0', 0};
 
 uint64_t fnv1a(const uint8_t *p, size_t n)
@@ -153,6 +158,7 @@ LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X
     a.epi_mode = d.epi_mode;
     a.rotate = h->cfg.rotation == DHQ_ROT_INPUT ? 1 : h->cfg.rotation == DHQ_ROT_BOTH ? 2 : 0;
     a.s_w = d.s_w; a.bias = d.bias; a.omega0 = (double)h->cfg.omega0; a.sine = l < h->L;
+    a.gabor_s0 = h->gabor_s0;
     a.qw_k4m = d.qw_k4m; a.cA = d.cA; a.cA_lo = d.cA_lo; a.cB = d.cB; a.act = d.act;
     a.fxP = d.fxP; a.fxQ = d.fxQ; a.fxB = d.fxB;
     return a;
@@ -254,7 +260,7 @@ dhq_status_t float_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
 dhq_status_t run_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, bool on_host, cudaStream_t st)
 {
     if (h->float_mode) return float_forward(h, coords, n, out, nullptr, st);
-    if (h->cfg.rotation == DHQ_ROT_BOTH) return layerwise_forward(h, coords, n, out, st);
+    if (h->cfg.rotation == DHQ_ROT_BOTH || h->gabor_s0 > 0.0) return layerwise_forward(h, coords, n, out, st);
     return fused_forward(h, coords, n, out, on_host, st);
 }
 
@@ -323,6 +329,8 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     float *d_bounds = nullptr;
     const bool both = cfg->rotation == DHQ_ROT_BOTH;
     h->float_mode = float_mode_of(*cfg);
+    h->gabor_s0 = cfg->activation == DHQ_ACT_GABOR ? (double)cfg->act_s0 : 0.0;
+    const bool gabor = h->gabor_s0 > 0.0;
     // the floating-point datapaths have no activation quantizer: nothing to calibrate
     const bool per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN || h->float_mode != 0;
     do {
@@ -333,7 +341,8 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
         for (int l = 1; l <= L && rc == DHQ_OK; ++l) {
             LayerDev &d = h->layer[l - 1];
             set_layer_dims(d, l, L, w, cfg->dims);
-            if (l == 1) d.epi_mode = per_token ? EPI_SINE_WIDE : EPI_SINE_FIXED; // coordinates are not bounded by the weights
+            // coordinates are not bounded by the weights; the wavelet's envelope needs the unwrapped phase
+            if (l == 1) d.epi_mode = (per_token || gabor) ? EPI_SINE_WIDE : EPI_SINE_FIXED;
             if (both) d.epi_mode = EPI_BOTH;
             d.has_f32 = h->float_mode == 2;
             if (!alloc_layer(d)) { rc = DHQ_ERR_ALLOC; break; }
@@ -371,10 +380,10 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             if (both) d.epi_mode = EPI_BOTH;
             else if (l == L) d.epi_mode = EPI_LINEAR;
             else if (l == 1) {}
-            else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit) ? EPI_SINE_FAST : EPI_SINE_WIDE;
+            else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit && !gabor) ? EPI_SINE_FAST : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;
-        if (!both && !h->float_mode) rc = fused_create(h); // the two-sided transform and the fp32 datapaths run layer by layer
+        if (!both && !h->float_mode && !gabor) rc = fused_create(h); // the two-sided transform and the fp32 datapaths run layer by layer
     } while (0);
     cudaFree(d_bounds);
     if (rc != DHQ_OK) {
@@ -475,7 +484,7 @@ dhq_status_t dhq_forward_fused_debug(dhq_handle_t h, const float *coords, int64_
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode) return DHQ_ERR_UNSUPPORTED; // run layer by layer: dhq_forward_debug observes them
+    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode || h->gabor_s0 > 0.0) return DHQ_ERR_UNSUPPORTED; // run layer by layer: dhq_forward_debug observes them
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
     DumpPtrs d;
@@ -516,7 +525,7 @@ dhq_status_t dhq_set_wait_limit(dhq_handle_t h, int64_t nanoseconds)
 dhq_status_t dhq_debug_stall_next_forward(dhq_handle_t h)
 {
     if (!h) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode) return DHQ_ERR_UNSUPPORTED;
+    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode || h->gabor_s0 > 0.0) return DHQ_ERR_UNSUPPORTED;
     h->stall_next_forward = true;
     return DHQ_OK;
 }
@@ -546,7 +555,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     // coordinates and writes the result through their device addresses, so the transfers happen
     // inside the kernel, tile by tile, beside the arithmetic.  (Calibration reads the coordinates
     // once per layer: it goes through the staged path below.)
-    if (h->calibrated && !h->float_mode && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
+    if (h->calibrated && !h->float_mode && !(h->gabor_s0 > 0.0) && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
         // one query per buffer: for page-locked memory it also gives the device alias (asked on every
         // call on purpose: an answer remembered per address could outlive the buffer it was given for)
         cudaPointerAttributes ai, ao;
@@ -571,7 +580,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     const int64_t round = fused_round_tokens(h);
     const int64_t rounds = (n + round - 1) / round;
     int chunks = (int)(rounds >= 16 ? 8 : rounds < 4 ? rounds : 4);
-    if (!h->calibrated || h->float_mode || h->cfg.rotation == DHQ_ROT_BOTH) chunks = 1; // the first forward freezes the per-tensor
+    if (!h->calibrated || h->float_mode || h->cfg.rotation == DHQ_ROT_BOTH || h->gabor_s0 > 0.0) chunks = 1; // the first forward freezes the per-tensor
                                                                  // scales on ALL of its coordinates; the layer-by-layer paths are not cut
     if (chunks <= 1) {
         CK(cudaMemcpyAsync(h->stage_in, coords_host, (size_t)n * 2 * sizeof(float), cudaMemcpyHostToDevice, st));
@@ -652,6 +661,7 @@ dhq_status_t dhq_export(dhq_handle_t h, void *host_buf, int64_t capacity, int64_
     hd.w_bits = h->cfg.w_bits; hd.a_bits = h->cfg.a_bits;
     hd.w_gran = (int)h->cfg.w_gran; hd.a_gran = (int)h->cfg.a_gran; hd.rotation = (int)h->cfg.rotation;
     hd.omega0 = h->cfg.omega0;
+    hd.activation = (int)h->cfg.activation; hd.act_s0 = h->cfg.act_s0;
     hd.calibrated = h->calibrated ? 1 : 0;
     hd.calib_layers_done = h->calib_layers_done;
     for (int l = 0; l < h->L; ++l) {
@@ -679,6 +689,7 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
     cfg.n_layers = hd.n_layers; cfg.dims = dims;
     cfg.w_bits = hd.w_bits; cfg.a_bits = hd.a_bits; cfg.omega0 = hd.omega0;
     cfg.w_gran = (dhq_gran_t)hd.w_gran; cfg.a_gran = (dhq_gran_t)hd.a_gran; cfg.rotation = (dhq_rot_t)hd.rotation;
+    cfg.activation = (dhq_act_t)hd.activation; cfg.act_s0 = hd.act_s0;
     dhq_status_t cs = check_config(&cfg);
     if (cs != DHQ_OK) return cs == DHQ_ERR_UNSUPPORTED ? DHQ_ERR_UNSUPPORTED : DHQ_ERR_INVALID_ARG;
     dhq_handle_s *h = new (std::nothrow) dhq_handle_s();
@@ -688,6 +699,7 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
     h->cfg.dims = h->dims;
     h->L = hd.n_layers; h->w = dims[1]; h->d_L = dims[hd.n_layers];
     h->float_mode = float_mode_of(cfg);
+    h->gabor_s0 = cfg.activation == DHQ_ACT_GABOR ? (double)cfg.act_s0 : 0.0;
     size_t payload = 0;
     for (int l = 1; l <= h->L; ++l) {
         LayerDev &d = h->layer[l - 1];
@@ -726,7 +738,7 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
         if (cudaStreamSynchronize(st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; } // host_buf may go after the call
         h->calibrated = hd.calibrated != 0;
         h->calib_layers_done = hd.calib_layers_done;
-        if (cfg.rotation != DHQ_ROT_BOTH && !h->float_mode) rc = fused_create(h);
+        if (cfg.rotation != DHQ_ROT_BOTH && !h->float_mode && !(h->gabor_s0 > 0.0)) rc = fused_create(h);
     } while (0);
     if (rc != DHQ_OK) {
         dhq_destroy(h);

@@ -58,6 +58,7 @@ struct dhq_handle_s {
     void *fused = nullptr;          // state of the fused path (device parameter block)
     unsigned long long wait_limit_ns = 2000000000ull; // bound of every wait inside the fused kernel (dhq_set_wait_limit)
     bool stall_next_forward = false; // test hook: see dhq_debug_stall_next_forward
+    double gabor_s0 = 0.0;          // > 0: wavelet activation (layer-by-layer path)
     int float_mode = 0;             // 0: fully quantized (DHQ); 1: W8A32 (activations fp32); 2: W32A32 (plain fp32 network)
 };
 
@@ -91,6 +92,7 @@ struct LayerArgs {
     const float *s_w, *bias;
     double omega0;
     int sine;
+    double gabor_s0;       // > 0: hidden layers apply sin(omega0 z) exp(-(s0 z)^2) instead of the sine
     float *Y;              // [n][M] or NULL
     float *out;            // [n][d_L] or NULL (last layer)
     float *dX; int8_t *dcodes; float *ds_x; int32_t *dacc; // dumps, may be NULL

@@ -113,6 +113,8 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
             float y;
             if (a.epi_mode == EPI_SINE_FIXED)
                 y = sine_fixed((int)cs[t * K + 0], (int)cs[t * K + 1], a.fxP[m], a.fxQ[m], a.fxB[m]);
+            else if (a.gabor_s0 > 0.0 && a.sine)
+                y = gabor_epilogue((float)acc[t], c_hi, c_lo, cB, (float)(a.gabor_s0 / a.omega0));
             else
                 y = epilogue(a.epi_mode, (float)acc[t], c_hi, c_lo, cB);
             if (a.dacc) a.dacc[tok * M + m] = acc[t];
@@ -147,6 +149,7 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
             double ph = a.omega0 * z;
             ph -= two_pi * rint(ph * (1.0 / two_pi));
             y = sin_approx((float)ph);
+            if (a.gabor_s0 > 0.0) y = __fmul_rn(y, (float)exp(-(a.gabor_s0 * z) * (a.gabor_s0 * z)));
         } else {
             y = (float)z;
         }

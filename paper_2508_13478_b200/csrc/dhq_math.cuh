@@ -83,6 +83,19 @@ __device__ __forceinline__ float epilogue(int mode, float accf, float c_hi, floa
     return __fmaf_rn(accf, c_hi, cb);
 }
 
+// Wavelet activation (reading of the paper's WIRE experiments, Section IV): the real Gabor wavelet
+// psi(z) = sin(omega0 z) exp(-(s0 z)^2), from the compensated phase x = omega0 z and c = s0 / omega0.
+// The envelope's exponent carries a relative error of a few 2^-24, the result stays within the
+// sine's own error.
+__device__ __forceinline__ float gabor_epilogue(float accf, float c_hi, float c_lo, float cb, float c)
+{
+    const float x = __fmaf_rn(accf, c_lo, __fmaf_rn(accf, c_hi, cb));
+    const float g = __fmul_rn(x, c);
+    float e;
+    asm("ex2.approx.f32 %0, %1;" : "=f"(e) : "f"(__fmul_rn(__fmul_rn(g, g), -1.4426950408889634f)));
+    return __fmul_rn(sin_wide(x), e);
+}
+
 // First layer, per-tensor activation scale.  The rotated padded coordinate [x, y, 0, 0] has the
 // codes [qs, qd, qs, qd], so acc[m] = qs * u_m + qd * v_m with u_m = q_w[m][0] + q_w[m][2],
 // v_m = q_w[m][1] + q_w[m][3].  With P = frac(c u_m / 2 pi), Q = frac(c v_m / 2 pi),

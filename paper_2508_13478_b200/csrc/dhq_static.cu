@@ -44,7 +44,7 @@ extern "C" dhq_status_t dhq_forward_static_scratch(dhq_handle_t h, const float *
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG; // the handle's buffers live on another GPU
     if (n > DHQ_STATIC_MAX_TOKENS) return DHQ_ERR_TOO_LARGE;
     if (n == 0) return DHQ_OK;
-    if (h->w > kMaxWidth || h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode) return DHQ_ERR_UNSUPPORTED;
+    if (h->w > kMaxWidth || h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode || h->gabor_s0 > 0.0) return DHQ_ERR_UNSUPPORTED;
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     float *scratch = nullptr;
     dhq_status_t s = scratch_for_current_device(&scratch);

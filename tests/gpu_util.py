@@ -13,10 +13,11 @@ def to_dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def prepare_pair(dims, weights, biases, omega0, w_bits, a_bits, w_gran, a_gran, rotate=True):
+def prepare_pair(dims, weights, biases, omega0, w_bits, a_bits, w_gran, a_gran, rotate=True, gabor_s0=0.0):
     h = dhq.dhq_prepare(dims, [to_dev(w) for w in weights], [to_dev(b) for b in biases], omega0,
-                        w_bits, a_bits, w_gran, a_gran, rotation=1 if rotate == "both" else 0 if rotate else 2)
-    net = orc.prepare(weights, biases, dims, omega0, w_bits, a_bits, w_gran, a_gran, rotate=rotate)
+                        w_bits, a_bits, w_gran, a_gran, rotation=1 if rotate == "both" else 0 if rotate else 2,
+                        activation=dhq.DHQ_ACT_GABOR if gabor_s0 > 0 else dhq.DHQ_ACT_SINE, act_s0=gabor_s0)
+    net = orc.prepare(weights, biases, dims, omega0, w_bits, a_bits, w_gran, a_gran, rotate=rotate, gabor_s0=gabor_s0)
     return h, net
 
 

@@ -170,6 +170,43 @@ def test_two_sided_transform_wide_phases_host_buffers_and_static_scratch():
         dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("name,count,rotate,s0", [("C1", 4096, True, 8.0), ("C2", 7000 + 3, True, 12.0), ("C3", 5000 + 1, True, 5.0),
+                                                  ("C4-W4A4", 3000 + 7, True, 10.0), ("C2", 4000, False, 12.0), ("C2", 4000, "both", 6.0),
+                                                  ("C5", 2000 + 5, True, 20.0)])
+def test_wavelet_activation_layer_by_layer(name, count, rotate, s0):
+    # DHQ_ACT_GABOR: sin(omega0 z) exp(-(s0 z)^2) on layers 1..L-1 (the reading of the WIRE experiments'
+    # activation); integer stages bit-exact, outputs within 1e-5 of the fp64 definition; dhq_forward and
+    # the host-buffer route give the same bits as the per-layer dumps
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    coords = w.coords()
+    coords = np.ascontiguousarray(coords[np.linspace(0, coords.shape[0] - 1, count).astype(np.int64)])
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran, rotate=rotate, gabor_s0=s0)
+    try:
+        check_weights(h, net)
+        cd = to_dev(coords)
+        if w.a_gran == 0:
+            dhq.dhq_calibrate(h, cd)
+        out_dbg, bufs = run_debug(h, net, cd)
+        worst = check_layers_against_oracle(h, net, coords, out_dbg, bufs)
+        out = torch.full_like(out_dbg, float("nan"))
+        dhq.dhq_forward(h, cd, out)
+        oh = torch.zeros(out.shape).pin_memory()
+        dhq.dhq_forward_host(h, torch.from_numpy(coords).pin_memory(), oh)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int32), out_dbg.view(torch.int32))
+        assert torch.equal(oh.view(torch.int32), out_dbg.cpu().view(torch.int32))
+        # the envelope is really applied: the hidden activations differ from the plain sine's
+        y1 = bufs["Y"][0].cpu().numpy()
+        assert np.abs(y1).max() <= 1.0 and np.abs(y1).mean() < 0.6
+        print(f"gabor {name} rotate={rotate}: outputs within {worst:.2e}")
+        with pytest.raises(dhq.DhqError) as e:
+            dhq.dhq_forward_fused_debug(h, cd, out)
+        assert e.value.code == 2
+    finally:
+        dhq.dhq_destroy(h)
+
+
 def test_trained_like_weights_and_wide_phases():
     # bell-shaped hidden weights, two-peaked last layer (Section III-A), and a first layer scaled up
     # so that phases reach hundreds of radians
