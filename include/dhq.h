@@ -71,9 +71,16 @@ typedef enum { DHQ_GRAN_TENSOR = 0, DHQ_GRAN_CHANNEL_OR_TOKEN = 1 } dhq_gran_t;
  * of weights and activations (the plain uniform quantizer the paper compares against, Section
  * IV-B) with everything else unchanged.  DHQ_ROT_BOTH is Eq. 4-5 taken literally, W~ = H_M W H_K /
  * (K M) (rows first, then columns, same fp32 butterfly order), with the layer output
- * z = H_M (s_w s_x acc) + b: the output-side rotation is undone in fp64 after dequantization
- * and before the bias.  It runs layer by layer (one kernel pass per layer, activations in device
- * memory between layers), not in the fused kernel; dhq_forward_static_scratch does not take it. */
+ * z = H_M (s_w s_x acc) + b: the output-side rotation is undone after the integer product and
+ * before the bias.  With one weight scale per tensor (w_gran = DHQ_GRAN_TENSOR) it runs inside
+ * the fused kernel: H_M is applied to the int32 accumulators, exactly (the library checks at
+ * prepare time that qmax_a * sum |q_w| < 2^31, so nothing can overflow), then the fp32 epilogue;
+ * about 1.6-1.7 times the time of DHQ_ROT_INPUT.  With per-output-channel weight scales the
+ * rotation has to act on the dequantized values; that case runs layer by layer (one kernel pass
+ * per layer, fp64 rotation), as does dhq_forward_debug for either.  Both routes are within 1e-5 of
+ * the definition; they are not bit-identical to each other (fp32 against fp64 epilogue), so for
+ * DHQ_ROT_BOTH dhq_forward and dhq_forward_debug need not agree bit for bit;
+ * dhq_forward_fused_debug observes the fused route.  dhq_forward_static_scratch does not take it. */
 typedef enum { DHQ_ROT_INPUT = 0, DHQ_ROT_BOTH = 1, DHQ_ROT_NONE = 2 } dhq_rot_t;
 
 /* Bit-width value that means "not quantized, fp32": the comparison datapaths of the paper's

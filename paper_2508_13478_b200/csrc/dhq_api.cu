@@ -24,7 +24,7 @@ template <typename T> bool dev_alloc(T **p, size_t count)
 // Every device array of a prepared layer with its size in bytes, in a fixed order (allocation,
 // release, export and import all walk this table).  Needs d.K, d.M, d.Mt.
 struct ArrayRef { void **ptr; size_t bytes; };
-constexpr int kLayerArrays = 17;
+constexpr int kLayerArrays = 19;
 void layer_arrays(LayerDev &d, ArrayRef (&t)[kLayerArrays])
 {
     const size_t MK = (size_t)d.M * d.K, M = (size_t)d.M;
@@ -46,6 +46,8 @@ void layer_arrays(LayerDev &d, ArrayRef (&t)[kLayerArrays])
     t[i++] = {(void **)&d.fxB, M * 4};
     t[i++] = {(void **)&d.act, 16};
     t[i++] = {(void **)&d.w_f32, d.has_f32 ? MK * 4 : 0};
+    t[i++] = {(void **)&d.l1U, d.has_uv ? M * 4 : 0};
+    t[i++] = {(void **)&d.l1V, d.has_uv ? M * 4 : 0};
 }
 
 bool alloc_layer(LayerDev &d)
@@ -116,12 +118,12 @@ struct BlobHeader {
     int32_t n_layers, dims[kMaxLayers + 1];
     int32_t w_bits, a_bits, w_gran, a_gran, rotation, activation;
     float omega0, act_s0;
-    int32_t calibrated, calib_layers_done;
+    int32_t calibrated, calib_layers_done, has_fused;
     int32_t epi_mode[kMaxLayers];
     float phase_bound[kMaxLayers];
     uint64_t payload_bytes, payload_fnv1a;
 };
-constexpr uint32_t kBlobVersion = 2;
+constexpr uint32_t kBlobVersion = 3;
 const char kBlobMagic[8] = {'D', 'H', 'Q', 'B', '2', '0', '0', 0};
 
 uint64_t fnv1a(const uint8_t *p, size_t n)
@@ -260,7 +262,7 @@ dhq_status_t float_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
 dhq_status_t run_forward(dhq_handle_s *h, const float *coords, int64_t n, float *out, bool on_host, cudaStream_t st)
 {
     if (h->float_mode) return float_forward(h, coords, n, out, nullptr, st);
-    if (h->cfg.rotation == DHQ_ROT_BOTH || h->gabor_s0 > 0.0) return layerwise_forward(h, coords, n, out, st);
+    if (!h->fused) return layerwise_forward(h, coords, n, out, st); // wavelet activation; two-sided transform with per-channel weight scales
     return fused_forward(h, coords, n, out, on_host, st);
 }
 
@@ -327,6 +329,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     cudaStream_t st = (cudaStream_t)stream;
     dhq_status_t rc = DHQ_OK;
     float *d_bounds = nullptr;
+    unsigned long long *d_sums = nullptr;
     const bool both = cfg->rotation == DHQ_ROT_BOTH;
     h->float_mode = float_mode_of(*cfg);
     h->gabor_s0 = cfg->activation == DHQ_ACT_GABOR ? (double)cfg->act_s0 : 0.0;
@@ -335,15 +338,16 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     const bool per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN || h->float_mode != 0;
     do {
         if (cudaGetDevice(&h->device) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
-        if (!dev_alloc(&h->d_status, 4) || !dev_alloc(&d_bounds, kMaxLayers)) { rc = DHQ_ERR_ALLOC; break; }
+        if (!dev_alloc(&h->d_status, 4) || !dev_alloc(&d_bounds, kMaxLayers) || !dev_alloc(&d_sums, kMaxLayers)) { rc = DHQ_ERR_ALLOC; break; }
         if (cudaMemsetAsync(h->d_status, 0, 16, st) != cudaSuccess ||
-            cudaMemsetAsync(d_bounds, 0, kMaxLayers * sizeof(float), st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+            cudaMemsetAsync(d_bounds, 0, kMaxLayers * sizeof(float), st) != cudaSuccess ||
+            cudaMemsetAsync(d_sums, 0, kMaxLayers * sizeof(unsigned long long), st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
         for (int l = 1; l <= L && rc == DHQ_OK; ++l) {
             LayerDev &d = h->layer[l - 1];
             set_layer_dims(d, l, L, w, cfg->dims);
             // coordinates are not bounded by the weights; the wavelet's envelope needs the unwrapped phase
             if (l == 1) d.epi_mode = (per_token || gabor) ? EPI_SINE_WIDE : EPI_SINE_FIXED;
-            if (both) d.epi_mode = EPI_BOTH;
+            d.has_uv = both && l == 1;
             d.has_f32 = h->float_mode == 2;
             if (!alloc_layer(d)) { rc = DHQ_ERR_ALLOC; break; }
             if (d.has_f32 && launch_prep_float_weights(W[l - 1], d.d_out, d.d_in, d.K, d.M, d.w_f32, st) != cudaSuccess) {
@@ -364,6 +368,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
             a.omega0 = (double)cfg->omega0;
             a.dev = d;
             a.phase_bound = d_bounds + (l - 1);
+            a.code_l1 = d_sums + (l - 1);
             if (launch_prepare(a, st, &h->launches) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
             if (per_token &&
                 launch_finalize(d, h->float_mode ? 8 : cfg->a_bits, 1, l < L, (double)cfg->omega0, st, &h->launches) != cudaSuccess) {
@@ -372,20 +377,28 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
         }
         if (rc != DHQ_OK) break;
         float bounds[kMaxLayers];
+        unsigned long long sums[kMaxLayers];
         if (cudaMemcpyAsync(bounds, d_bounds, sizeof(bounds), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaMemcpyAsync(sums, d_sums, sizeof(sums), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
             cudaStreamSynchronize(st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+        // Two-sided transform in the fused kernel: the output-side rotation runs on the int32 accumulators,
+        // which needs one weight scale per tensor and |H_M acc| <= sum_m |acc_m| <= qmax_a * sum |q_w| < 2^31.
+        bool both_fused = both && cfg->w_gran == DHQ_GRAN_TENSOR && !gabor && !h->float_mode;
+        for (int l = 1; l <= L && both_fused; ++l)
+            if (sums[l - 1] * (unsigned long long)((1 << (cfg->a_bits - 1)) - 1) >= (1ull << 31)) both_fused = false;
         for (int l = 1; l <= L; ++l) {
             LayerDev &d = h->layer[l - 1];
             d.phase_bound = bounds[l - 1];
-            if (both) d.epi_mode = EPI_BOTH;
-            else if (l == L) d.epi_mode = EPI_LINEAR;
+            if (l == L) d.epi_mode = EPI_LINEAR;
             else if (l == 1) {}
-            else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit && !gabor) ? EPI_SINE_FAST : EPI_SINE_WIDE;
+            // (two-sided: the quantization error of all M rows meets in every output; no tight phase bound)
+            else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit && !gabor && !both) ? EPI_SINE_FAST : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;
-        if (!both && !h->float_mode && !gabor) rc = fused_create(h); // the two-sided transform and the fp32 datapaths run layer by layer
+        if ((!both || both_fused) && !h->float_mode && !gabor) rc = fused_create(h); // the two-sided transform and the fp32 datapaths run layer by layer
     } while (0);
     cudaFree(d_bounds);
+    cudaFree(d_sums);
     if (rc != DHQ_OK) {
         dhq_destroy(h);
         return rc;
@@ -484,7 +497,7 @@ dhq_status_t dhq_forward_fused_debug(dhq_handle_t h, const float *coords, int64_
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode || h->gabor_s0 > 0.0) return DHQ_ERR_UNSUPPORTED; // run layer by layer: dhq_forward_debug observes them
+    if (!h->fused) return DHQ_ERR_UNSUPPORTED; // run layer by layer: dhq_forward_debug observes them
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
     DumpPtrs d;
@@ -525,7 +538,7 @@ dhq_status_t dhq_set_wait_limit(dhq_handle_t h, int64_t nanoseconds)
 dhq_status_t dhq_debug_stall_next_forward(dhq_handle_t h)
 {
     if (!h) return DHQ_ERR_INVALID_ARG;
-    if (h->cfg.rotation == DHQ_ROT_BOTH || h->float_mode || h->gabor_s0 > 0.0) return DHQ_ERR_UNSUPPORTED;
+    if (!h->fused) return DHQ_ERR_UNSUPPORTED;
     h->stall_next_forward = true;
     return DHQ_OK;
 }
@@ -555,7 +568,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     // coordinates and writes the result through their device addresses, so the transfers happen
     // inside the kernel, tile by tile, beside the arithmetic.  (Calibration reads the coordinates
     // once per layer: it goes through the staged path below.)
-    if (h->calibrated && !h->float_mode && !(h->gabor_s0 > 0.0) && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
+    if (h->calibrated && h->fused && !((uintptr_t)coords_host & 7) && !((uintptr_t)out_host & 3)) {
         // one query per buffer: for page-locked memory it also gives the device alias (asked on every
         // call on purpose: an answer remembered per address could outlive the buffer it was given for)
         cudaPointerAttributes ai, ao;
@@ -580,7 +593,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
     const int64_t round = fused_round_tokens(h);
     const int64_t rounds = (n + round - 1) / round;
     int chunks = (int)(rounds >= 16 ? 8 : rounds < 4 ? rounds : 4);
-    if (!h->calibrated || h->float_mode || h->cfg.rotation == DHQ_ROT_BOTH || h->gabor_s0 > 0.0) chunks = 1; // the first forward freezes the per-tensor
+    if (!h->calibrated || !h->fused) chunks = 1; // the first forward freezes the per-tensor
                                                                  // scales on ALL of its coordinates; the layer-by-layer paths are not cut
     if (chunks <= 1) {
         CK(cudaMemcpyAsync(h->stage_in, coords_host, (size_t)n * 2 * sizeof(float), cudaMemcpyHostToDevice, st));
@@ -664,6 +677,7 @@ dhq_status_t dhq_export(dhq_handle_t h, void *host_buf, int64_t capacity, int64_
     hd.activation = (int)h->cfg.activation; hd.act_s0 = h->cfg.act_s0;
     hd.calibrated = h->calibrated ? 1 : 0;
     hd.calib_layers_done = h->calib_layers_done;
+    hd.has_fused = h->fused ? 1 : 0;
     for (int l = 0; l < h->L; ++l) {
         hd.epi_mode[l] = h->layer[l].epi_mode;
         hd.phase_bound[l] = h->layer[l].phase_bound;
@@ -705,6 +719,7 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
         LayerDev &d = h->layer[l - 1];
         set_layer_dims(d, l, h->L, h->w, dims);
         d.has_f32 = h->float_mode == 2;
+        d.has_uv = cfg.rotation == DHQ_ROT_BOTH && l == 1;
         ArrayRef t[kLayerArrays];
         layer_arrays(d, t);
         for (const ArrayRef &a : t) payload += a.bytes;
@@ -738,7 +753,7 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
         if (cudaStreamSynchronize(st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; } // host_buf may go after the call
         h->calibrated = hd.calibrated != 0;
         h->calib_layers_done = hd.calib_layers_done;
-        if (cfg.rotation != DHQ_ROT_BOTH && !h->float_mode && !(h->gabor_s0 > 0.0)) rc = fused_create(h);
+        if (hd.has_fused) rc = fused_create(h);
     } while (0);
     if (rc != DHQ_OK) {
         dhq_destroy(h);

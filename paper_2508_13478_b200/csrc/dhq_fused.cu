@@ -19,6 +19,26 @@ static fused_fn pick_kernel(int W, bool per_token, bool rot, bool spread, bool a
     return nullptr;
 }
 
+static fused_fn pick_both_kernel(int W, bool per_token)
+{
+    switch (W) {
+    case 64: return fused_pick_both_64(per_token);
+    case 128: return fused_pick_both_128(per_token);
+    case 256: return fused_pick_both_256(per_token);
+    case 512: return fused_pick_both_512(per_token);
+    }
+    return nullptr;
+}
+static fused_dump_fn pick_both_dump_kernel(int W, bool per_token)
+{
+    switch (W) {
+    case 64: return fused_pick_both_dump_64(per_token);
+    case 128: return fused_pick_both_dump_128(per_token);
+    case 256: return fused_pick_both_dump_256(per_token);
+    case 512: return fused_pick_both_dump_512(per_token);
+    }
+    return nullptr;
+}
 static fused_dump_fn pick_dump_kernel(int W, bool per_token, bool rot)
 {
     switch (W) {
@@ -41,6 +61,7 @@ dhq_status_t fused_create(dhq_handle_s *h)
     p.per_token = h->cfg.a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
     p.qmaxf = (float)((1 << (h->cfg.a_bits - 1)) - 1);
     p.status = h->d_status;
+    const bool both = h->cfg.rotation == DHQ_ROT_BOTH;
     int words = 0;
     for (int l = 0; l < h->L; ++l) {
         const LayerDev &d = h->layer[l];
@@ -50,15 +71,16 @@ dhq_status_t fused_create(dhq_handle_s *h)
         f.cA = d.cA; f.cA_lo = d.cA_lo; f.cB = d.cB;
         f.fxP = d.fxP; f.fxQ = d.fxQ; f.fxB = d.fxB;
         f.act = d.act;
+        f.l1U = d.l1U; f.l1V = d.l1V;
         f.epi_mode = d.epi_mode;
         f.c_off = words;
         if (l < h->L - 1) {
-            int areas = (l == 0) ? (d.epi_mode == EPI_SINE_FIXED ? 3 : 4) : (d.epi_mode == EPI_SINE_WIDE ? 3 : 2);
+            int areas = (l == 0) ? (d.epi_mode == EPI_SINE_FIXED ? 3 : (both ? 5 : 4)) : (d.epi_mode == EPI_SINE_WIDE ? 3 : 2);
             words += areas * h->w;
         }
     }
     p.const_words = words;
-    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false, false);
+    fused_fn fn = both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false, false);
     if (!fn) return DHQ_ERR_UNSUPPORTED;
     int dev = 0, max_optin = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -81,11 +103,12 @@ dhq_status_t fused_create(dhq_handle_s *h)
     if (bytes < (size_t)kMinSmem) bytes = kMinSmem;
     fs->smem_bytes = bytes;
     for (int v = 0; v < 4; ++v) { // every variant of this handle's kernel
-        fused_fn f = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, (v & 1) != 0, (v & 2) != 0);
+        fused_fn f = both ? pick_both_kernel(h->w, p.per_token)
+                          : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, (v & 1) != 0, (v & 2) != 0);
         if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
-    fused_dump_fn fd = pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    fused_dump_fn fd = both ? pick_both_dump_kernel(h->w, p.per_token) : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     if (!fd || cudaFuncSetAttribute(fd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
         return DHQ_ERR_CUDA;
     return DHQ_OK;
@@ -126,8 +149,9 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
         h->stall_next_forward = false;
     }
     const int slots = (h->w == 512) ? 1 : 2;
-    const bool spread = slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
-    fused_fn fn = pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
+    const bool both = h->cfg.rotation == DHQ_ROT_BOTH;
+    const bool spread = !both && slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
+    fused_fn fn = both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
@@ -146,7 +170,8 @@ dhq_status_t fused_forward_dump(dhq_handle_s *h, const float *coords, int64_t n,
     fill_call(h, p, coords, n, out);
     p.d = d;
     const int slots = (h->w == 512) ? 1 : 2;
-    fused_dump_fn fn = pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    fused_dump_fn fn = h->cfg.rotation == DHQ_ROT_BOTH ? pick_both_dump_kernel(h->w, p.per_token)
+                                                        : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     const long long ctas = (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);

@@ -97,6 +97,7 @@ struct FusedLayer {
     const float *cA, *cA_lo, *cB;
     const uint32_t *fxP, *fxQ, *fxB;
     const float *act;
+    const int32_t *l1U, *l1V; // two-sided transform, layer 1: H_M applied to the two distinct weight-code sums
     int epi_mode;
     int c_off; // word offset of this layer's constants in the shared-memory constant area
 };
@@ -455,7 +456,7 @@ __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, 
 // Layer 1 for the CH columns starting at column m0.  Fixed-point mode: areas A = P, B = B, C = Q.
 // Float mode (per-token scales): A = cA, B = cB, C = cA_lo, D = the weight codes, one word per
 // column, and acc = dp4a(codes of the token, codes of the column's feature).
-template <int W, int CH, bool PER_TOKEN, bool ROT, bool DUMP = false>
+template <int W, int CH, bool PER_TOKEN, bool ROT, bool DUMP = false, bool BOTH = false>
 __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int qd, uint32_t qx, float s_x, uint32_t (&v)[CH],
                                              float *dump_y = nullptr)
 {
@@ -475,11 +476,17 @@ __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int
             } else {
                 const float4 wq = lds128(cbase + (3 * W + m0 + i) * 4);
                 const float wv[4] = {wq.x, wq.y, wq.z, wq.w};
+                float4 wq2 = make_float4(0.f, 0.f, 0.f, 0.f);
+                if constexpr (BOTH) wq2 = lds128(cbase + (4 * W + m0 + i) * 4);
+                const float wv2[4] = {wq2.x, wq2.y, wq2.z, wq2.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     float c_hi, c_lo;
                     token_const(Av[e], Cv[e], s_x, c_hi, c_lo);
-                    const int acc = __dp4a((int)qx, (int)__float_as_uint(wv[e]), 0);
+                    // two-sided transform: areas D, E hold U' = H_M u and V' = H_M v (u, v: the sums of the weight
+                    // codes that meet the two distinct input codes), so acc' = qs U' + qd V' needs no butterfly
+                    const int acc = BOTH ? qs * (int)__float_as_uint(wv[e]) + qd * (int)__float_as_uint(wv2[e])
+                                         : __dp4a((int)qx, (int)__float_as_uint(wv[e]), 0);
                     y[e] = epilogue(EPI_SINE_WIDE, (float)acc, c_hi, c_lo, Bv[e]);
                 }
             }
@@ -604,7 +611,77 @@ template <int W, int CH> __device__ __forceinline__ void dump_acc_chunk(int32_t 
     for (int i = 0; i < CH; ++i) arow[fused_feature(m0 + i, W)] = (int32_t)v[i];
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP>
+// Two-sided transform (Eq. 4-5 literally): the layer output is z = H_M (s_w s_x acc) + b.  With one
+// weight scale per tensor the rotation acts on the integers, acc' = H_M acc, exactly (32-bit
+// wrap-around arithmetic; the host has checked that no value can leave the int32 range).  First the
+// stages inside a chunk: tensor-memory column 2i is feature i, column 2i+1 feature i + CH/2.
+template <int CH> __device__ __forceinline__ void int_butterfly_chunk(uint32_t (&v)[CH])
+{
+    constexpr int NP = CH / 2;
+#pragma unroll
+    for (int h = 1; h < NP; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            if ((i & h) == 0) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const uint32_t a = v[2 * i + e], b = v[2 * (i + h) + e];
+                    v[2 * i + e] = a + b;
+                    v[2 * (i + h) + e] = a - b;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        const uint32_t a = v[2 * i], b = v[2 * i + 1];
+        v[2 * i] = a + b;
+        v[2 * i + 1] = a - b;
+    }
+}
+// ... then the stages across chunks, on groups of G positions of every chunk (as pass 2 does for
+// the forward rotation), in place in tensor memory.  Both sides of it are barriers of the R warps
+// that share the rows.  Returns false if a wait ran out.
+template <int W> __device__ __forceinline__ bool int_butterfly_across(SlotCtx &c)
+{
+    using C = Cfg<W>;
+    constexpr int NCH = C::NCH, G = C::G, CH = C::CH;
+    ptx::tmem_wait_st();
+    ptx::tc_fence_before();
+    if (!slot_barrier<false>(c)) return false;
+    ptx::tc_fence_after();
+#pragma unroll 1
+    for (int gg = 0; gg < C::GPT; ++gg) {
+        const int g = c.sub * C::GPT + gg;
+        uint32_t u[NCH][G];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
+        ptx::tmem_wait_ld();
+#pragma unroll
+        for (int h = 1; h < NCH; h <<= 1) {
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                if ((ch & h) == 0) {
+#pragma unroll
+                    for (int i = 0; i < G; ++i) {
+                        const uint32_t a = u[ch][i], b = u[ch + h][i];
+                        u[ch][i] = a + b;
+                        u[ch + h][i] = a - b;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tmem_st<G>(c.taddr + ch * CH + g * G, u[ch]);
+    }
+    ptx::tmem_wait_st();
+    ptx::tc_fence_before();
+    if (!slot_barrier<false>(c)) return false;
+    ptx::tc_fence_after();
+    return true;
+}
+
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP, bool BOTH>
 __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
@@ -728,7 +805,7 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                     }
                 }
             }
-            layer1_chunk<W, CH, PER_TOKEN, ROT, DUMP>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v, dY);
+            layer1_chunk<W, CH, PER_TOKEN, ROT, DUMP, BOTH>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v, dY);
             tmem_st<CH>(c.taddr + ch * CH, v);
         }
         if (!finish_layer<W, PER_TOKEN, ROT, DUMP>(c, next_s, next_inv, s_x, dC)) return;
@@ -759,10 +836,31 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
             }
             const uint32_t cbase = consts + ly.c_off * 4;
             const bool fast = ly.epi_mode == EPI_SINE_FAST;
+            if constexpr (BOTH) {
+                // pass 0: acc' = H_W acc on the integers, in place in tensor memory
+#pragma unroll
+                for (int cc = 0; cc < C::CPT; ++cc) {
+                    const int ch = chunk_of<W>(sub, cc);
+                    if constexpr (C::NHALF == 2) {
+                        if (cc == 1) {
+                            if (!wait_bar_warp<PER_TOKEN>(bar_acc + 8, acc_parity, abort_flag, p.status)) return;
+                            acc_parity ^= 1;
+                            ptx::tc_fence_after();
+                        }
+                    }
+                    uint32_t v[CH];
+                    tmem_ld<CH>(c.taddr + ch * CH, v);
+                    ptx::tmem_wait_ld();
+                    if constexpr (DUMP) dump_acc_chunk<W, CH>((valid && p.d.acc[l - 1]) ? p.d.acc[l - 1] + tok * W : nullptr, ch * CH, v);
+                    int_butterfly_chunk<CH>(v);
+                    tmem_st<CH>(c.taddr + ch * CH, v);
+                }
+                if (!int_butterfly_across<W>(c)) return;
+            }
 #pragma unroll
             for (int cc = 0; cc < C::CPT; ++cc) {
                 const int ch = chunk_of<W>(sub, cc);
-                if constexpr (C::NHALF == 2) {
+                if constexpr (C::NHALF == 2 && !BOTH) {
                     // width 512: the thread's second chunk lies in the second half of the output columns,
                     // whose MMAs run while the first chunk is worked on
                     if (cc == 1) {
@@ -776,7 +874,7 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                 ptx::tmem_wait_ld();
                 if constexpr (DUMP) {
                     dY = (valid && p.d.Y[l - 1]) ? p.d.Y[l - 1] + tok * W : nullptr;
-                    dump_acc_chunk<W, CH>((valid && p.d.acc[l - 1]) ? p.d.acc[l - 1] + tok * W : nullptr, ch * CH, v);
+                    if constexpr (!BOTH) dump_acc_chunk<W, CH>((valid && p.d.acc[l - 1]) ? p.d.acc[l - 1] + tok * W : nullptr, ch * CH, v);
                 }
                 if (fast) hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_FAST, DUMP>(cbase, ch * CH, s_x, v, dY);
                 else hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_WIDE, DUMP>(cbase, ch * CH, s_x, v, dY);
@@ -797,6 +895,11 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                 uint32_t u[4];
                 ptx::tmem_ld4(c.taddr, u);
                 ptx::tmem_wait_ld();
+                [[maybe_unused]] uint32_t raw[4] = {u[0], u[1], u[2], u[3]};
+                if constexpr (BOTH) { // z = H_4 (s_w s_x acc) + b over the four padded outputs, on the integers
+                    const uint32_t a0 = u[0] + u[1], a1 = u[0] - u[1], a2 = u[2] + u[3], a3 = u[2] - u[3];
+                    u[0] = a0 + a2; u[2] = a0 - a2; u[1] = a1 + a3; u[3] = a1 - a3;
+                }
                 // Host-buffer variant: a whole tile's results (128 x d_L floats, contiguous in `out`) are
                 // collected in shared memory and leave by one bulk store: over the host link one large
                 // write instead of 128 x d_L four-byte ones.  The slot's 128 sub-0 threads meet on an
@@ -817,7 +920,7 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                         for (int m = 0; m < 4; ++m) {
                             float c_hi = __ldg(ly.cA + m);
                             if (PER_TOKEN) c_hi = __fmul_rn(c_hi, s_x);
-                            if (p.d.acc[p.L - 1]) p.d.acc[p.L - 1][tok * 4 + m] = (int32_t)u[m];
+                            if (p.d.acc[p.L - 1]) p.d.acc[p.L - 1][tok * 4 + m] = (int32_t)raw[m];
                             if (p.d.Y[p.L - 1]) p.d.Y[p.L - 1][tok * 4 + m] = epilogue(EPI_LINEAR, (float)(int)u[m], c_hi, 0.f, __ldg(ly.cB + m));
                         }
                     }
@@ -1024,7 +1127,7 @@ __device__ void xy_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_b
     }
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP = false>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP = false, bool BOTH = false>
 __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_constant__ ParamsOf<DUMP> p)
 {
     using C = Cfg<W>;
@@ -1077,13 +1180,17 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
             const uint32_t *srcA = fixed ? ly.fxP : reinterpret_cast<const uint32_t *>(ly.cA);
             const uint32_t *srcB = fixed ? ly.fxB : reinterpret_cast<const uint32_t *>(ly.cB);
             const uint32_t *srcC = fixed ? ly.fxQ : reinterpret_cast<const uint32_t *>(ly.cA_lo);
-            const int areas = (l == 0) ? (fixed ? 3 : 4) : (ly.epi_mode == EPI_SINE_WIDE ? 3 : 2);
+            const int areas = (l == 0) ? (fixed ? 3 : (BOTH ? 5 : 4)) : (ly.epi_mode == EPI_SINE_WIDE ? 3 : 2);
             for (int i = threadIdx.x; i < W; i += C::THREADS) { // i: tensor-memory column, m: its feature
                 const int m = fused_feature(i, W);
                 d[i] = __ldg(srcA + m);
                 d[W + i] = __ldg(srcB + m);
                 if (areas >= 3) d[2 * W + i] = __ldg(srcC + m);
-                if (areas >= 4) d[3 * W + i] = __ldg(ly.qw_k4m + m);
+                if (areas == 4) d[3 * W + i] = __ldg(ly.qw_k4m + m);
+                if (areas == 5) {
+                    d[3 * W + i] = (uint32_t)__ldg(ly.l1U + m);
+                    d[4 * W + i] = (uint32_t)__ldg(ly.l1V + m);
+                }
             }
         }
     }
@@ -1093,7 +1200,7 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
+        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP, BOTH>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_role<W, SPREAD>(p, sm, smem_base, tmem_base, abort_flag);
     } else if (warp == kLoadWarp) {
@@ -1133,6 +1240,15 @@ template <int W, bool AHEAD_OK> fused_dump_fn pick_dump_width(bool per_token, bo
     if (rot) return per_token ? fused_kernel<W, true, true, false, AHEAD_OK, true> : fused_kernel<W, false, true, false, AHEAD_OK, true>;
     return per_token ? fused_kernel<W, true, false, false, AHEAD_OK, true> : fused_kernel<W, false, false, false, AHEAD_OK, true>;
 }
+// The two-sided transform's kernels: not spread, coordinates not fetched ahead.
+template <int W> fused_fn pick_both_width(bool per_token)
+{
+    return per_token ? fused_kernel<W, true, true, false, false, false, true> : fused_kernel<W, false, true, false, false, false, true>;
+}
+template <int W> fused_dump_fn pick_both_dump_width(bool per_token)
+{
+    return per_token ? fused_kernel<W, true, true, false, false, true, true> : fused_kernel<W, false, true, false, false, true, true>;
+}
 // One translation unit per width (dhq_fused_w*.cu) instantiates the kernels of that width.
 fused_fn fused_pick_64(bool per_token, bool rot, bool spread, bool ahead);
 fused_fn fused_pick_128(bool per_token, bool rot, bool spread, bool ahead);
@@ -1142,5 +1258,13 @@ fused_dump_fn fused_pick_dump_64(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_128(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_256(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_512(bool per_token, bool rot);
+fused_fn fused_pick_both_64(bool per_token);
+fused_fn fused_pick_both_128(bool per_token);
+fused_fn fused_pick_both_256(bool per_token);
+fused_fn fused_pick_both_512(bool per_token);
+fused_dump_fn fused_pick_both_dump_64(bool per_token);
+fused_dump_fn fused_pick_both_dump_128(bool per_token);
+fused_dump_fn fused_pick_both_dump_256(bool per_token);
+fused_dump_fn fused_pick_both_dump_512(bool per_token);
 
 } // namespace dhq

@@ -6,5 +6,7 @@ namespace dhq {
 
 fused_fn fused_pick_128(bool per_token, bool rot, bool spread, bool ahead) { return pick_width<128, true>(per_token, rot, spread, ahead); }
 fused_dump_fn fused_pick_dump_128(bool per_token, bool rot) { return pick_dump_width<128, true>(per_token, rot); }
+fused_fn fused_pick_both_128(bool per_token) { return pick_both_width<128>(per_token); }
+fused_dump_fn fused_pick_both_dump_128(bool per_token) { return pick_both_dump_width<128>(per_token); }
 
 } // namespace dhq

@@ -30,6 +30,8 @@ struct LayerDev {
     float *cA = nullptr, *cA_lo = nullptr, *cB = nullptr; // [M] epilogue constants
     uint32_t *fxP = nullptr, *fxQ = nullptr, *fxB = nullptr; // [M] fixed-point phase constants (EPI_SINE_FIXED)
     float *act = nullptr;      // [4]: frozen absmax (max taken on the bit pattern), s_x, inv, unused
+    int has_uv = 0;            // two-sided transform, layer 1: l1U, l1V below
+    int32_t *l1U = nullptr, *l1V = nullptr; // [M] H_M applied to u_m = q[m][0]+q[m][2] and v_m = q[m][1]+q[m][3]
     int has_f32 = 0;           // W32A32 handles keep the unquantized weights too
     float *w_f32 = nullptr;    // [K/4][M] float4: fp32 weights, zero padded (has_f32 only)
 };
@@ -132,6 +134,7 @@ struct PrepArgs {
     double omega0;
     LayerDev dev;
     float *phase_bound;    // device scalar
+    unsigned long long *code_l1; // device scalar: sum over the layer of |q_w[m][k]| (bounds the rotated accumulators)
 };
 cudaError_t launch_prepare(const PrepArgs &a, cudaStream_t st, int64_t *launches);
 // Epilogue constants from s_w and (per-tensor) the frozen activation scale.

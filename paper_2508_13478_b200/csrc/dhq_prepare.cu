@@ -149,6 +149,7 @@ __global__ void prep_bound_kernel(PrepArgs a)
     for (int m = threadIdx.x; m < a.M; m += blockDim.x) {
         float qsum = 0.f;
         for (int k = 0; k < K; ++k) qsum += fabsf((float)a.dev.qw[(size_t)m * K + k]);
+        atomicAdd(a.code_l1, (unsigned long long)qsum); // exact: at most 512 * 127 per row
         const float sw = a.dev.s_w[m];
         const float slack = 0.5f * sw * xsum + 0.5f * sx_max * sw * qsum;
         worst = fmaxf(worst, (float)a.omega0 * (a.dev.row_l1[m] + slack) * 1.0001f);
@@ -160,6 +161,35 @@ __global__ void prep_bound_kernel(PrepArgs a)
         float r = 0.f;
         for (int i = 0; i < (blockDim.x + 31) / 32; ++i) r = fmaxf(r, red[i]);
         *a.phase_bound = r;
+    }
+}
+
+// Two-sided transform, layer 1 (K = 4): the rotated padded coordinate has the codes [qs, qd, qs, qd],
+// so acc_m = qs u_m + qd v_m with u_m = q[m][0] + q[m][2], v_m = q[m][1] + q[m][3], and the rotated
+// accumulators are acc'_j = qs (H_M u)_j + qd (H_M v)_j.  One block computes H_M u and H_M v.
+__global__ void prep_l1_both_kernel(LayerDev dev)
+{
+    extern __shared__ int uv[]; // [2][M]
+    const int M = dev.M;
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+        const int8_t *q = dev.qw + (size_t)m * 4;
+        uv[m] = (int)q[0] + (int)q[2];
+        uv[M + m] = (int)q[1] + (int)q[3];
+    }
+    for (int h = 1; h < M; h <<= 1) {
+        __syncthreads();
+        for (int p = threadIdx.x; p < M; p += blockDim.x) { // M/2 pairs for each of the two vectors
+            const int which = p / (M / 2), j = p % (M / 2);
+            const int i = which * M + (((j & ~(h - 1)) << 1) | (j & (h - 1)));
+            const int x = uv[i], y = uv[i + h];
+            uv[i] = x + y;
+            uv[i + h] = x - y;
+        }
+    }
+    __syncthreads();
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+        dev.l1U[m] = uv[m];
+        dev.l1V[m] = uv[M + m];
     }
 }
 
@@ -191,7 +221,11 @@ __global__ void finalize_kernel(LayerDev dev, int a_bits, int per_token, int sin
         if (dev.epi_mode == EPI_SINE_FIXED) {
             const double inv_two_pi = 0.15915494309189533576888;
             const int8_t *q = dev.qw + (size_t)m * 4;   // layer 1: K = 4
-            const double u = (double)((int)q[0] + (int)q[2]), v = (double)((int)q[1] + (int)q[3]);
+            double u = (double)((int)q[0] + (int)q[2]), v = (double)((int)q[1] + (int)q[3]);
+            if (dev.has_uv) { // two-sided transform: the phase of output j comes from the rotated sums
+                u = (double)dev.l1U[m];
+                v = (double)dev.l1V[m];
+            }
             auto to_fix = [](double turns) { return (uint32_t)(unsigned long long)llrint(turns * 4294967296.0); };
             dev.fxP[m] = to_fix(A * u * inv_two_pi);
             dev.fxQ[m] = to_fix(A * v * inv_two_pi);
@@ -215,6 +249,10 @@ cudaError_t launch_prepare(const PrepArgs &a, cudaStream_t st, int64_t *launches
     prep_quant_kernel<<<(total + 255) / 256, 256, 0, st>>>(a);
     prep_bound_kernel<<<1, 256, 0, st>>>(a);
     *launches += 4;
+    if (a.dev.has_uv) {
+        prep_l1_both_kernel<<<1, 256, 2 * a.M * sizeof(int), st>>>(a.dev);
+        *launches += 1;
+    }
     return cudaGetLastError();
 }
 

@@ -239,3 +239,47 @@ def test_free_running_chains_differ_only_through_code_flips_at_rounding_ties():
               f"{flips} with a first code flip (all by one step at a tie), max |d| = {np.abs(got - ref).max():.2e}")
     finally:
         dhq.dhq_destroy(h)
+
+
+@pytest.mark.parametrize("width,a_gran", [(64, 0), (64, 1), (128, 1), (256, 0), (256, 1), (512, 0), (512, 1)])
+def test_two_sided_transform_inside_the_fused_kernel(width, a_gran):
+    # DHQ_ROT_BOTH with one weight scale per tensor: z = H_M (s_w s_x acc) + b with the rotation taken
+    # on the int32 accumulators (exact), then the fp32 epilogue.  Accumulators are dumped before that
+    # rotation (they are the definition's q_x q_W^T); the outputs must be within 1e-5 of the fp64 H_M product.
+    wl = dhq_inputs.Workload("both", (2, width, width, width, 3), 30.0, 900 + width + a_gran, 8, 8, 0, a_gran, (8, 8))
+    n = 148 * (1 if width == 512 else 2) * 128 + 300
+    coords = dhq_inputs.grid_coords(251, 157)[:n]
+    weights, biases = wl.network()
+    h, net = prepare_pair(wl.dims, weights, biases, wl.omega0, 8, 8, 0, a_gran, rotate="both")
+    try:
+        check_weights(h, net)
+        if a_gran == 0:
+            dhq.dhq_calibrate(h, to_dev(coords))
+        worst = _observe(h, net, coords, calib_is_this_set=False)
+        # the host-buffer route runs the same kernel
+        oh = torch.zeros((n, 3)).pin_memory()
+        dhq.dhq_forward_host(h, torch.from_numpy(coords).pin_memory(), oh)
+        out = torch.empty((n, 3), device="cuda")
+        dhq.dhq_forward(h, to_dev(coords), out)
+        torch.cuda.synchronize()
+        assert torch.equal(oh.view(torch.int32), out.cpu().view(torch.int32))
+        print(f"two-sided, fused, width {width}, a_gran {a_gran}: outputs within {worst:.2e}")
+    finally:
+        dhq.dhq_destroy(h)
+
+
+def test_two_sided_transform_with_per_channel_weight_scales_stays_layer_by_layer():
+    w = dhq_inputs.WORKLOADS["C3"]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, 8, 8, 1, 1, rotate="both")
+    try:
+        cd = to_dev(w.coords()[:300])
+        out = torch.empty((300, 3), device="cuda")
+        with pytest.raises(dhq.DhqError) as e:
+            dhq.dhq_forward_fused_debug(h, cd, out)
+        assert e.value.code == 2
+        dhq.dhq_forward(h, cd, out)                      # runs, layer by layer
+        torch.cuda.synchronize()
+        assert torch.isfinite(out).all() and dhq.dhq_last_status(h) == 0
+    finally:
+        dhq.dhq_destroy(h)
