@@ -32,6 +32,9 @@
  *   - Argument errors are reported by the return value and enqueue nothing.  Conditions found on
  *     the device (a bounded wait that ran out) are recorded in a status word read by
  *     dhq_last_status.  Nothing traps, aborts or throws.
+ *   - With the environment variable DHQ_LOG set (to anything but "0") dhq_prepare, dhq_calibrate,
+ *     dhq_forward and dhq_forward_host write one line per call to stderr (size, shape, route, status,
+ *     kernels enqueued).
  *   - One forward may be in flight per handle at a time.  Handles belong to the device that was
  *     current in dhq_prepare; that device must be current in later calls (INVALID_ARG otherwise).
  */

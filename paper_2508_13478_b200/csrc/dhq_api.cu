@@ -2,6 +2,7 @@
 // kernels on the caller's stream.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include "dhq_internal.cuh"
@@ -305,8 +306,8 @@ void dhq_destroy(dhq_handle_t h)
     delete h;
 }
 
-dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const float *const *b,
-                         void *stream, dhq_handle_t *out)
+static dhq_status_t prepare_impl(const dhq_config_t *cfg, const float *const *W, const float *const *b,
+                                 void *stream, dhq_handle_t *out)
 {
     if (!cfg || !W || !b || !out || !cfg->dims) return DHQ_ERR_INVALID_ARG;
     *out = nullptr;
@@ -407,7 +408,7 @@ dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const f
     return DHQ_OK;
 }
 
-dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void *stream)
+static dhq_status_t calibrate_entry(dhq_handle_t h, const float *coords, int64_t n, void *stream)
 {
     if (!h || !coords || n < 1) return DHQ_ERR_INVALID_ARG;
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
@@ -543,7 +544,7 @@ dhq_status_t dhq_debug_stall_next_forward(dhq_handle_t h)
     return DHQ_OK;
 }
 
-dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *out, void *stream)
+static dhq_status_t forward_entry(dhq_handle_t h, const float *coords, int64_t n, float *out, void *stream)
 {
     if (!h || n < 0 || (n > 0 && (!coords || !out))) return DHQ_ERR_INVALID_ARG;
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
@@ -557,8 +558,8 @@ dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *
     return run_forward(h, coords, n, out, false, st);
 }
 
-dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t n, float *out_host,
-                              void *stream)
+static dhq_status_t forward_host_entry(dhq_handle_t h, const float *coords_host, int64_t n, float *out_host,
+                                       void *stream)
 {
     if (!h || n < 0 || (n > 0 && (!coords_host || !out_host))) return DHQ_ERR_INVALID_ARG;
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
@@ -597,7 +598,7 @@ dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t 
                                                                  // scales on ALL of its coordinates; the layer-by-layer paths are not cut
     if (chunks <= 1) {
         CK(cudaMemcpyAsync(h->stage_in, coords_host, (size_t)n * 2 * sizeof(float), cudaMemcpyHostToDevice, st));
-        dhq_status_t s = dhq_forward(h, h->stage_in, n, h->stage_out, stream);
+        dhq_status_t s = forward_entry(h, h->stage_in, n, h->stage_out, stream);
         if (s != DHQ_OK) return s;
         CK(cudaMemcpyAsync(out_host, h->stage_out, (size_t)n * h->d_L * sizeof(float), cudaMemcpyDeviceToHost, st));
         return DHQ_OK;
@@ -798,5 +799,54 @@ dhq_status_t dhq_last_status(dhq_handle_t h)
 }
 
 int64_t dhq_launch_count(dhq_handle_t h) { return h ? h->launches : 0; }
+
+// Call log: with the environment variable DHQ_LOG set (to anything but "0") the main entry points
+// write one line per call to stderr - the call, its size, the handle's shape, the status returned and
+// the number of kernels it enqueued.  Read once per process; costs one predictable branch otherwise.
+static bool log_enabled()
+{
+    static const bool on = [] {
+        const char *v = getenv("DHQ_LOG");
+        return v && v[0] && !(v[0] == '0' && !v[1]);
+    }();
+    return on;
+}
+static void log_call(const char *fn, dhq_handle_t h, int64_t n, int64_t launches_before, dhq_status_t s)
+{
+    if (!h) { fprintf(stderr, "[dhq] %s n=%lld -> %s\n", fn, (long long)n, dhq_status_string(s)); return; }
+    fprintf(stderr, "[dhq] %s n=%lld (L=%d w=%d d_L=%d W%dA%d rot=%d gran=%d/%d%s) -> %s, %lld kernel(s)\n", fn, (long long)n,
+            h->L, h->w, h->d_L, h->cfg.w_bits, h->cfg.a_bits, (int)h->cfg.rotation, (int)h->cfg.w_gran, (int)h->cfg.a_gran,
+            h->fused ? ", fused" : ", layer by layer", dhq_status_string(s), (long long)(h->launches - launches_before));
+}
+
+dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W, const float *const *b, void *stream, dhq_handle_t *out)
+{
+    const dhq_status_t s = prepare_impl(cfg, W, b, stream, out);
+    if (log_enabled()) log_call("dhq_prepare", (s == DHQ_OK && out) ? *out : nullptr, 0, 0, s);
+    return s;
+}
+dhq_status_t dhq_calibrate(dhq_handle_t h, const float *coords, int64_t n, void *stream)
+{
+    const int64_t before = h ? h->launches : 0;
+    const dhq_status_t s = calibrate_entry(h, coords, n, stream);
+    if (log_enabled()) log_call("dhq_calibrate", h, n, before, s);
+    return s;
+}
+dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *out, void *stream)
+{
+    if (!log_enabled()) return forward_entry(h, coords, n, out, stream);
+    const int64_t before = h ? h->launches : 0;
+    const dhq_status_t s = forward_entry(h, coords, n, out, stream);
+    log_call("dhq_forward", h, n, before, s);
+    return s;
+}
+dhq_status_t dhq_forward_host(dhq_handle_t h, const float *coords_host, int64_t n, float *out_host, void *stream)
+{
+    if (!log_enabled()) return forward_host_entry(h, coords_host, n, out_host, stream);
+    const int64_t before = h ? h->launches : 0;
+    const dhq_status_t s = forward_host_entry(h, coords_host, n, out_host, stream);
+    log_call("dhq_forward_host", h, n, before, s);
+    return s;
+}
 
 } // extern "C"

@@ -57,3 +57,26 @@ def test_export_import_round_trip_is_bit_identical(name):
         dhq.dhq_destroy(h)
         if h2:
             dhq.dhq_destroy(h2)
+
+
+@pytest.mark.gpu
+def test_call_log_is_written_when_asked_for():
+    # DHQ_LOG is read once per process: run a small forward in a child process
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import torch, dhq_inputs, paper_2508_13478_b200 as d\n"
+        "w = dhq_inputs.WORKLOADS['C1']; W, B = w.network()\n"
+        "h = d.dhq_prepare(w.dims, [torch.from_numpy(x).cuda() for x in W], [torch.from_numpy(x).cuda() for x in B])\n"
+        "c = torch.from_numpy(w.coords()[:300]).cuda(); o = torch.empty((300, 1), device='cuda')\n"
+        "d.dhq_forward(h, c, o); torch.cuda.synchronize(); d.dhq_destroy(h)\n")
+    for setting, expect in (("1", True), ("0", False)):
+        env = dict(os.environ, DHQ_LOG=setting, PYTHONPATH=root)
+        r = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0, r.stderr
+        assert ("[dhq] dhq_forward n=300" in r.stderr) == expect
+        assert ("[dhq] dhq_prepare" in r.stderr) == expect
+        if expect:
+            assert "-> ok" in r.stderr and "fused" in r.stderr
