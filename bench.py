@@ -286,6 +286,18 @@ class Runner:
         self.dhq.dhq_destroy(self.h)
 
 
+def launch_clock(dhq, run):
+    """SM clock inside a launch of this workload: three back-to-back launches of the observing
+    instantiation of the fused kernel (no dump buffers: the same work as the timed kernel), which
+    carries a cycle-counter / nanosecond-timer probe that the timed instantiations leave out."""
+    try:
+        for _ in range(3):
+            dhq.dhq_forward_fused_debug(run.h, run.coords, run.out)
+        return dhq.dhq_last_launch_clock(run.h)
+    except Exception:
+        return None, None
+
+
 def packed_weight_bytes(dims):
     """Bytes of the prepared int8 weights a launch reads once (tensor-core images of the hidden and
     last layers, one word per feature for the first)."""
@@ -304,7 +316,7 @@ def dram_traffic(workload, rotation, n):
     return fixed + (captured - fixed) * (n / coords)
 
 
-def roofline_of(workload, rotation, n, ms_per_step, sm_max_mhz, sampled_mhz, fma_peak):
+def roofline_of(workload, rotation, n, ms_per_step, sm_max_mhz, sampled_mhz, fma_peak, kernel_mhz=None):
     """ALU roofline of one launch: algorithmic lane-ops over the CUDA-event duration, against (a) the
     derived peak SMs x fp32 lanes x max SM clock, (b) the same at the SM clock sampled during the
     timed steps, (c) the FMA loop's rate measured in this run."""
@@ -317,6 +329,8 @@ def roofline_of(workload, rotation, n, ms_per_step, sm_max_mhz, sampled_mhz, fma
          "peak_source": "148 SMs x 128 fp32 lanes x max SM clock (derived from unit counts and clock)"}
     if sampled_mhz:
         r["frac_at_sampled_clock"] = achieved / (SM_COUNT * FP32_LANES_PER_SM * sampled_mhz * 1e6 / 1e12)
+    if kernel_mhz:   # cycle counter over nanosecond timer inside a launch of the same work (launch_clock)
+        r["frac_at_kernel_clock"] = achieved / (SM_COUNT * FP32_LANES_PER_SM * kernel_mhz * 1e6 / 1e12)
     if fma_peak:
         r["peak_measured_fma"] = fma_peak / 1e12
         r["frac_of_measured_fma"] = achieved / (fma_peak / 1e12)
@@ -353,6 +367,7 @@ def run_ours(args, workload):
     with ClockSampler(physical_gpu_index(local_rank)) as clocks:
         total_ms = run.timed(run.forward, args.steps, flush, barrier)
     launches = dhq.dhq_launch_count(run.h) - launches0
+    kernel_mhz, kernel_ms = launch_clock(dhq, run)
     e2e_ms = run.timed(run.forward_host, args.steps, flush, barrier)
     status = dhq.dhq_last_status(run.h)
 
@@ -370,6 +385,8 @@ def run_ours(args, workload):
             pass
         sm_max = float(peaks.get("sm_max_mhz", 1965.0))
         csum = clocks.summary()
+        csum["sm_mhz_in_kernel"] = kernel_mhz
+        csum["kernel_ms_in_kernel"] = kernel_ms
         try:
             fma_peak, _ = dhq.dhq_measure_pipe("ffma", 2000)
         except Exception:
@@ -387,7 +404,7 @@ def run_ours(args, workload):
                              "the result over the host link through the buffers' device mapping, every step "
                              "(whole tiles by bulk copy where the width's kernel has that variant)"},
             "gpu_launches": launches,
-            "roofline": roofline_of(workload, args.rotation, n, ms_per_step, sm_max, csum["sm_mhz"], fma_peak),
+            "roofline": roofline_of(workload, args.rotation, n, ms_per_step, sm_max, csum["sm_mhz"], fma_peak, kernel_mhz),
             "device_status": status,
         }
         # The same launch against the other pipes' ceilings, each measured now on this GPU by the
@@ -429,9 +446,11 @@ def run_ours(args, workload):
             with ClockSampler(physical_gpu_index(local_rank)) as ck:
                 ms = r.timed(r.forward, steps, flush, barrier) / steps
             st = dhq.dhq_last_status(r.h)
-            roof = roofline_of(other, args.rotation, r.n, ms, sm_max, ck.summary()["sm_mhz"], fma_peak)
+            k_mhz = launch_clock(dhq, r)[0]
+            roof = roofline_of(other, args.rotation, r.n, ms, sm_max, ck.summary()["sm_mhz"], fma_peak, k_mhz)
             per[name] = {"coords_per_step": r.n, "steps": steps, "ms_per_step": ms, "value": r.n / (ms * 1e-3),
                          "roofline_frac": roof["frac"], "frac_of_measured_fma": roof.get("frac_of_measured_fma"),
+                         "sm_mhz_in_kernel": k_mhz, "frac_at_kernel_clock": roof.get("frac_at_kernel_clock"),
                          "traffic": roof["traffic"], "device_status": st}
             r.close()
         line["per_config"] = per

@@ -341,6 +341,19 @@ DHQ_API dhq_status_t dhq_layer_dims(dhq_handle_t h, int layer, int *K, int *M);
  */
 DHQ_API dhq_status_t dhq_last_status(dhq_handle_t h);
 
+/*
+ * The SM clock that the handle's last dhq_forward_fused_debug launch really ran at: in that
+ * instantiation of the fused kernel two threads of the first CTA read the SM's cycle counter and
+ * the global nanosecond timer before and after the work; sm_mhz = cycles / time.  (NVML reports the
+ * clock the driver asks for; inside the launches the SMs were seen 4-8 % below it.  The timed
+ * instantiations do not carry the probe: a dhq_forward_fused_debug call without dump buffers does
+ * the same work at nearly the same speed and serves as the clock measurement.)  milliseconds: that
+ * CTA's run time, close to the launch's.  Synchronizes the device.  Either pointer may be NULL.
+ * (No counterpart in the paper: measurement.)
+ * Errors: INVALID_ARG (no such launch yet), UNSUPPORTED (handle runs layer by layer), CUDA.
+ */
+DHQ_API dhq_status_t dhq_last_launch_clock(dhq_handle_t h, double *sm_mhz, double *milliseconds);
+
 /* Number of kernels the library has launched for this handle since it was created. */
 DHQ_API int64_t dhq_launch_count(dhq_handle_t h);
 

@@ -11,6 +11,6 @@ from .binding import (  # noqa: F401
     DHQ_STATIC_MAX_TOKENS, dhq_get_layer,
     dhq_layer_dims, dhq_last_status, dhq_launch_count, dhq_destroy, dhq_status_string,
     dhq_measure_pipe, library_path, load_library, dhq_forward_fused_debug, dhq_set_wait_limit,
-    dhq_debug_stall_next_forward, dhq_measure_sine_error, dhq_export, dhq_import, DHQ_ROT_BOTH, DHQ_ROT_NONE, DHQ_BITS_FLOAT, DHQ_ACT_SINE, DHQ_ACT_GABOR,
+    dhq_debug_stall_next_forward, dhq_measure_sine_error, dhq_export, dhq_import, dhq_last_launch_clock, DHQ_ROT_BOTH, DHQ_ROT_NONE, DHQ_BITS_FLOAT, DHQ_ACT_SINE, DHQ_ACT_GABOR,
 )
 from .sharded import calibrate_sharded, shard_range  # noqa: F401,E402

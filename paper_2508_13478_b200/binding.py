@@ -75,6 +75,8 @@ def load_library():
     L.dhq_forward_debug.argtypes = [vp, vp, c_i64, vp, ctypes.POINTER(_DebugBufs), vp]
     L.dhq_forward_fused_debug.argtypes = [vp, vp, c_i64, vp, ctypes.POINTER(_DebugBufs), vp]
     L.dhq_set_wait_limit.argtypes = [vp, c_i64]
+    L.dhq_last_launch_clock.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    L.dhq_last_launch_clock.restype = c_i
     L.dhq_export.argtypes = [vp, vp, c_i64, ctypes.POINTER(c_i64)]
     L.dhq_import.argtypes = [ctypes.c_char_p, c_i64, vp, ctypes.POINTER(vp)]
     L.dhq_debug_stall_next_forward.argtypes = [vp]
@@ -275,6 +277,13 @@ def dhq_import(blob: bytes, stream=None):
 
 def dhq_last_status(handle) -> int:
     return int(load_library().dhq_last_status(handle))
+
+
+def dhq_last_launch_clock(handle):
+    """(SM MHz, milliseconds) of the handle's last fused-kernel launch, measured inside the kernel."""
+    mhz, ms = ctypes.c_double(), ctypes.c_double()
+    _check(load_library().dhq_last_launch_clock(handle, ctypes.byref(mhz), ctypes.byref(ms)), "dhq_last_launch_clock")
+    return mhz.value, ms.value
 
 
 def dhq_launch_count(handle) -> int:

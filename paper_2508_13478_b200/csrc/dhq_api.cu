@@ -339,8 +339,8 @@ static dhq_status_t prepare_impl(const dhq_config_t *cfg, const float *const *W,
     const bool per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN || h->float_mode != 0;
     do {
         if (cudaGetDevice(&h->device) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
-        if (!dev_alloc(&h->d_status, 4) || !dev_alloc(&d_bounds, kMaxLayers) || !dev_alloc(&d_sums, kMaxLayers)) { rc = DHQ_ERR_ALLOC; break; }
-        if (cudaMemsetAsync(h->d_status, 0, 16, st) != cudaSuccess ||
+        if (!dev_alloc(&h->d_status, 16) || !dev_alloc(&d_bounds, kMaxLayers) || !dev_alloc(&d_sums, kMaxLayers)) { rc = DHQ_ERR_ALLOC; break; }
+        if (cudaMemsetAsync(h->d_status, 0, 64, st) != cudaSuccess ||
             cudaMemsetAsync(d_bounds, 0, kMaxLayers * sizeof(float), st) != cudaSuccess ||
             cudaMemsetAsync(d_sums, 0, kMaxLayers * sizeof(unsigned long long), st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
         for (int l = 1; l <= L && rc == DHQ_OK; ++l) {
@@ -393,7 +393,8 @@ static dhq_status_t prepare_impl(const dhq_config_t *cfg, const float *const *W,
             if (l == L) d.epi_mode = EPI_LINEAR;
             else if (l == 1) {}
             // (two-sided: the quantization error of all M rows meets in every output; no tight phase bound)
-            else d.epi_mode = (bounds[l - 1] <= kFastPhaseLimit && !gabor && !both) ? EPI_SINE_FAST : EPI_SINE_WIDE;
+            else d.epi_mode = (bounds[l - 1] <= (cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN ? kFastPhaseLimitPerToken : kFastPhaseLimit) &&
+                               !gabor && !both) ? EPI_SINE_FAST : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;
         if ((!both || both_fused) && !h->float_mode && !gabor) rc = fused_create(h); // the two-sided transform and the fp32 datapaths run layer by layer
@@ -738,8 +739,8 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
     dhq_status_t rc = DHQ_OK;
     do {
         if (cudaGetDevice(&h->device) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
-        if (!dev_alloc(&h->d_status, 4)) { rc = DHQ_ERR_ALLOC; break; }
-        if (cudaMemsetAsync(h->d_status, 0, 16, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
+        if (!dev_alloc(&h->d_status, 16)) { rc = DHQ_ERR_ALLOC; break; }
+        if (cudaMemsetAsync(h->d_status, 0, 64, st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
         for (int l = 0; l < h->L && rc == DHQ_OK; ++l) {
             LayerDev &d = h->layer[l];
             if (!alloc_layer(d)) { rc = DHQ_ERR_ALLOC; break; }
@@ -796,6 +797,20 @@ dhq_status_t dhq_last_status(dhq_handle_t h)
     CK(cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));
     CK(cudaMemset(h->d_status, 0, sizeof(int)));
     return v == 0 ? DHQ_OK : DHQ_ERR_TIMEOUT;
+}
+
+dhq_status_t dhq_last_launch_clock(dhq_handle_t h, double *sm_mhz, double *milliseconds)
+{
+    if (!h || !on_own_device(h)) return DHQ_ERR_INVALID_ARG;
+    if (!h->fused) return DHQ_ERR_UNSUPPORTED;
+    long long words[5] = {0, 0, 0, 0, 0};
+    CK(cudaDeviceSynchronize());
+    CK(cudaMemcpy(words, h->d_status, sizeof(words), cudaMemcpyDeviceToHost));
+    const double cycles = (double)(words[3] - words[1]), ns = (double)(words[4] - words[2]);
+    if (!(ns > 0.0)) return DHQ_ERR_INVALID_ARG; // no fused launch yet
+    if (sm_mhz) *sm_mhz = cycles / ns * 1e3;
+    if (milliseconds) *milliseconds = ns * 1e-6;
+    return DHQ_OK;
 }
 
 int64_t dhq_launch_count(dhq_handle_t h) { return h ? h->launches : 0; }

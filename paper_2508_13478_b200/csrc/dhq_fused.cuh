@@ -1205,6 +1205,16 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
         if (lane == 0) mma_role<W, SPREAD>(p, sm, smem_base, tmem_base, abort_flag);
     } else if (warp == kLoadWarp) {
         if (lane == 0) load_role<W, SPREAD>(p, sm, smem_base, abort_flag);
+        if constexpr (DUMP) {
+            // Observing instantiation only (in the timed kernels these few instructions cost 3-4 %): an
+            // otherwise idle lane of CTA 0 notes the SM's cycle counter and the global nanosecond timer
+            // before the work (status words 2-5); the MMA warp notes them again after it (words 6-9).
+            // The ratio of the differences is the SM clock the launch really ran at.
+            if (lane == 1 && blockIdx.x == 0) {
+                reinterpret_cast<long long *>(p.status)[1] = clock64();
+                reinterpret_cast<unsigned long long *>(p.status)[2] = ptx::globaltimer();
+            }
+        }
     } else {
         if constexpr (C::BULK_XY) {
             if (lane == 0) xy_role<W, SPREAD>(p, sm, smem_base, abort_flag);
@@ -1215,6 +1225,12 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
     if (warp == kMmaWarp) {
         __syncwarp();
         ptx::tmem_dealloc(tmem_base, 512);
+        if constexpr (DUMP) {
+            if (lane == 0 && blockIdx.x == 0) {
+                reinterpret_cast<long long *>(p.status)[3] = clock64();
+                reinterpret_cast<unsigned long long *>(p.status)[4] = ptx::globaltimer();
+            }
+        }
     }
 }
 

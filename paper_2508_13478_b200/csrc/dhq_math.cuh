@@ -24,8 +24,11 @@ enum EpiMode : int {
 // hardware approximation itself, measured on B200 against the fp64 sine over 2^24 arguments per
 // range (dhq_measure_sine_error): 6.2e-7 for |x| <= 3.2, 2.3e-6 to 16, 4.4e-6 to 32, 4.6e-6 to 40,
 // 5.0e-6 to 48, 8.3e-6 to 56 - its internal multiply by 1/(2 pi) loses absolute accuracy as the
-// argument grows.  Sum at 36: 8.7e-6.
+// argument grows.  Sum at 36: 8.7e-6.  With a per-token activation scale the constant is the product
+// fl32(cA * s_x) of two rounded factors (twice the constant error) and the limit is 32 rad, where the
+// fma result still has half the ulp: 0.95e-6 + 3.8e-6 + 1e-7 + 4.4e-6 = 9.3e-6.
 constexpr float kFastPhaseLimit = 36.0f;
+constexpr float kFastPhaseLimitPerToken = 32.0f;
 
 __device__ __forceinline__ float qmax_of(int bits) { return (float)((1 << (bits - 1)) - 1); }
 
