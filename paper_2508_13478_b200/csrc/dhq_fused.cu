@@ -19,6 +19,16 @@ static fused_fn pick_kernel(int W, bool per_token, bool rot, bool spread, bool a
     return nullptr;
 }
 
+static fused_fn pick_calib_kernel(int W, bool rot)
+{
+    switch (W) {
+    case 64: return fused_pick_calib_64(rot);
+    case 128: return fused_pick_calib_128(rot);
+    case 256: return fused_pick_calib_256(rot);
+    case 512: return fused_pick_calib_512(rot);
+    }
+    return nullptr;
+}
 static fused_fn pick_both_kernel(int W, bool per_token)
 {
     switch (W) {
@@ -108,6 +118,11 @@ dhq_status_t fused_create(dhq_handle_s *h)
         if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
+    if (!both && !p.per_token) {
+        fused_fn fc = pick_calib_kernel(h->w, h->cfg.rotation == DHQ_ROT_INPUT);
+        if (!fc || cudaFuncSetAttribute(fc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+            return DHQ_ERR_CUDA;
+    }
     fused_dump_fn fd = both ? pick_both_dump_kernel(h->w, p.per_token) : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     if (!fd || cudaFuncSetAttribute(fd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
         return DHQ_ERR_CUDA;
@@ -153,6 +168,46 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     const bool spread = !both && slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
     fused_fn fn = both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
+    int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
+    fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
+    h->launches++;
+    return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;
+}
+
+// Layer 1's rotated input is H_4 [x, y, 0, 0] = [x+y, x-y, x+y, x-y] (or [x, y, 0, 0] without the
+// rotation): its absmax over the coordinate set needs no network.
+__global__ void calib_l1_kernel(const float *coords, long long n, int rot, float *act)
+{
+    float amax = 0.f;
+    for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < n; t += (long long)gridDim.x * blockDim.x) {
+        const float2 xy = __ldg(reinterpret_cast<const float2 *>(coords) + t);
+        const float a = rot ? __fadd_rn(xy.x, xy.y) : xy.x, b = rot ? __fsub_rn(xy.x, xy.y) : xy.y;
+        amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+    }
+    for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(reinterpret_cast<unsigned int *>(act), __float_as_uint(amax));
+}
+
+// One calibration pass by the fused kernel: the maximum of |rotated input of layer l| over the
+// coordinates, with layers < l run as they are frozen, is accumulated into the layer's act[0]
+// (which the caller has cleared).  Per-tensor activation scales, one-sided or no rotation.
+dhq_status_t fused_calibrate_layer(dhq_handle_s *h, int l, const float *coords, int64_t n, cudaStream_t st)
+{
+    FusedState *fs = static_cast<FusedState *>(h->fused);
+    if (!fs || fs->p.per_token || h->cfg.rotation == DHQ_ROT_BOTH || l < 1 || l > h->L) return DHQ_ERR_INVALID_ARG;
+    if (n <= 0) return DHQ_OK;
+    if (l == 1) {
+        const long long blocks = (n + 255) / 256;
+        calib_l1_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), 256, 0, st>>>(coords, n, h->cfg.rotation == DHQ_ROT_INPUT, h->layer[0].act);
+        h->launches++;
+        return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;
+    }
+    FusedParams p = fs->p;
+    fill_call(h, p, coords, n, nullptr);
+    p.L = l; // the network up to the rotated input of layer l
+    const int slots = (h->w == 512) ? 1 : 2;
+    fused_fn fn = pick_calib_kernel(h->w, h->cfg.rotation == DHQ_ROT_INPUT);
+    const long long ctas = (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
     h->launches++;

@@ -602,6 +602,59 @@ __device__ __forceinline__ bool finish_layer(SlotCtx &c, float static_s, float s
     return true;
 }
 
+// Calibration instantiation (per-tensor activation scales, Section III-C's run-time statistic taken
+// once): in place of the quantizer, the maximum of |x~| over the tile's valid tokens goes to the
+// calibrated layer's act[0] (atomic maximum on the bit pattern: non-negative floats order as
+// integers).  Same barrier, loads and butterfly stages as finish_layer up to that point.
+template <int W, bool ROT> __device__ __forceinline__ bool calib_finish(SlotCtx &c, bool valid, float *act)
+{
+    using C = Cfg<W>;
+    constexpr int NCH = C::NCH, G = C::G, CH = C::CH;
+    ptx::tmem_wait_st();
+    ptx::tc_fence_before();
+    if (!slot_barrier<false>(c)) return false;
+    ptx::tc_fence_after();
+    float amax = 0.f;
+#pragma unroll 1
+    for (int gg = 0; gg < C::GPT; ++gg) {
+        const int g = c.sub * C::GPT + gg;
+        uint32_t u[NCH][G];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) tmem_ld<G>(c.taddr + ch * CH + g * G, u[ch]);
+        ptx::tmem_wait_ld();
+#pragma unroll
+        for (int h = 1; h < (ROT ? NCH : 1); h <<= 1) {
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                if ((ch & h) == 0) {
+#pragma unroll
+                    for (int i = 0; i < G; i += 2) {
+                        f32x2 a = pack2u(u[ch][i], u[ch][i + 1]), b = pack2u(u[ch + h][i], u[ch + h][i + 1]);
+                        bfly2(a, b);
+                        unpack2u(a, u[ch][i], u[ch][i + 1]);
+                        unpack2u(b, u[ch + h][i], u[ch + h][i + 1]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) {
+#pragma unroll
+            for (int i = 0; i < G; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(u[ch][i])));
+        }
+    }
+    if (!valid) amax = 0.f; // rows past the end of the coordinate set do not count
+#pragma unroll
+    for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((c.row & 31) == 0) atomicMax(reinterpret_cast<unsigned int *>(act), __float_as_uint(amax));
+    // the next tile's first layer writes these tensor-memory columns: every warp of the row group
+    // must have finished reading them
+    ptx::tc_fence_before();
+    if (!slot_barrier<false>(c)) return false;
+    ptx::tc_fence_after();
+    return true;
+}
+
 // Observing instantiation: the int32 accumulators of CH tensor-memory columns starting at column
 // m0, as they were read from tensor memory, to the row of an [n][W] dump at their feature indices.
 template <int W, int CH> __device__ __forceinline__ void dump_acc_chunk(int32_t *arow, int m0, const uint32_t (&v)[CH])
@@ -681,7 +734,7 @@ template <int W> __device__ __forceinline__ bool int_butterfly_across(SlotCtx &c
     return true;
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP, bool BOTH>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP, bool BOTH, bool CALIB>
 __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
@@ -808,6 +861,13 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
             layer1_chunk<W, CH, PER_TOKEN, ROT, DUMP, BOTH>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v, dY);
             tmem_st<CH>(c.taddr + ch * CH, v);
         }
+        if constexpr (CALIB) {
+            // calibration of layer p.L: the network is run up to that layer's rotated input
+            if (p.L == 2) {
+                if (!calib_finish<W, ROT>(c, valid, const_cast<float *>(p.layer[1].act))) return;
+                continue;
+            }
+        }
         if (!finish_layer<W, PER_TOKEN, ROT, DUMP>(c, next_s, next_inv, s_x, dC)) return;
         if constexpr (DUMP) {
             if (valid && sub == 0 && p.d.s_x[1]) p.d.s_x[1][tok] = s_x;
@@ -881,12 +941,18 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                 tmem_st<CH>(c.taddr + ch * CH, v);
             }
             if constexpr (DUMP) dC = (valid && p.d.codes[l]) ? p.d.codes[l] + tok * W : nullptr;
+            if constexpr (CALIB) {
+                if (l == p.L - 1) {
+                    if (!calib_finish<W, ROT>(c, valid, const_cast<float *>(p.layer[l].act))) return;
+                    continue;
+                }
+            }
             if (!finish_layer<W, PER_TOKEN, ROT, DUMP>(c, next_s, next_inv, s_x, dC)) return;
             if constexpr (DUMP) {
                 if (valid && sub == 0 && p.d.s_x[l]) p.d.s_x[l][tok] = s_x;
             }
         }
-        {
+        if constexpr (!CALIB) {
             const FusedLayer &ly = p.layer[p.L - 1];
             if (!wait_bar_warp<PER_TOKEN>(bar_last, last_parity, abort_flag, p.status)) return;
             last_parity ^= 1;
@@ -951,7 +1017,7 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
     if (!AHEAD && !C::BULK_XY && sub == 0 && c.row == 0) ptx::bulk_wait_all(); // the last tiles' stores
 }
 
-template <int W, bool SPREAD>
+template <int W, bool SPREAD, bool CALIB>
 __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, uint32_t tmem_base,
                          volatile int *abort_flag)
 {
@@ -1027,6 +1093,7 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
             }
         }
         if (!ok) break;
+        if constexpr (CALIB) continue; // the calibrated layer itself is not computed
         // last layer: N = 16, its weights stay in shared memory
         if (!wait_bar<0, kHintNs>(smem_base + sm.last_full, 0, abort_flag, p.status)) { ok = false; break; }
         for (int s = 0; s < active; ++s) {
@@ -1050,14 +1117,14 @@ __device__ void mma_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_
     }
 }
 
-template <int W, bool SPREAD>
+template <int W, bool SPREAD, bool CALIB>
 __device__ void load_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_base, volatile int *abort_flag)
 {
     using C = Cfg<W>;
     const uint32_t slab = C::PIECE_BYTES;
     // (test hook: with skip_last_weights set the copy is left out and nothing ever completes
     // last_full, so the waits for it run out, the abort path runs and the kernel returns)
-    if (!p.skip_last_weights) {
+    if (!p.skip_last_weights && !CALIB) {
         ptx::mbar_expect_tx(smem_base + sm.last_full, 16 * W);
         ptx::bulk_g2s(smem_base + sm.last_w, p.layer[p.L - 1].qw_umma, 16 * W, smem_base + sm.last_full);
     }
@@ -1127,7 +1194,7 @@ __device__ void xy_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_b
     }
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP = false, bool BOTH = false>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP = false, bool BOTH = false, bool CALIB = false>
 __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_constant__ ParamsOf<DUMP> p)
 {
     using C = Cfg<W>;
@@ -1200,11 +1267,11 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP, BOTH>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
+        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP, BOTH, CALIB>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
-        if (lane == 0) mma_role<W, SPREAD>(p, sm, smem_base, tmem_base, abort_flag);
+        if (lane == 0) mma_role<W, SPREAD, CALIB>(p, sm, smem_base, tmem_base, abort_flag);
     } else if (warp == kLoadWarp) {
-        if (lane == 0) load_role<W, SPREAD>(p, sm, smem_base, abort_flag);
+        if (lane == 0) load_role<W, SPREAD, CALIB>(p, sm, smem_base, abort_flag);
         if constexpr (DUMP) {
             // Observing instantiation only (in the timed kernels these few instructions cost 3-4 %): an
             // otherwise idle lane of CTA 0 notes the SM's cycle counter and the global nanosecond timer
@@ -1265,6 +1332,12 @@ template <int W> fused_dump_fn pick_both_dump_width(bool per_token)
 {
     return per_token ? fused_kernel<W, true, true, false, false, true, true> : fused_kernel<W, false, true, false, false, true, true>;
 }
+// Calibration kernels (per-tensor activation scales): the network up to the rotated input of layer
+// p.L, whose absmax they take.
+template <int W> fused_fn pick_calib_width(bool rot)
+{
+    return rot ? fused_kernel<W, false, true, false, false, false, false, true> : fused_kernel<W, false, false, false, false, false, false, true>;
+}
 // One translation unit per width (dhq_fused_w*.cu) instantiates the kernels of that width.
 fused_fn fused_pick_64(bool per_token, bool rot, bool spread, bool ahead);
 fused_fn fused_pick_128(bool per_token, bool rot, bool spread, bool ahead);
@@ -1274,6 +1347,10 @@ fused_dump_fn fused_pick_dump_64(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_128(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_256(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_512(bool per_token, bool rot);
+fused_fn fused_pick_calib_64(bool rot);
+fused_fn fused_pick_calib_128(bool rot);
+fused_fn fused_pick_calib_256(bool rot);
+fused_fn fused_pick_calib_512(bool rot);
 fused_fn fused_pick_both_64(bool per_token);
 fused_fn fused_pick_both_128(bool per_token);
 fused_fn fused_pick_both_256(bool per_token);

@@ -182,6 +182,9 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
 // Per-layer dump targets of the observing instantiation of the fused kernel: device pointers
 // laid out as dhq_debug_bufs_t describes, entry l-1 for layer l, NULL entries skipped.  X is only
 // used for layer 1; the input of a later layer is the output of the one before it.
+// One calibration pass of layer l (1-based) by the fused kernel; needs a fused handle with per-tensor
+// activation scales and not the two-sided transform.
+dhq_status_t fused_calibrate_layer(dhq_handle_s *h, int l, const float *coords, int64_t n, cudaStream_t st);
 struct DumpPtrs {
     float *X[kMaxLayers];
     int8_t *codes[kMaxLayers];

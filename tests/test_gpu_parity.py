@@ -502,3 +502,38 @@ def test_pipe_micro_benchmarks_run():
     for pipe in ("ffma", "mufu_sin", "tensor_i8", "pass1", "pass2", "pass12"):
         ops, ms = dhq.dhq_measure_pipe(pipe, 200)
         assert ops > 1e11 and ms > 0
+
+
+def test_two_handles_on_two_streams_at_once():
+    # Two networks, each on its own stream, launches interleaved without waiting: every launch wants
+    # all SMs and all of an SM's tensor memory, so the kernels queue behind each other on the device;
+    # results must equal the serial ones and no bounded wait may run out.
+    wa, wb = dhq_inputs.WORKLOADS["C2"], dhq_inputs.WORKLOADS["C3"]
+    weights_a, biases_a = wa.network()
+    weights_b, biases_b = wb.network()
+    ha, _ = prepare_pair(wa.dims, weights_a, biases_a, wa.omega0, 8, 8, 0, 0)
+    hb, _ = prepare_pair(wb.dims, weights_b, biases_b, wb.omega0, 8, 8, 1, 1)
+    try:
+        ca, cb = to_dev(wa.coords()), to_dev(wb.coords()[:100000])
+        dhq.dhq_calibrate(ha, ca)
+        ref_a = torch.empty((ca.shape[0], 3), device="cuda")
+        ref_b = torch.empty((cb.shape[0], 3), device="cuda")
+        dhq.dhq_forward(ha, ca, ref_a)
+        dhq.dhq_forward(hb, cb, ref_b)
+        torch.cuda.synchronize()
+        sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        outs_a = [torch.zeros_like(ref_a) for _ in range(6)]
+        outs_b = [torch.zeros_like(ref_b) for _ in range(6)]
+        for i in range(6):
+            dhq.dhq_forward(ha, ca, outs_a[i], stream=sa)
+            dhq.dhq_forward(hb, cb, outs_b[i], stream=sb)
+        sa.synchronize()
+        sb.synchronize()
+        assert dhq.dhq_last_status(ha) == 0 and dhq.dhq_last_status(hb) == 0
+        for o in outs_a:
+            assert torch.equal(o.view(torch.int32), ref_a.view(torch.int32))
+        for o in outs_b:
+            assert torch.equal(o.view(torch.int32), ref_b.view(torch.int32))
+    finally:
+        dhq.dhq_destroy(ha)
+        dhq.dhq_destroy(hb)
