@@ -41,12 +41,12 @@ import dhq_inputs  # noqa: E402
 # amount per coordinate, so it is scaled to the timed launch by the coordinate count.  An entry is
 # removed (traffic: null) when the kernel changes after its capture.
 NCU_DRAM_BYTES = {
-    ("C1", "input"): (100352, 4096),
-    ("C2", "input"): (787456, 65536),
-    ("C3", "input"): (2502656, 262144),
-    ("C4-W4A4", "input"): (2865152, 303104),
-    ("C4-W6A6", "input"): (2838784, 303104),
-    ("C5", "input"): (3345152, 303104),
+    ("C1", "input"): (101120, 4096),
+    ("C2", "input"): (782592, 65536),
+    ("C3", "input"): (2507264, 262144),
+    ("C4-W4A4", "input"): (2858496, 303104),
+    ("C4-W6A6", "input"): (2837504, 303104),
+    ("C5", "input"): (3344896, 303104),
 }
 METRIC = "coords/sec, fused W8A8 DHQ INR forward"
 UNIT = "coords/s"

@@ -396,3 +396,25 @@ def test_two_sided_network_converges_to_the_unquantized_siren():
     assert e12 < e8 / 4 and e16 < e12 / 4
     _, g16_one = _net_error(16, rotate=True)
     assert np.abs(g16 - g16_one).max() < 1e-3
+
+
+def test_two_sided_transform_makes_first_and_last_layer_weights_bell_shaped():
+    # Section III-B / Fig. 4: after the Hadamard transform the uniform first layer and the two-peaked
+    # last layer become bell-shaped.  Sanity statistic, not a parity gate: the excess kurtosis of the
+    # entries moves from the flat / two-peaked range (about -1.2 and below -1) to near 0 (Gaussian),
+    # while the input-side fold alone leaves a 2-input first layer as flat as it was (K = 4 mixes
+    # two values).
+    def excess_kurtosis(v):
+        v = np.asarray(v, dtype=np.float64).ravel()
+        v = v - v.mean()
+        return float((v ** 4).mean() / (v ** 2).mean() ** 2 - 3.0)
+    dims = (2, 256, 256, 256, 3)
+    weights, _ = dhq_inputs.trained_like_init(dims, 30.0, 5)
+    first = np.zeros((256, 4)); first[:, :2] = weights[0]
+    last = np.zeros((4, 256)); last[:3] = weights[-1]
+    assert excess_kurtosis(weights[0]) < -1.0                        # uniform
+    assert excess_kurtosis(weights[-1]) < -1.0                       # two peaks
+    k_first = excess_kurtosis(odef.transform_2d(first))
+    k_last = excess_kurtosis(odef.transform_2d(last))
+    assert abs(k_first) < 0.5 and abs(k_last) < 0.6
+    assert excess_kurtosis(odef.input_side_fold(first)[:, :2]) < -0.5
