@@ -104,9 +104,11 @@ typedef enum { DHQ_ROT_INPUT = 0, DHQ_ROT_BOTH = 1, DHQ_ROT_NONE = 2 } dhq_rot_t
 /* Activation of layers 1..L-1.  DHQ_ACT_SINE: sin(omega0 z), the SIREN of the paper's method
  * sections.  DHQ_ACT_GABOR: the real Gabor wavelet sin(omega0 z) exp(-(act_s0 z)^2), this
  * library's reading of the "wavelet activation" of the WIRE experiments (Section IV; the paper
- * gives no formula, the complex form of the WIRE paper is not built).  The wavelet runs layer by
- * layer (one kernel pass per layer), not in the fused kernel; it needs omega0 != 0, and the
- * floating-point datapaths, dhq_forward_fused_debug and dhq_forward_static_scratch do not take it. */
+ * gives no formula, the complex form of the WIRE paper is not built).  dhq_forward runs it inside
+ * the fused kernel (an instantiation whose epilogue multiplies the sine by the envelope; same
+ * arithmetic as the layer-by-layer kernel, so dhq_forward_debug agrees with it bit for bit);
+ * combined with DHQ_ROT_BOTH it runs layer by layer.  It needs omega0 != 0; the floating-point
+ * datapaths, dhq_forward_fused_debug and dhq_forward_static_scratch do not take it. */
 typedef enum { DHQ_ACT_SINE = 0, DHQ_ACT_GABOR = 1 } dhq_act_t;
 
 typedef struct {

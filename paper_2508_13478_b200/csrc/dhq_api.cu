@@ -171,7 +171,7 @@ LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X
 // layers < l run as they are frozen, is left in the layer's act[0] (not yet turned into scales).
 dhq_status_t calibrate_layer_pass(dhq_handle_s *h, int l, const float *coords, int64_t n, cudaStream_t st)
 {
-    if (h->fused && h->cfg.rotation != DHQ_ROT_BOTH && ((uintptr_t)coords & 7) == 0) {
+    if (h->fused && h->cfg.rotation != DHQ_ROT_BOTH && !(h->gabor_s0 > 0.0) && ((uintptr_t)coords & 7) == 0) {
         // the fused kernel run up to layer l's rotated input: one launch instead of l layer passes per
         // 64 Ki coordinates; same arithmetic, so the same maximum bit for bit
         CK(cudaMemsetAsync(h->layer[l - 1].act, 0, 4 * sizeof(float), st));
@@ -403,7 +403,9 @@ static dhq_status_t prepare_impl(const dhq_config_t *cfg, const float *const *W,
                                !gabor && !both) ? EPI_SINE_FAST : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;
-        if ((!both || both_fused) && !h->float_mode && !gabor) rc = fused_create(h); // the two-sided transform and the fp32 datapaths run layer by layer
+        // layer by layer: the fp32 datapaths, the two-sided transform with per-channel weight scales, and the
+        // wavelet combined with the two-sided transform
+        if ((!both || both_fused) && !h->float_mode && !(gabor && both)) rc = fused_create(h);
     } while (0);
     cudaFree(d_bounds);
     cudaFree(d_sums);
@@ -505,7 +507,7 @@ dhq_status_t dhq_forward_fused_debug(dhq_handle_t h, const float *coords, int64_
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
-    if (!h->fused) return DHQ_ERR_UNSUPPORTED; // run layer by layer: dhq_forward_debug observes them
+    if (!h->fused || h->gabor_s0 > 0.0) return DHQ_ERR_UNSUPPORTED; // run layer by layer, or no observing instantiation: dhq_forward_debug
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
     DumpPtrs d;

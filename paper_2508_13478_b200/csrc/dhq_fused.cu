@@ -19,6 +19,16 @@ static fused_fn pick_kernel(int W, bool per_token, bool rot, bool spread, bool a
     return nullptr;
 }
 
+static fused_fn pick_gabor_kernel(int W, bool per_token, bool rot)
+{
+    switch (W) {
+    case 64: return fused_pick_gabor_64(per_token, rot);
+    case 128: return fused_pick_gabor_128(per_token, rot);
+    case 256: return fused_pick_gabor_256(per_token, rot);
+    case 512: return fused_pick_gabor_512(per_token, rot);
+    }
+    return nullptr;
+}
 static fused_fn pick_calib_kernel(int W, bool rot)
 {
     switch (W) {
@@ -72,6 +82,8 @@ dhq_status_t fused_create(dhq_handle_s *h)
     p.qmaxf = (float)((1 << (h->cfg.a_bits - 1)) - 1);
     p.status = h->d_status;
     const bool both = h->cfg.rotation == DHQ_ROT_BOTH;
+    const bool gabor = h->gabor_s0 > 0.0;
+    p.gabor_c = gabor ? (float)(h->gabor_s0 / (double)h->cfg.omega0) : 0.f;
     int words = 0;
     for (int l = 0; l < h->L; ++l) {
         const LayerDev &d = h->layer[l];
@@ -90,7 +102,9 @@ dhq_status_t fused_create(dhq_handle_s *h)
         }
     }
     p.const_words = words;
-    fused_fn fn = both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false, false);
+    fused_fn fn = gabor ? pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+                  : both ? pick_both_kernel(h->w, p.per_token)
+                         : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false, false);
     if (!fn) return DHQ_ERR_UNSUPPORTED;
     int dev = 0, max_optin = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -113,17 +127,19 @@ dhq_status_t fused_create(dhq_handle_s *h)
     if (bytes < (size_t)kMinSmem) bytes = kMinSmem;
     fs->smem_bytes = bytes;
     for (int v = 0; v < 4; ++v) { // every variant of this handle's kernel
-        fused_fn f = both ? pick_both_kernel(h->w, p.per_token)
+        fused_fn f = gabor ? pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+                     : both ? pick_both_kernel(h->w, p.per_token)
                           : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, (v & 1) != 0, (v & 2) != 0);
         if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
-    if (!both && !p.per_token) {
+    if (!both && !gabor && !p.per_token) {
         fused_fn fc = pick_calib_kernel(h->w, h->cfg.rotation == DHQ_ROT_INPUT);
         if (!fc || cudaFuncSetAttribute(fc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
     fused_dump_fn fd = both ? pick_both_dump_kernel(h->w, p.per_token) : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    if (gabor) return DHQ_OK; // no observing instantiation for the wavelet: its per-layer dumps come from the layer-by-layer path
     if (!fd || cudaFuncSetAttribute(fd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
         return DHQ_ERR_CUDA;
     return DHQ_OK;
@@ -165,8 +181,10 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     }
     const int slots = (h->w == 512) ? 1 : 2;
     const bool both = h->cfg.rotation == DHQ_ROT_BOTH;
-    const bool spread = !both && slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
-    fused_fn fn = both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
+    const bool gabor = h->gabor_s0 > 0.0;
+    const bool spread = !both && !gabor && slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
+    fused_fn fn = gabor ? pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+                  : both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
@@ -194,7 +212,7 @@ __global__ void calib_l1_kernel(const float *coords, long long n, int rot, float
 dhq_status_t fused_calibrate_layer(dhq_handle_s *h, int l, const float *coords, int64_t n, cudaStream_t st)
 {
     FusedState *fs = static_cast<FusedState *>(h->fused);
-    if (!fs || fs->p.per_token || h->cfg.rotation == DHQ_ROT_BOTH || l < 1 || l > h->L) return DHQ_ERR_INVALID_ARG;
+    if (!fs || fs->p.per_token || h->cfg.rotation == DHQ_ROT_BOTH || h->gabor_s0 > 0.0 || l < 1 || l > h->L) return DHQ_ERR_INVALID_ARG;
     if (n <= 0) return DHQ_OK;
     if (l == 1) {
         const long long blocks = (n + 255) / 256;

@@ -116,6 +116,7 @@ struct FusedParams {
     unsigned long long wait_limit_ns; // every bounded wait gives up after this long (a handle setting)
     int skip_last_weights;            // test hook: the copy role leaves out the last layer's weights once
     FusedLayer layer[kMaxLayers];
+    float gabor_c;                    // wavelet activation: s0 / omega0 (read by the GABOR instantiations only)
 };
 
 struct FusedParamsDump : FusedParams {
@@ -418,8 +419,9 @@ template <int W> __device__ __forceinline__ void dump_y4(float *yrow, int col, f
 
 // Hidden layer: dequantize + bias + sine of the CH columns starting at column m0.  Constants come
 // from shared memory in column order: area A = cA, B = cB, C = cA_lo, each W words.
-template <int W, int CH, bool PER_TOKEN, bool ROT, int MODE, bool DUMP = false>
-__device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH], float *dump_y = nullptr)
+template <int W, int CH, bool PER_TOKEN, bool ROT, int MODE, bool DUMP = false, bool GABOR = false>
+__device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH], float *dump_y = nullptr,
+                                             float gabor_c = 0.f)
 {
     chunk_pipeline<CH, ROT>(v, [&](int j, f32x2 *out) {
 #pragma unroll
@@ -443,7 +445,8 @@ __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, 
                 for (int e = 0; e < 4; ++e) {
                     float c_hi = av[e], c_lo = lv[e];
                     if (PER_TOKEN) token_const(av[e], lv[e], s_x, c_hi, c_lo);
-                    y[e] = epilogue(MODE, (float)(int)v[i + e], c_hi, c_lo, bv[e]);
+                    y[e] = GABOR ? gabor_epilogue((float)(int)v[i + e], c_hi, c_lo, bv[e], gabor_c)
+                                 : epilogue(MODE, (float)(int)v[i + e], c_hi, c_lo, bv[e]);
                 }
                 out[2 * q] = pack2(y[0], y[1]);
                 out[2 * q + 1] = pack2(y[2], y[3]);
@@ -456,9 +459,9 @@ __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, 
 // Layer 1 for the CH columns starting at column m0.  Fixed-point mode: areas A = P, B = B, C = Q.
 // Float mode (per-token scales): A = cA, B = cB, C = cA_lo, D = the weight codes, one word per
 // column, and acc = dp4a(codes of the token, codes of the column's feature).
-template <int W, int CH, bool PER_TOKEN, bool ROT, bool DUMP = false, bool BOTH = false>
+template <int W, int CH, bool PER_TOKEN, bool ROT, bool DUMP = false, bool BOTH = false, bool GABOR = false>
 __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int qd, uint32_t qx, float s_x, uint32_t (&v)[CH],
-                                             float *dump_y = nullptr)
+                                             float *dump_y = nullptr, float gabor_c = 0.f)
 {
     chunk_pipeline<CH, ROT>(v, [&](int j, f32x2 *out) {
 #pragma unroll
@@ -469,7 +472,7 @@ __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int
             const float4 Cc = lds128(cbase + (2 * W + m0 + i) * 4);
             const float Av[4] = {A.x, A.y, A.z, A.w}, Bv[4] = {B.x, B.y, B.z, B.w}, Cv[4] = {Cc.x, Cc.y, Cc.z, Cc.w};
             float y[4];
-            if constexpr (!PER_TOKEN) {
+            if constexpr (!PER_TOKEN && !GABOR) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
                     y[e] = sine_fixed(qs, qd, __float_as_uint(Av[e]), __float_as_uint(Cv[e]), __float_as_uint(Bv[e]));
@@ -481,13 +484,14 @@ __device__ __forceinline__ void layer1_chunk(uint32_t cbase, int m0, int qs, int
                 const float wv2[4] = {wq2.x, wq2.y, wq2.z, wq2.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    float c_hi, c_lo;
-                    token_const(Av[e], Cv[e], s_x, c_hi, c_lo);
+                    float c_hi = Av[e], c_lo = Cv[e]; // per-tensor scale (wavelet route): the constants hold s_x already
+                    if (PER_TOKEN) token_const(Av[e], Cv[e], s_x, c_hi, c_lo);
                     // two-sided transform: areas D, E hold U' = H_M u and V' = H_M v (u, v: the sums of the weight
                     // codes that meet the two distinct input codes), so acc' = qs U' + qd V' needs no butterfly
                     const int acc = BOTH ? qs * (int)__float_as_uint(wv[e]) + qd * (int)__float_as_uint(wv2[e])
                                          : __dp4a((int)qx, (int)__float_as_uint(wv[e]), 0);
-                    y[e] = epilogue(EPI_SINE_WIDE, (float)acc, c_hi, c_lo, Bv[e]);
+                    // (the wavelet's envelope needs the unwrapped phase, which the fixed-point route does not have)
+                    y[e] = GABOR ? gabor_epilogue((float)acc, c_hi, c_lo, Bv[e], gabor_c) : epilogue(EPI_SINE_WIDE, (float)acc, c_hi, c_lo, Bv[e]);
                 }
             }
             out[2 * q] = pack2(y[0], y[1]);
@@ -734,7 +738,7 @@ template <int W> __device__ __forceinline__ bool int_butterfly_across(SlotCtx &c
     return true;
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP, bool BOTH, bool CALIB>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP, bool BOTH, bool CALIB, bool GABOR>
 __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
@@ -858,7 +862,7 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                     }
                 }
             }
-            layer1_chunk<W, CH, PER_TOKEN, ROT, DUMP, BOTH>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v, dY);
+            layer1_chunk<W, CH, PER_TOKEN, ROT, DUMP, BOTH, GABOR>(consts + l1.c_off * 4, ch * CH, qs, qd, qx, s_x, v, dY, p.gabor_c);
             tmem_st<CH>(c.taddr + ch * CH, v);
         }
         if constexpr (CALIB) {
@@ -937,7 +941,7 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                     if constexpr (!BOTH) dump_acc_chunk<W, CH>((valid && p.d.acc[l - 1]) ? p.d.acc[l - 1] + tok * W : nullptr, ch * CH, v);
                 }
                 if (fast) hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_FAST, DUMP>(cbase, ch * CH, s_x, v, dY);
-                else hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_WIDE, DUMP>(cbase, ch * CH, s_x, v, dY);
+                else hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_WIDE, DUMP, GABOR>(cbase, ch * CH, s_x, v, dY, p.gabor_c);
                 tmem_st<CH>(c.taddr + ch * CH, v);
             }
             if constexpr (DUMP) dC = (valid && p.d.codes[l]) ? p.d.codes[l] + tok * W : nullptr;
@@ -1194,7 +1198,8 @@ __device__ void xy_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_b
     }
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP = false, bool BOTH = false, bool CALIB = false>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP = false, bool BOTH = false, bool CALIB = false,
+          bool GABOR = false>
 __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_constant__ ParamsOf<DUMP> p)
 {
     using C = Cfg<W>;
@@ -1267,7 +1272,7 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP, BOTH, CALIB>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
+        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP, BOTH, CALIB, GABOR>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_role<W, SPREAD, CALIB>(p, sm, smem_base, tmem_base, abort_flag);
     } else if (warp == kLoadWarp) {
@@ -1338,6 +1343,14 @@ template <int W> fused_fn pick_calib_width(bool rot)
 {
     return rot ? fused_kernel<W, false, true, false, false, false, false, true> : fused_kernel<W, false, false, false, false, false, false, true>;
 }
+// The wavelet activation's kernels: not spread, coordinates not fetched ahead.
+template <int W> fused_fn pick_gabor_width(bool per_token, bool rot)
+{
+    if (rot) return per_token ? fused_kernel<W, true, true, false, false, false, false, false, true>
+                              : fused_kernel<W, false, true, false, false, false, false, false, true>;
+    return per_token ? fused_kernel<W, true, false, false, false, false, false, false, true>
+                     : fused_kernel<W, false, false, false, false, false, false, false, true>;
+}
 // One translation unit per width (dhq_fused_w*.cu) instantiates the kernels of that width.
 fused_fn fused_pick_64(bool per_token, bool rot, bool spread, bool ahead);
 fused_fn fused_pick_128(bool per_token, bool rot, bool spread, bool ahead);
@@ -1347,6 +1360,10 @@ fused_dump_fn fused_pick_dump_64(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_128(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_256(bool per_token, bool rot);
 fused_dump_fn fused_pick_dump_512(bool per_token, bool rot);
+fused_fn fused_pick_gabor_64(bool per_token, bool rot);
+fused_fn fused_pick_gabor_128(bool per_token, bool rot);
+fused_fn fused_pick_gabor_256(bool per_token, bool rot);
+fused_fn fused_pick_gabor_512(bool per_token, bool rot);
 fused_fn fused_pick_calib_64(bool rot);
 fused_fn fused_pick_calib_128(bool rot);
 fused_fn fused_pick_calib_256(bool rot);

@@ -9,5 +9,6 @@ fused_dump_fn fused_pick_dump_64(bool per_token, bool rot) { return pick_dump_wi
 fused_fn fused_pick_both_64(bool per_token) { return pick_both_width<64>(per_token); }
 fused_dump_fn fused_pick_both_dump_64(bool per_token) { return pick_both_dump_width<64>(per_token); }
 fused_fn fused_pick_calib_64(bool rot) { return pick_calib_width<64>(rot); }
+fused_fn fused_pick_gabor_64(bool per_token, bool rot) { return pick_gabor_width<64>(per_token, rot); }
 
 } // namespace dhq

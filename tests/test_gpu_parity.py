@@ -183,8 +183,9 @@ def test_two_sided_transform_wide_phases_host_buffers_and_static_scratch():
                                                   ("C5", 2000 + 5, True, 20.0)])
 def test_wavelet_activation_layer_by_layer(name, count, rotate, s0):
     # DHQ_ACT_GABOR: sin(omega0 z) exp(-(s0 z)^2) on layers 1..L-1 (the reading of the WIRE experiments'
-    # activation); integer stages bit-exact, outputs within 1e-5 of the fp64 definition; dhq_forward and
-    # the host-buffer route give the same bits as the per-layer dumps
+    # activation); integer stages bit-exact, outputs within 1e-5 of the fp64 definition on the per-layer
+    # dumps (layer-by-layer kernel); dhq_forward and the host-buffer route - the fused tensor-core kernel
+    # with the wavelet epilogue, except for the two-sided transform - give the same bits
     w = dhq_inputs.WORKLOADS[name]
     weights, biases = w.network()
     coords = w.coords()
