@@ -283,3 +283,37 @@ def test_two_sided_transform_with_per_channel_weight_scales_stays_layer_by_layer
         assert torch.isfinite(out).all() and dhq.dhq_last_status(h) == 0
     finally:
         dhq.dhq_destroy(h)
+
+
+@pytest.mark.skipif(not __import__("os").environ.get("DHQ_FULL_PARITY"), reason="every coordinate of the large grids through the oracle: "
+                    "minutes of CPU time per configuration; set DHQ_FULL_PARITY=1")
+@pytest.mark.parametrize("name", ["C4-W4A4", "C4-W6A6", "C5"])
+def test_every_coordinate_of_the_large_grids(name):
+    # All 1,048,576 (C4) / 4,194,304 (C5) coordinates through the observed fused kernel and the oracle,
+    # 65,536 at a time.  With per-tensor scales (C5) the frozen absmax of EVERY layer must equal the
+    # maximum of the oracle's rotated absmax over the whole grid (the kernel's own layer inputs).
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h, net = prepare_pair(w.dims, weights, biases, w.omega0, w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        check_weights(h, net)
+        coords = w.coords()
+        L = len(net.layers)
+        if w.a_gran == 0:
+            dhq.dhq_calibrate(h, to_dev(coords))
+        seen = np.zeros(L, np.float32)
+        worst = 0.0
+        for t0 in range(0, w.n, 65536):
+            chunk = np.ascontiguousarray(coords[t0:t0 + 65536])
+            cd = to_dev(chunk)
+            out_dump, bufs = run_debug(h, net, cd, fused=True)
+            worst = max(worst, check_layers_against_oracle(h, net, chunk, out_dump, bufs, calib_is_this_set=False))
+            if w.a_gran == 0:
+                for l in range(1, L + 1):
+                    seen[l - 1] = max(seen[l - 1], orc.rotated_absmax(net, l, bufs["X"][l - 1].cpu().numpy()).max())
+        if w.a_gran == 0:
+            frozen = np.array([dhq.dhq_get_layer(h, l)[2] for l in range(1, L + 1)], np.float32)
+            assert np.array_equal(frozen.view(np.uint32), seen.view(np.uint32)), (frozen, seen)
+        print(f"{name}: all {w.n} coordinates, integer stages exact, outputs within {worst:.2e}")
+    finally:
+        dhq.dhq_destroy(h)
