@@ -150,7 +150,8 @@ typedef struct {
  * Allocates device memory; enqueues the preparation kernels on `stream` and returns.  W and b
  * may be released once that stream work has completed.
  * Errors: INVALID_ARG (NULL, n_layers out of range), UNSUPPORTED (dims[0] != 2, width not a
- * power of two in 64..512 or not uniform, d_L outside 1..4, bits outside 2..8), ALLOC, CUDA.
+ * power of two in 64..512 or not uniform, d_L outside 1..4, a bit-width combination other than
+ * those listed at DHQ_BITS_FLOAT, unknown rotation or activation), ALLOC, CUDA.
  */
 DHQ_API dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W,
                                  const float *const *b, void *stream, dhq_handle_t *out);
