@@ -8,6 +8,7 @@
 //           z  = s_w[m] * sum_k q_w[m][k] x~_k + b[m]          (q_w exact in fp32)
 //   W32A32: z  = sum_k W[m][k] x_k + b[m]
 //   y = sin(omega0 z) for hidden layers (explicit 2 pi reduction), z for the last layer.
+#include <type_traits>
 #include "dhq_internal.cuh"
 
 namespace dhq {
@@ -41,39 +42,64 @@ __global__ void __launch_bounds__(FL_THREADS) float_layer_kernel(FloatLayerArgs 
     }
     __syncthreads();
     const int K4 = K / 4;
-    for (int m = tid; m < M; m += FL_THREADS) {
-        float acc[FTB];
+    // Each thread takes CPT output channels (m, m + FL_THREADS, ...) for all FTB tokens at once, so that one
+    // broadcast read of four activations feeds 4 * CPT multiply-adds (with one channel per pass the
+    // shared-memory reads, not the FMAs, set the pace).
+    auto run = [&](auto cpt_tag) {
+        constexpr int CPT = decltype(cpt_tag)::value;
+        for (int m0 = tid; m0 < M; m0 += FL_THREADS * CPT) {
+            float acc[CPT][FTB];
 #pragma unroll
-        for (int t = 0; t < FTB; ++t) acc[t] = 0.f;
-        for (int k4 = 0; k4 < K4; ++k4) {
-            float w0, w1, w2, w3;
-            if (a.w8) {
-                const uint32_t word = a.qw_k4m[(size_t)k4 * M + m]; // four consecutive-k codes of channel m
-                w0 = (float)(int8_t)(word & 0xff);
-                w1 = (float)(int8_t)((word >> 8) & 0xff);
-                w2 = (float)(int8_t)((word >> 16) & 0xff);
-                w3 = (float)(int8_t)(word >> 24);
-            } else {
-                const float4 w = a.w_f32[(size_t)k4 * M + m];
-                w0 = w.x; w1 = w.y; w2 = w.z; w3 = w.w;
+            for (int c = 0; c < CPT; ++c)
+#pragma unroll
+                for (int t = 0; t < FTB; ++t) acc[c][t] = 0.f;
+            for (int k4 = 0; k4 < K4; ++k4) {
+                float w[CPT][4];
+#pragma unroll
+                for (int c = 0; c < CPT; ++c) {
+                    const int m = m0 + c * FL_THREADS;
+                    if (m < M) {
+                        if (a.w8) {
+                            const uint32_t word = a.qw_k4m[(size_t)k4 * M + m]; // four consecutive-k codes of channel m
+                            w[c][0] = (float)(int8_t)(word & 0xff);
+                            w[c][1] = (float)(int8_t)((word >> 8) & 0xff);
+                            w[c][2] = (float)(int8_t)((word >> 16) & 0xff);
+                            w[c][3] = (float)(int8_t)(word >> 24);
+                        } else {
+                            const float4 wv = a.w_f32[(size_t)k4 * M + m];
+                            w[c][0] = wv.x; w[c][1] = wv.y; w[c][2] = wv.z; w[c][3] = wv.w;
+                        }
+                    } else {
+                        w[c][0] = w[c][1] = w[c][2] = w[c][3] = 0.f;
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < FTB; ++t) {
+                    const float4 x = *reinterpret_cast<const float4 *>(&xs[t * K + 4 * k4]);
+#pragma unroll
+                    for (int c = 0; c < CPT; ++c)
+                        acc[c][t] = __fmaf_rn(w[c][3], x.w, __fmaf_rn(w[c][2], x.z, __fmaf_rn(w[c][1], x.y, __fmaf_rn(w[c][0], x.x, acc[c][t]))));
+                }
             }
 #pragma unroll
-            for (int t = 0; t < FTB; ++t) {
-                const float4 x = *reinterpret_cast<const float4 *>(&xs[t * K + 4 * k4]);
-                acc[t] = __fmaf_rn(w3, x.w, __fmaf_rn(w2, x.z, __fmaf_rn(w1, x.y, __fmaf_rn(w0, x.x, acc[t]))));
+            for (int c = 0; c < CPT; ++c) {
+                const int m = m0 + c * FL_THREADS;
+                if (m >= M) continue;
+                const float bm = a.bias[m], sw = a.w8 ? a.s_w[m] : 1.0f;
+#pragma unroll
+                for (int t = 0; t < FTB; ++t) {
+                    const int64_t tok = base + t;
+                    if (tok >= a.n) continue;
+                    const float z = a.w8 ? __fmaf_rn(acc[c][t], sw, bm) : __fadd_rn(acc[c][t], bm);
+                    const float y = a.sine ? sin_wide(__fmul_rn(a.omega0, z)) : z;
+                    if (a.Y) a.Y[tok * M + m] = y;
+                    if (a.out && m < a.d_L) a.out[tok * a.d_L + m] = y;
+                }
             }
         }
-        const float bm = a.bias[m], sw = a.w8 ? a.s_w[m] : 1.0f;
-#pragma unroll
-        for (int t = 0; t < FTB; ++t) {
-            const int64_t tok = base + t;
-            if (tok >= a.n) continue;
-            const float z = a.w8 ? __fmaf_rn(acc[t], sw, bm) : __fadd_rn(acc[t], bm);
-            const float y = a.sine ? sin_wide(__fmul_rn(a.omega0, z)) : z;
-            if (a.Y) a.Y[tok * M + m] = y;
-            if (a.out && m < a.d_L) a.out[tok * a.d_L + m] = y;
-        }
-    }
+    };
+    if (M >= 2 * FL_THREADS) run(std::integral_constant<int, 2>());
+    else run(std::integral_constant<int, 1>());
 }
 
 // fp32 weights of one layer, zero padded to [M][K], as [K/4][M] float4 (four consecutive k of a
