@@ -41,12 +41,12 @@ import dhq_inputs  # noqa: E402
 # amount per coordinate, so it is scaled to the timed launch by the coordinate count.  An entry is
 # removed (traffic: null) when the kernel changes after its capture.
 NCU_DRAM_BYTES = {
-    ("C1", "input"): (101120, 4096),
-    ("C2", "input"): (782592, 65536),
-    ("C3", "input"): (2507264, 262144),
-    ("C4-W4A4", "input"): (2858496, 303104),
-    ("C4-W6A6", "input"): (2837504, 303104),
-    ("C5", "input"): (3344896, 303104),
+    ("C1", "input"): (100608, 4096),
+    ("C2", "input"): (784640, 65536),
+    ("C3", "input"): (2508544, 262144),
+    ("C4-W4A4", "input"): (2859776, 303104),
+    ("C4-W6A6", "input"): (2841344, 303104),
+    ("C5", "input"): (3344640, 303104),
 }
 METRIC = "coords/sec, fused W8A8 DHQ INR forward"
 UNIT = "coords/s"
@@ -184,7 +184,7 @@ def config_of(workload, args, world):
     mode = "one grid split over the ranks" if args.shard else "independent replica(s)"
     return {"workload": workload.name, "dims": list(workload.dims), "coords_per_step": workload.n if args.limit_coords <= 0 else min(workload.n, args.limit_coords),
             "bits": [workload.w_bits, workload.a_bits], "w_gran": workload.w_gran, "a_gran": workload.a_gran,
-            "rotation": args.rotation, "variant": args.variant, "l2": "flushed between steps (256 MB write)",
+            "rotation": args.rotation, "variant": args.variant, "activation": "gabor" if getattr(args, "gabor_s0", 0.0) > 0 else "sine", "l2": "flushed between steps (256 MB write)",
             "parallelism": f"{world} x {mode}"}
 
 
@@ -227,7 +227,7 @@ def aggregate_throughput(total_coords, ms_per_step):
 class Runner:
     """One workload on this rank's GPU: handle, device and pinned host buffers, timed loops."""
 
-    def __init__(self, dhq, workload, rotation, limit_coords=0, shard=None, group=None):
+    def __init__(self, dhq, workload, rotation, limit_coords=0, shard=None, group=None, gabor_s0=0.0):
         import torch
         self.dhq, self.torch, self.workload = dhq, torch, workload
         weights, biases = workload.network()
@@ -243,7 +243,8 @@ class Runner:
         self.h = dhq.dhq_prepare(workload.dims, [torch.from_numpy(w).cuda() for w in weights],
                                  [torch.from_numpy(b).cuda() for b in biases], workload.omega0, workload.w_bits,
                                  workload.a_bits, workload.w_gran, workload.a_gran,
-                                 rotation={"input": 0, "both": 1, "none": 2}[rotation])
+                                 rotation={"input": 0, "both": 1, "none": 2}[rotation],
+                                 activation=dhq.DHQ_ACT_GABOR if gabor_s0 > 0 else dhq.DHQ_ACT_SINE, act_s0=gabor_s0)
         self.coords = torch.from_numpy(coords_np).cuda()
         self.out = torch.empty((self.n, self.d_L), dtype=torch.float32, device="cuda")
         self.coords_host = torch.from_numpy(coords_np).pin_memory()
@@ -359,7 +360,7 @@ def run_ours(args, workload):
             dist.barrier()
         torch.cuda.synchronize()
 
-    run = Runner(dhq, workload, args.rotation, args.limit_coords, shard=(rank, world) if args.shard else None)
+    run = Runner(dhq, workload, args.rotation, args.limit_coords, shard=(rank, world) if args.shard else None, gabor_s0=args.gabor_s0)
     n = run.n
     warmup = max(args.warmup, 3)
     run.warm(warmup)
@@ -531,12 +532,17 @@ def main():
     ap.add_argument("--variant", default="w8a8", choices=["w8a8", "w8a32", "w32a32"],
                     help="datapath (Section I / Table 2 of the paper): the workload's fully quantized network, the same "
                          "with fp32 activations, or the plain fp32 network")
+    ap.add_argument("--gabor-s0", type=float, default=0.0,
+                    help="> 0: the wavelet activation sin(omega0 z) exp(-(s0 z)^2) instead of the sine (the WIRE reading)")
     ap.add_argument("--limit-coords", type=int, default=0,
                     help="use only the first N coordinates of the workload's grid (profiling captures)")
     ap.add_argument("--sweep", action="store_true", help="batch-size sweep 2^12..2^24 instead of the timed steps")
     ap.add_argument("--sweep-reps", type=int, default=20)
     args = ap.parse_args()
     workload = dhq_inputs.WORKLOADS[args.workload]
+    if args.gabor_s0 > 0:
+        args.no_per_config = True
+        args.no_cpu_baseline = True
     if args.variant != "w8a8":
         import dataclasses
         workload = dataclasses.replace(workload, w_bits=32 if args.variant == "w32a32" else workload.w_bits, a_bits=32)

@@ -40,7 +40,7 @@ def test_roofline_object_and_traffic_scaling():
 
 
 def test_config_object_is_the_same_for_both_arms_and_reference_line_is_complete():
-    args = types.SimpleNamespace(shard=False, limit_coords=0, rotation="input", variant="w8a8")
+    args = types.SimpleNamespace(shard=False, limit_coords=0, rotation="input", variant="w8a8", gabor_s0=0.0)
     w = dhq_inputs.WORKLOADS["C5"]
     cfg = bench.config_of(w, args, 1)
     assert cfg["workload"] == "C5" and cfg["coords_per_step"] == 4194304 and "model" not in cfg
