@@ -507,7 +507,7 @@ dhq_status_t dhq_forward_fused_debug(dhq_handle_t h, const float *coords, int64_
     if (!on_own_device(h)) return DHQ_ERR_INVALID_ARG;
     if (n == 0) return DHQ_OK;
     if (((uintptr_t)coords & 7) || ((uintptr_t)out & 3)) return DHQ_ERR_INVALID_ARG;
-    if (!h->fused || h->gabor_s0 > 0.0) return DHQ_ERR_UNSUPPORTED; // run layer by layer, or no observing instantiation: dhq_forward_debug
+    if (!h->fused) return DHQ_ERR_UNSUPPORTED; // this handle runs layer by layer: dhq_forward_debug
     if (!h->calibrated) return DHQ_ERR_NOT_CALIBRATED;
     cudaStream_t st = (cudaStream_t)stream;
     DumpPtrs d;

@@ -59,6 +59,17 @@ static fused_dump_fn pick_both_dump_kernel(int W, bool per_token)
     }
     return nullptr;
 }
+static fused_dump_fn pick_gabor_dump_kernel(int W, bool per_token, bool rot)
+{
+    switch (W) {
+    case 64: return fused_pick_gabor_dump_64(per_token, rot);
+    case 128: return fused_pick_gabor_dump_128(per_token, rot);
+    case 256: return fused_pick_gabor_dump_256(per_token, rot);
+    case 512: return fused_pick_gabor_dump_512(per_token, rot);
+    }
+    return nullptr;
+}
+
 static fused_dump_fn pick_dump_kernel(int W, bool per_token, bool rot)
 {
     switch (W) {
@@ -138,8 +149,9 @@ dhq_status_t fused_create(dhq_handle_s *h)
         if (!fc || cudaFuncSetAttribute(fc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
-    fused_dump_fn fd = both ? pick_both_dump_kernel(h->w, p.per_token) : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
-    if (gabor) return DHQ_OK; // no observing instantiation for the wavelet: its per-layer dumps come from the layer-by-layer path
+    fused_dump_fn fd = gabor ? pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+                       : both ? pick_both_dump_kernel(h->w, p.per_token)
+                              : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     if (!fd || cudaFuncSetAttribute(fd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
         return DHQ_ERR_CUDA;
     return DHQ_OK;
@@ -243,8 +255,9 @@ dhq_status_t fused_forward_dump(dhq_handle_s *h, const float *coords, int64_t n,
     fill_call(h, p, coords, n, out);
     p.d = d;
     const int slots = (h->w == 512) ? 1 : 2;
-    fused_dump_fn fn = h->cfg.rotation == DHQ_ROT_BOTH ? pick_both_dump_kernel(h->w, p.per_token)
-                                                        : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    fused_dump_fn fn = h->gabor_s0 > 0.0 ? pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+                       : h->cfg.rotation == DHQ_ROT_BOTH ? pick_both_dump_kernel(h->w, p.per_token)
+                                                         : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     const long long ctas = (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);

@@ -1351,6 +1351,13 @@ template <int W> fused_fn pick_gabor_width(bool per_token, bool rot)
     return per_token ? fused_kernel<W, true, false, false, false, false, false, false, true>
                      : fused_kernel<W, false, false, false, false, false, false, false, true>;
 }
+template <int W> fused_dump_fn pick_gabor_dump_width(bool per_token, bool rot)
+{
+    if (rot) return per_token ? fused_kernel<W, true, true, false, false, true, false, false, true>
+                              : fused_kernel<W, false, true, false, false, true, false, false, true>;
+    return per_token ? fused_kernel<W, true, false, false, false, true, false, false, true>
+                     : fused_kernel<W, false, false, false, false, true, false, false, true>;
+}
 // One translation unit per width (dhq_fused_w*.cu) instantiates the kernels of that width.
 fused_fn fused_pick_64(bool per_token, bool rot, bool spread, bool ahead);
 fused_fn fused_pick_128(bool per_token, bool rot, bool spread, bool ahead);
@@ -1364,6 +1371,10 @@ fused_fn fused_pick_gabor_64(bool per_token, bool rot);
 fused_fn fused_pick_gabor_128(bool per_token, bool rot);
 fused_fn fused_pick_gabor_256(bool per_token, bool rot);
 fused_fn fused_pick_gabor_512(bool per_token, bool rot);
+fused_dump_fn fused_pick_gabor_dump_64(bool per_token, bool rot);
+fused_dump_fn fused_pick_gabor_dump_128(bool per_token, bool rot);
+fused_dump_fn fused_pick_gabor_dump_256(bool per_token, bool rot);
+fused_dump_fn fused_pick_gabor_dump_512(bool per_token, bool rot);
 fused_fn fused_pick_calib_64(bool rot);
 fused_fn fused_pick_calib_128(bool rot);
 fused_fn fused_pick_calib_256(bool rot);

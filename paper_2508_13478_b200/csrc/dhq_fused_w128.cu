@@ -10,5 +10,6 @@ fused_fn fused_pick_both_128(bool per_token) { return pick_both_width<128>(per_t
 fused_dump_fn fused_pick_both_dump_128(bool per_token) { return pick_both_dump_width<128>(per_token); }
 fused_fn fused_pick_calib_128(bool rot) { return pick_calib_width<128>(rot); }
 fused_fn fused_pick_gabor_128(bool per_token, bool rot) { return pick_gabor_width<128>(per_token, rot); }
+fused_dump_fn fused_pick_gabor_dump_128(bool per_token, bool rot) { return pick_gabor_dump_width<128>(per_token, rot); }
 
 } // namespace dhq

@@ -10,5 +10,6 @@ fused_fn fused_pick_both_512(bool per_token) { return pick_both_width<512>(per_t
 fused_dump_fn fused_pick_both_dump_512(bool per_token) { return pick_both_dump_width<512>(per_token); }
 fused_fn fused_pick_calib_512(bool rot) { return pick_calib_width<512>(rot); }
 fused_fn fused_pick_gabor_512(bool per_token, bool rot) { return pick_gabor_width<512>(per_token, rot); }
+fused_dump_fn fused_pick_gabor_dump_512(bool per_token, bool rot) { return pick_gabor_dump_width<512>(per_token, rot); }
 
 } // namespace dhq
