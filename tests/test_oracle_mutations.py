@@ -138,3 +138,50 @@ def test_a_planted_mistake_fails_a_pin(name, old, new, tmp_path, swap_oracle_lib
     pin, err = _first_failure()
     assert pin is not None, f"no pin noticed the planted mistake '{name}'"
     print(f"{name}: caught by '{pin}'")
+
+
+# The oracle's Python driver (padding, chaining, calibration) gets the same treatment: one function
+# at a time is re-created from its source text with one mistake and put in the module's place.
+DRIVER_MUTATIONS = [
+    ("coordinates_padded_into_the_wrong_slots", "pad_coords", "X[:, : c.shape[1]] = c", "X[:, 4 - c.shape[1]:] = c"),
+    ("bias_padded_at_the_wrong_end", "prepare", "b_pad[:d_out] = _f32(biases[l - 1])", "b_pad[M_pad - d_out:] = _f32(biases[l - 1])"),
+    ("last_layer_marked_as_a_sine_layer", "prepare", "sine=(l < L)", "sine=True"),
+    ("padded_sizes_of_the_last_layer_not_applied", "pad_dims", "M_pad = 4 if l == L else int(dims[l])", "M_pad = 4 if l == 1 else int(dims[l])"),
+    ("calibration_takes_the_mean", "calibrate", "rotated_absmax(net, l, X).max()", "rotated_absmax(net, l, X).mean()"),
+    ("calibration_does_not_advance_through_the_layers", "calibrate",
+     'X = layer(net, l, X, want=("Y",))["Y"].astype(np.float32)', "X = np.zeros((X.shape[0], net.layers[l].K_pad), np.float32) + X[:, :1]"),
+    ("granularity_flag_inverted", "layer", "per_token = int(net.a_gran == 1)", "per_token = int(net.a_gran == 0)"),
+    ("forward_returns_the_wrong_output_columns", "forward", 'out = r["Y"][:, : net.dims[-1]]', 'out = r["Y"][:, -net.dims[-1]:]'),
+    ("chain_not_rounded_to_fp32_inputs_but_restarted", "forward", 'X = r["Y"].astype(np.float32)', 'X = np.abs(r["Y"]).astype(np.float32)'),
+]
+
+
+def _driver_battery():
+    return [
+        ("padding of first and last layer", pins.test_first_layer_pads_coordinates_and_last_layer_pads_outputs),
+        ("brute force, 2 bits", lambda: pins.test_brute_force_all_code_vectors_on_a_4_wide_layer(2)),
+        ("integer matmul and sine", pins.test_integer_matmul_matches_int64_product_and_hidden_layers_apply_sine),
+        ("calibration", pins.test_per_tensor_calibration_is_the_layerwise_maximum_and_freezes),
+        ("zero token", pins.test_zero_token_has_zero_codes_per_token),
+        ("two tiers", lambda: tiers.test_fp32_oracle_codes_agree_with_the_fp64_orthonormal_statement("C1", 4096, 0, 0)),
+        ("convergence", pins.test_quantized_network_converges_to_the_unquantized_siren),
+    ]
+
+
+@pytest.mark.parametrize("name,fn_name,old,new", DRIVER_MUTATIONS, ids=[m[0] for m in DRIVER_MUTATIONS])
+def test_a_planted_mistake_in_the_driver_fails_a_pin(name, fn_name, old, new, monkeypatch):
+    import inspect
+    src = inspect.getsource(getattr(orc, fn_name))
+    assert src.count(old) == 1, "the text to mutate must occur exactly once in the function"
+    made = {}
+    exec(compile(src.replace(old, new), f"<{fn_name} with a planted mistake>", "exec"), orc.__dict__, made)
+    monkeypatch.setattr(orc, fn_name, made[fn_name])
+    caught = None
+    for pin_name, pin in _driver_battery():
+        try:
+            pin()
+        except (AssertionError, ValueError, IndexError, RuntimeError, OverflowError):
+            caught = pin_name
+            break
+    assert caught is not None, f"no pin noticed the planted mistake '{name}'"
+    print(f"{name}: caught by '{caught}'")
