@@ -241,6 +241,27 @@ def test_free_running_chains_differ_only_through_code_flips_at_rounding_ties():
         dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("width,a_gran", [(64, 0), (128, 1), (256, 0), (256, 1), (512, 0), (512, 1)])
+@pytest.mark.parametrize("n_linear", [2, 3, 16])
+def test_depths_from_one_hidden_layer_to_the_maximum(n_linear, width, a_gran):
+    # L = 2 has no hidden layer on the tensor core (layer 1 on the CUDA cores, then the N = 16 last
+    # layer), L = 3 one; 16 (the library's maximum) no longer keeps its weights resident in shared
+    # memory at width 256 and leaves the width-512 ring few stages beside the per-layer constants
+    dims = (2,) + (width,) * (n_linear - 1) + (3,)
+    wl = dhq_inputs.Workload("depth", dims, 30.0, 1300 + width + n_linear, 8, 8, a_gran, a_gran, (8, 8))
+    n = 148 * (1 if width == 512 else 2) * 128 + 77
+    coords = dhq_inputs.grid_coords(233, 171)[:n]
+    weights, biases = wl.network()
+    h, net = prepare_pair(wl.dims, weights, biases, wl.omega0, 8, 8, a_gran, a_gran)
+    try:
+        check_weights(h, net)
+        if a_gran == 0:
+            dhq.dhq_calibrate(h, to_dev(coords))
+        _observe(h, net, coords)
+    finally:
+        dhq.dhq_destroy(h)
+
+
 @pytest.mark.parametrize("rotate", [True, False])
 @pytest.mark.parametrize("width,a_gran,s0", [(64, 0, 6.0), (64, 1, 6.0), (128, 0, 9.0), (256, 0, 12.0), (256, 1, 12.0), (512, 0, 20.0), (512, 1, 20.0)])
 def test_wavelet_activation_inside_the_fused_kernel(width, a_gran, s0, rotate):
