@@ -241,6 +241,34 @@ def test_free_running_chains_differ_only_through_code_flips_at_rounding_ties():
         dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("w_bits,a_bits,d_out,omega0,width,gran", [
+    (2, 2, 3, 30.0, 256, 0), (2, 2, 1, 30.0, 128, 1), (3, 5, 2, 30.0, 64, 1), (4, 8, 4, 30.0, 256, 1), (8, 4, 3, 30.0, 512, 0),
+    (7, 7, 4, 30.0, 512, 1), (8, 8, 2, -30.0, 256, 0), (8, 8, 3, 1.0, 128, 0), (8, 8, 1, 75.0, 256, 1), (8, 8, 3, 75.0, 512, 0),
+    (6, 8, 3, 0.0, 256, 0), (8, 8, 3, 0.0, 64, 1)])
+def test_unequal_bit_widths_output_sizes_and_other_frequencies(w_bits, a_bits, d_out, omega0, width, gran):
+    # every supported bit-width pair is a pair of 2..8; d_L is 1..4 (padded to 4); omega0 any finite
+    # number: negative, small (phases of a fraction of a radian), large (phases of a hundred radians:
+    # the explicit-reduction sine) and zero (every hidden activation is sin(0) = 0, so every later
+    # layer sees the degenerate absmax 0 and the output is the last bias)
+    dims = (2, width, width, width, d_out)
+    wl = dhq_inputs.Workload("mix", dims, 30.0, 1700 + w_bits * 10 + a_bits + d_out, w_bits, a_bits, gran, gran, (8, 8))
+    n = 148 * (1 if width == 512 else 2) * 128 + 41
+    coords = dhq_inputs.grid_coords(229, 173)[:n]
+    weights, biases = wl.network()
+    h, net = prepare_pair(dims, weights, biases, omega0, w_bits, a_bits, gran, gran)
+    try:
+        check_weights(h, net)
+        if gran == 0:
+            dhq.dhq_calibrate(h, to_dev(coords))
+        _observe(h, net, coords)
+        if omega0 == 0.0:
+            out = torch.empty((n, d_out), device="cuda")
+            dhq.dhq_forward(h, to_dev(coords), out)
+            assert torch.equal(out, torch.from_numpy(biases[-1]).cuda().expand(n, d_out))
+    finally:
+        dhq.dhq_destroy(h)
+
+
 @pytest.mark.parametrize("width,a_gran", [(64, 0), (128, 1), (256, 0), (256, 1), (512, 0), (512, 1)])
 @pytest.mark.parametrize("n_linear", [2, 3, 16])
 def test_depths_from_one_hidden_layer_to_the_maximum(n_linear, width, a_gran):
