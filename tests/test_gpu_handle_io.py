@@ -60,6 +60,44 @@ def test_export_import_round_trip_is_bit_identical(name):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("name,kw", [
+    ("C2", dict(rotation=1)),                                   # two-sided transform inside the fused kernel (H_M u, H_M v travel too)
+    ("C3", dict(rotation=1)),                                   # two-sided, per-channel scales: layer by layer
+    ("C2", dict(rotation=2)),                                   # no rotation
+    ("C2", dict(activation=1, act_s0=9.0)),                     # wavelet activation
+    ("C5", dict(activation=1, act_s0=20.0, rotation=2)),
+    ("C2", dict(a_bits=32)),                                    # W8A32
+    ("C2", dict(w_bits=32, a_bits=32)),                         # W32A32 (fp32 weights travel)
+    ("C4-W4A4", dict()),
+])
+def test_export_import_round_trip_of_the_other_datapaths(name, kw):
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    args = dict(w_bits=w.w_bits, a_bits=w.a_bits, w_gran=w.w_gran, a_gran=w.a_gran)
+    args.update(kw)
+    h = dhq.dhq_prepare(w.dims, [to_dev(x) for x in weights], [to_dev(x) for x in biases], w.omega0, **args)
+    h2 = None
+    try:
+        coords = to_dev(w.coords()[: 20000 + 13])
+        dhq.dhq_calibrate(h, coords)
+        blob = dhq.dhq_export(h)
+        h2 = dhq.dhq_import(blob)
+        out1 = torch.empty((coords.shape[0], w.dims[-1]), device="cuda")
+        out2 = torch.full_like(out1, float("nan"))
+        dhq.dhq_forward(h, coords, out1)
+        dhq.dhq_forward(h2, coords, out2)
+        torch.cuda.synchronize()
+        assert dhq.dhq_last_status(h2) == 0
+        assert torch.isfinite(out1).all()
+        assert torch.equal(out1.view(torch.int32), out2.view(torch.int32))
+        assert dhq.dhq_export(h2) == blob
+    finally:
+        dhq.dhq_destroy(h)
+        if h2:
+            dhq.dhq_destroy(h2)
+
+
+@pytest.mark.gpu
 def test_call_log_is_written_when_asked_for():
     # DHQ_LOG is read once per process: run a small forward in a child process
     import os
