@@ -107,8 +107,9 @@ typedef enum { DHQ_ROT_INPUT = 0, DHQ_ROT_BOTH = 1, DHQ_ROT_NONE = 2 } dhq_rot_t
  * gives no formula, the complex form of the WIRE paper is not built).  dhq_forward runs it inside
  * the fused kernel (an instantiation whose epilogue multiplies the sine by the envelope; same
  * arithmetic as the layer-by-layer kernel, so dhq_forward_debug agrees with it bit for bit);
- * dhq_forward_fused_debug observes that instantiation's per-layer values; combined with
- * DHQ_ROT_BOTH it runs layer by layer.  It needs omega0 != 0; the floating-point datapaths and
+ * dhq_forward_fused_debug observes that instantiation's per-layer values; DHQ_ROT_BOTH combines
+ * with it under the same rule as for the sine (fused with one weight scale per tensor, else
+ * layer by layer).  It needs omega0 != 0; the floating-point datapaths and
  * dhq_forward_static_scratch do not take it. */
 typedef enum { DHQ_ACT_SINE = 0, DHQ_ACT_GABOR = 1 } dhq_act_t;
 
@@ -252,7 +253,7 @@ DHQ_API dhq_status_t dhq_forward_debug(dhq_handle_t h, const float *coords, int6
  *          input codes); acc[0] holds codes . weight codes computed for the dump.
  *          X[0] must be 16-byte aligned, the other buffers 4-byte aligned.
  * Requires frozen scales when a_gran = per tensor (NOT_CALIBRATED otherwise).  A handle that runs
- * layer by layer (DHQ_ROT_BOTH with per-channel weight scales or with the wavelet activation, the
+ * layer by layer (DHQ_ROT_BOTH with per-channel weight scales, the
  * floating-point datapaths) is observed by dhq_forward_debug: UNSUPPORTED here.
  * Errors: INVALID_ARG, UNSUPPORTED, NOT_CALIBRATED, CUDA.
  */

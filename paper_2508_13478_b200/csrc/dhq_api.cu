@@ -390,7 +390,7 @@ static dhq_status_t prepare_impl(const dhq_config_t *cfg, const float *const *W,
             cudaStreamSynchronize(st) != cudaSuccess) { rc = DHQ_ERR_CUDA; break; }
         // Two-sided transform in the fused kernel: the output-side rotation runs on the int32 accumulators,
         // which needs one weight scale per tensor and |H_M acc| <= sum_m |acc_m| <= qmax_a * sum |q_w| < 2^31.
-        bool both_fused = both && cfg->w_gran == DHQ_GRAN_TENSOR && !gabor && !h->float_mode;
+        bool both_fused = both && cfg->w_gran == DHQ_GRAN_TENSOR && !h->float_mode;
         for (int l = 1; l <= L && both_fused; ++l)
             if (sums[l - 1] * (unsigned long long)((1 << (cfg->a_bits - 1)) - 1) >= (1ull << 31)) both_fused = false;
         for (int l = 1; l <= L; ++l) {
@@ -405,7 +405,7 @@ static dhq_status_t prepare_impl(const dhq_config_t *cfg, const float *const *W,
         h->calibrated = per_token;
         // layer by layer: the fp32 datapaths, the two-sided transform with per-channel weight scales, and the
         // wavelet combined with the two-sided transform
-        if ((!both || both_fused) && !h->float_mode && !(gabor && both)) rc = fused_create(h);
+        if ((!both || both_fused) && !h->float_mode) rc = fused_create(h);
     } while (0);
     cudaFree(d_bounds);
     cudaFree(d_sums);

@@ -59,6 +59,28 @@ static fused_dump_fn pick_both_dump_kernel(int W, bool per_token)
     }
     return nullptr;
 }
+static fused_fn pick_gabor_both_kernel(int W, bool per_token)
+{
+    switch (W) {
+    case 64: return fused_pick_gabor_both_64(per_token);
+    case 128: return fused_pick_gabor_both_128(per_token);
+    case 256: return fused_pick_gabor_both_256(per_token);
+    case 512: return fused_pick_gabor_both_512(per_token);
+    }
+    return nullptr;
+}
+
+static fused_dump_fn pick_gabor_both_dump_kernel(int W, bool per_token)
+{
+    switch (W) {
+    case 64: return fused_pick_gabor_both_dump_64(per_token);
+    case 128: return fused_pick_gabor_both_dump_128(per_token);
+    case 256: return fused_pick_gabor_both_dump_256(per_token);
+    case 512: return fused_pick_gabor_both_dump_512(per_token);
+    }
+    return nullptr;
+}
+
 static fused_dump_fn pick_gabor_dump_kernel(int W, bool per_token, bool rot)
 {
     switch (W) {
@@ -113,7 +135,7 @@ dhq_status_t fused_create(dhq_handle_s *h)
         }
     }
     p.const_words = words;
-    fused_fn fn = gabor ? pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+    fused_fn fn = gabor ? (both ? pick_gabor_both_kernel(h->w, p.per_token) : pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
                   : both ? pick_both_kernel(h->w, p.per_token)
                          : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false, false);
     if (!fn) return DHQ_ERR_UNSUPPORTED;
@@ -138,7 +160,7 @@ dhq_status_t fused_create(dhq_handle_s *h)
     if (bytes < (size_t)kMinSmem) bytes = kMinSmem;
     fs->smem_bytes = bytes;
     for (int v = 0; v < 4; ++v) { // every variant of this handle's kernel
-        fused_fn f = gabor ? pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+        fused_fn f = gabor ? (both ? pick_gabor_both_kernel(h->w, p.per_token) : pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
                      : both ? pick_both_kernel(h->w, p.per_token)
                           : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, (v & 1) != 0, (v & 2) != 0);
         if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
@@ -149,7 +171,7 @@ dhq_status_t fused_create(dhq_handle_s *h)
         if (!fc || cudaFuncSetAttribute(fc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
-    fused_dump_fn fd = gabor ? pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+    fused_dump_fn fd = gabor ? (both ? pick_gabor_both_dump_kernel(h->w, p.per_token) : pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
                        : both ? pick_both_dump_kernel(h->w, p.per_token)
                               : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     if (!fd || cudaFuncSetAttribute(fd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
@@ -195,7 +217,7 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     const bool both = h->cfg.rotation == DHQ_ROT_BOTH;
     const bool gabor = h->gabor_s0 > 0.0;
     const bool spread = !both && !gabor && slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
-    fused_fn fn = gabor ? pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+    fused_fn fn = gabor ? (both ? pick_gabor_both_kernel(h->w, p.per_token) : pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
                   : both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
@@ -256,7 +278,7 @@ dhq_status_t fused_forward_dump(dhq_handle_s *h, const float *coords, int64_t n,
     fill_call(h, p, coords, n, out);
     p.d = d;
     const int slots = (h->w == 512) ? 1 : 2;
-    fused_dump_fn fn = h->gabor_s0 > 0.0 ? pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT)
+    fused_dump_fn fn = h->gabor_s0 > 0.0 ? (h->cfg.rotation == DHQ_ROT_BOTH ? pick_gabor_both_dump_kernel(h->w, p.per_token) : pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
                        : h->cfg.rotation == DHQ_ROT_BOTH ? pick_both_dump_kernel(h->w, p.per_token)
                                                          : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
     const long long ctas = (p.n_tiles + slots - 1) / slots;

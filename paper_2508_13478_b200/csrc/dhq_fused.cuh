@@ -1352,6 +1352,15 @@ template <int W> fused_fn pick_gabor_width(bool per_token, bool rot)
     return per_token ? fused_kernel<W, true, false, false, false, false, false, false, true>
                      : fused_kernel<W, false, false, false, false, false, false, false, true>;
 }
+// The wavelet activation with the two-sided transform.
+template <int W> fused_fn pick_gabor_both_width(bool per_token)
+{
+    return per_token ? fused_kernel<W, true, true, false, false, false, true, false, true> : fused_kernel<W, false, true, false, false, false, true, false, true>;
+}
+template <int W> fused_dump_fn pick_gabor_both_dump_width(bool per_token)
+{
+    return per_token ? fused_kernel<W, true, true, false, false, true, true, false, true> : fused_kernel<W, false, true, false, false, true, true, false, true>;
+}
 template <int W> fused_dump_fn pick_gabor_dump_width(bool per_token, bool rot)
 {
     if (rot) return per_token ? fused_kernel<W, true, true, false, false, true, false, false, true>
@@ -1372,6 +1381,14 @@ fused_fn fused_pick_gabor_64(bool per_token, bool rot);
 fused_fn fused_pick_gabor_128(bool per_token, bool rot);
 fused_fn fused_pick_gabor_256(bool per_token, bool rot);
 fused_fn fused_pick_gabor_512(bool per_token, bool rot);
+fused_fn fused_pick_gabor_both_64(bool per_token);
+fused_fn fused_pick_gabor_both_128(bool per_token);
+fused_fn fused_pick_gabor_both_256(bool per_token);
+fused_fn fused_pick_gabor_both_512(bool per_token);
+fused_dump_fn fused_pick_gabor_both_dump_64(bool per_token);
+fused_dump_fn fused_pick_gabor_both_dump_128(bool per_token);
+fused_dump_fn fused_pick_gabor_both_dump_256(bool per_token);
+fused_dump_fn fused_pick_gabor_both_dump_512(bool per_token);
 fused_dump_fn fused_pick_gabor_dump_64(bool per_token, bool rot);
 fused_dump_fn fused_pick_gabor_dump_128(bool per_token, bool rot);
 fused_dump_fn fused_pick_gabor_dump_256(bool per_token, bool rot);

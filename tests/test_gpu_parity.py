@@ -179,13 +179,14 @@ def test_two_sided_transform_wide_phases_host_buffers_and_static_scratch():
 
 
 @pytest.mark.parametrize("name,count,rotate,s0", [("C1", 4096, True, 8.0), ("C2", 7000 + 3, True, 12.0), ("C3", 5000 + 1, True, 5.0),
-                                                  ("C4-W4A4", 3000 + 7, True, 10.0), ("C2", 4000, False, 12.0), ("C2", 4000, "both", 6.0),
+                                                  ("C4-W4A4", 3000 + 7, True, 10.0), ("C2", 4000, False, 12.0), ("C2", 4000, "both", 6.0), ("C3", 3000, "both", 6.0),
                                                   ("C5", 2000 + 5, True, 20.0)])
 def test_wavelet_activation_layer_by_layer(name, count, rotate, s0):
     # DHQ_ACT_GABOR: sin(omega0 z) exp(-(s0 z)^2) on layers 1..L-1 (the reading of the WIRE experiments'
     # activation); integer stages bit-exact, outputs within 1e-5 of the fp64 definition on the per-layer
     # dumps (layer-by-layer kernel); dhq_forward and the host-buffer route - the fused tensor-core kernel
-    # with the wavelet epilogue, except for the two-sided transform - give the same bits
+    # with the wavelet epilogue, except for the two-sided transform with per-channel weight scales - give
+    # the same bits (two-sided: within 1e-5 of the definition on each route, fp64 against fp32 epilogue)
     w = dhq_inputs.WORKLOADS[name]
     weights, biases = w.network()
     coords = w.coords()
@@ -203,19 +204,26 @@ def test_wavelet_activation_layer_by_layer(name, count, rotate, s0):
         oh = torch.zeros(out.shape).pin_memory()
         dhq.dhq_forward_host(h, torch.from_numpy(coords).pin_memory(), oh)
         torch.cuda.synchronize()
-        assert torch.equal(out.view(torch.int32), out_dbg.view(torch.int32))
-        assert torch.equal(oh.view(torch.int32), out_dbg.cpu().view(torch.int32))
+        if rotate == "both" and w.w_gran == 0:
+            # fused two-sided route (integer H_M, fp32 epilogue) against the layer-by-layer one (fp64 H_M):
+            # each layer within 1e-5 of the definition on either route, but not the same bits, and the
+            # free-running chains then part at rounding ties; the fused route is checked layer by layer below
+            assert torch.equal(oh.view(torch.int32), out.cpu().view(torch.int32))
+        else:
+            assert torch.equal(out.view(torch.int32), out_dbg.view(torch.int32))
+            assert torch.equal(oh.view(torch.int32), out_dbg.cpu().view(torch.int32))
         # the envelope is really applied: the hidden activations differ from the plain sine's
         y1 = bufs["Y"][0].cpu().numpy()
         assert np.abs(y1).max() <= 1.0 and np.abs(y1).mean() < 0.6
         print(f"gabor {name} rotate={rotate}: outputs within {worst:.2e}")
-        if rotate == "both":   # the combination runs layer by layer: nothing fused to observe
+        if rotate == "both" and w.w_gran == 1:   # two-sided with per-channel weight scales runs layer by layer: nothing fused to observe
             with pytest.raises(dhq.DhqError) as e:
                 dhq.dhq_forward_fused_debug(h, cd, out)
             assert e.value.code == 2
         else:                  # the fused kernel's own per-layer values, same checks
             out_obs, bufs_obs = run_debug(h, net, cd, fused=True)
-            check_layers_against_oracle(h, net, coords, out_obs, bufs_obs)
+            # (two-sided: the frozen maxima were taken on the layer-by-layer route's activations)
+            check_layers_against_oracle(h, net, coords, out_obs, bufs_obs, calib_is_this_set=(rotate != "both"))
             assert torch.equal(out_obs.view(torch.int32), out.view(torch.int32))
     finally:
         dhq.dhq_destroy(h)
