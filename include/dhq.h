@@ -166,7 +166,7 @@ DHQ_API dhq_status_t dhq_prepare(const dhq_config_t *cfg, const float *const *W,
  * not depend on the batch it arrives in).
  *   coords device [n][2] fp32, n >= 1.
  * Enqueues L passes on `stream` (one launch of the fused kernel per layer, run up to that layer's
- * rotated input; layer-by-layer kernels for DHQ_ROT_BOTH).  With a_gran = per
+ * rotated input; layer-by-layer kernels for handles without a fused kernel).  With a_gran = per
  * token the call is a no-op returning DHQ_OK.
  * Errors: INVALID_ARG, ALLOC, CUDA.
  */

@@ -171,7 +171,7 @@ LayerArgs layer_args(dhq_handle_s *h, int l, const float *coords, const float *X
 // layers < l run as they are frozen, is left in the layer's act[0] (not yet turned into scales).
 dhq_status_t calibrate_layer_pass(dhq_handle_s *h, int l, const float *coords, int64_t n, cudaStream_t st)
 {
-    if (h->fused && h->cfg.rotation != DHQ_ROT_BOTH && ((uintptr_t)coords & 7) == 0) {
+    if (h->fused && ((uintptr_t)coords & 7) == 0) {
         // the fused kernel run up to layer l's rotated input: one launch instead of l layer passes per
         // 64 Ki coordinates; same arithmetic, so the same maximum bit for bit
         CK(cudaMemsetAsync(h->layer[l - 1].act, 0, 4 * sizeof(float), st));

@@ -29,13 +29,13 @@ static fused_fn pick_gabor_kernel(int W, bool per_token, bool rot)
     }
     return nullptr;
 }
-static fused_fn pick_calib_kernel(int W, bool rot, bool gabor)
+static fused_fn pick_calib_kernel(int W, bool rot, bool gabor, bool both)
 {
     switch (W) {
-    case 64: return fused_pick_calib_64(rot, gabor);
-    case 128: return fused_pick_calib_128(rot, gabor);
-    case 256: return fused_pick_calib_256(rot, gabor);
-    case 512: return fused_pick_calib_512(rot, gabor);
+    case 64: return fused_pick_calib_64(rot, gabor, both);
+    case 128: return fused_pick_calib_128(rot, gabor, both);
+    case 256: return fused_pick_calib_256(rot, gabor, both);
+    case 512: return fused_pick_calib_512(rot, gabor, both);
     }
     return nullptr;
 }
@@ -166,8 +166,8 @@ dhq_status_t fused_create(dhq_handle_s *h)
         if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
-    if (!both && !p.per_token) {
-        fused_fn fc = pick_calib_kernel(h->w, h->cfg.rotation == DHQ_ROT_INPUT, gabor);
+    if (!p.per_token) {
+        fused_fn fc = pick_calib_kernel(h->w, h->cfg.rotation == DHQ_ROT_INPUT, gabor, both);
         if (!fc || cudaFuncSetAttribute(fc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
@@ -242,16 +242,16 @@ __global__ void calib_l1_kernel(const float *coords, long long n, int rot, float
 
 // One calibration pass by the fused kernel: the maximum of |rotated input of layer l| over the
 // coordinates, with layers < l run as they are frozen, is accumulated into the layer's act[0]
-// (which the caller has cleared).  Per-tensor activation scales, one-sided or no rotation, either
-// activation.
+// (which the caller has cleared).  Per-tensor activation scales; every rotation mode and activation
+// that has a fused kernel.
 dhq_status_t fused_calibrate_layer(dhq_handle_s *h, int l, const float *coords, int64_t n, cudaStream_t st)
 {
     FusedState *fs = static_cast<FusedState *>(h->fused);
-    if (!fs || fs->p.per_token || h->cfg.rotation == DHQ_ROT_BOTH || l < 1 || l > h->L) return DHQ_ERR_INVALID_ARG;
+    if (!fs || fs->p.per_token || l < 1 || l > h->L) return DHQ_ERR_INVALID_ARG;
     if (n <= 0) return DHQ_OK;
     if (l == 1) {
         const long long blocks = (n + 255) / 256;
-        calib_l1_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), 256, 0, st>>>(coords, n, h->cfg.rotation == DHQ_ROT_INPUT, h->layer[0].act);
+        calib_l1_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), 256, 0, st>>>(coords, n, h->cfg.rotation != DHQ_ROT_NONE, h->layer[0].act);
         h->launches++;
         return cudaGetLastError() == cudaSuccess ? DHQ_OK : DHQ_ERR_CUDA;
     }
@@ -259,7 +259,7 @@ dhq_status_t fused_calibrate_layer(dhq_handle_s *h, int l, const float *coords, 
     fill_call(h, p, coords, n, nullptr);
     p.L = l; // the network up to the rotated input of layer l
     const int slots = (h->w == 512) ? 1 : 2;
-    fused_fn fn = pick_calib_kernel(h->w, h->cfg.rotation == DHQ_ROT_INPUT, h->gabor_s0 > 0.0);
+    fused_fn fn = pick_calib_kernel(h->w, h->cfg.rotation == DHQ_ROT_INPUT, h->gabor_s0 > 0.0, h->cfg.rotation == DHQ_ROT_BOTH);
     const long long ctas = (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);

@@ -1339,8 +1339,9 @@ template <int W> fused_dump_fn pick_both_dump_width(bool per_token)
 }
 // Calibration kernels (per-tensor activation scales): the network up to the rotated input of layer
 // p.L, whose absmax they take.
-template <int W> fused_fn pick_calib_width(bool rot, bool gabor)
+template <int W> fused_fn pick_calib_width(bool rot, bool gabor, bool both)
 {
+    if (both) return gabor ? fused_kernel<W, false, true, false, false, false, true, true, true> : fused_kernel<W, false, true, false, false, false, true, true, false>;
     if (gabor) return rot ? fused_kernel<W, false, true, false, false, false, false, true, true> : fused_kernel<W, false, false, false, false, false, false, true, true>;
     return rot ? fused_kernel<W, false, true, false, false, false, false, true> : fused_kernel<W, false, false, false, false, false, false, true>;
 }
@@ -1393,10 +1394,10 @@ fused_dump_fn fused_pick_gabor_dump_64(bool per_token, bool rot);
 fused_dump_fn fused_pick_gabor_dump_128(bool per_token, bool rot);
 fused_dump_fn fused_pick_gabor_dump_256(bool per_token, bool rot);
 fused_dump_fn fused_pick_gabor_dump_512(bool per_token, bool rot);
-fused_fn fused_pick_calib_64(bool rot, bool gabor);
-fused_fn fused_pick_calib_128(bool rot, bool gabor);
-fused_fn fused_pick_calib_256(bool rot, bool gabor);
-fused_fn fused_pick_calib_512(bool rot, bool gabor);
+fused_fn fused_pick_calib_64(bool rot, bool gabor, bool both);
+fused_fn fused_pick_calib_128(bool rot, bool gabor, bool both);
+fused_fn fused_pick_calib_256(bool rot, bool gabor, bool both);
+fused_fn fused_pick_calib_512(bool rot, bool gabor, bool both);
 fused_fn fused_pick_both_64(bool per_token);
 fused_fn fused_pick_both_128(bool per_token);
 fused_fn fused_pick_both_256(bool per_token);

@@ -8,7 +8,7 @@ fused_fn fused_pick_256(bool per_token, bool rot, bool spread, bool ahead) { ret
 fused_dump_fn fused_pick_dump_256(bool per_token, bool rot) { return pick_dump_width<256, true>(per_token, rot); }
 fused_fn fused_pick_both_256(bool per_token) { return pick_both_width<256>(per_token); }
 fused_dump_fn fused_pick_both_dump_256(bool per_token) { return pick_both_dump_width<256>(per_token); }
-fused_fn fused_pick_calib_256(bool rot, bool gabor) { return pick_calib_width<256>(rot, gabor); }
+fused_fn fused_pick_calib_256(bool rot, bool gabor, bool both) { return pick_calib_width<256>(rot, gabor, both); }
 fused_fn fused_pick_gabor_256(bool per_token, bool rot) { return pick_gabor_width<256>(per_token, rot); }
 fused_dump_fn fused_pick_gabor_dump_256(bool per_token, bool rot) { return pick_gabor_dump_width<256>(per_token, rot); }
 fused_fn fused_pick_gabor_both_256(bool per_token) { return pick_gabor_both_width<256>(per_token); }

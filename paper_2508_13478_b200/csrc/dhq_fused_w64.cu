@@ -8,7 +8,7 @@ fused_fn fused_pick_64(bool per_token, bool rot, bool spread, bool ahead) { retu
 fused_dump_fn fused_pick_dump_64(bool per_token, bool rot) { return pick_dump_width<64, true>(per_token, rot); }
 fused_fn fused_pick_both_64(bool per_token) { return pick_both_width<64>(per_token); }
 fused_dump_fn fused_pick_both_dump_64(bool per_token) { return pick_both_dump_width<64>(per_token); }
-fused_fn fused_pick_calib_64(bool rot, bool gabor) { return pick_calib_width<64>(rot, gabor); }
+fused_fn fused_pick_calib_64(bool rot, bool gabor, bool both) { return pick_calib_width<64>(rot, gabor, both); }
 fused_fn fused_pick_gabor_64(bool per_token, bool rot) { return pick_gabor_width<64>(per_token, rot); }
 fused_dump_fn fused_pick_gabor_dump_64(bool per_token, bool rot) { return pick_gabor_dump_width<64>(per_token, rot); }
 fused_fn fused_pick_gabor_both_64(bool per_token) { return pick_gabor_both_width<64>(per_token); }

@@ -307,9 +307,7 @@ def test_wavelet_activation_inside_the_fused_kernel(width, a_gran, s0, rotate):
         check_weights(h, net)
         if a_gran == 0:
             dhq.dhq_calibrate(h, to_dev(coords))
-        # (two-sided: the calibration runs layer by layer with the fp64 H_M, so the frozen maxima belong to
-        # that route's activations, which differ from the fused route's in the last bits)
-        worst = _observe(h, net, coords, calib_is_this_set=(rotate != "both"))
+        worst = _observe(h, net, coords)
         print(f"wavelet, width {width}, a_gran {a_gran}, rotate {rotate}: outputs within {worst:.2e}")
     finally:
         dhq.dhq_destroy(h)
@@ -329,7 +327,7 @@ def test_two_sided_transform_inside_the_fused_kernel(width, a_gran):
         check_weights(h, net)
         if a_gran == 0:
             dhq.dhq_calibrate(h, to_dev(coords))
-        worst = _observe(h, net, coords, calib_is_this_set=False)
+        worst = _observe(h, net, coords)   # the frozen maxima too: the calibration runs the same kernel
         # the host-buffer route runs the same kernel
         oh = torch.zeros((n, 3)).pin_memory()
         dhq.dhq_forward_host(h, torch.from_numpy(coords).pin_memory(), oh)
