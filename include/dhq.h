@@ -205,6 +205,9 @@ DHQ_API dhq_status_t dhq_set_act_absmax(dhq_handle_t h, int layer, float absmax,
  * activation scales and none are frozen yet, this call first calibrates on its own coordinates
  * (as dhq_calibrate) and freezes them; later calls reuse them.
  * Non-finite coordinates give unspecified values but do not hang.
+ * On a handle with a fused kernel and frozen (or per-token) scales the call enqueues that one
+ * launch and nothing else - no allocation, no synchronisation - so it may be recorded by stream
+ * capture into a CUDA graph and replayed on new contents of the same buffers.
  * Errors: INVALID_ARG, ALLOC, CUDA.
  */
 DHQ_API dhq_status_t dhq_forward(dhq_handle_t h, const float *coords, int64_t n, float *out,

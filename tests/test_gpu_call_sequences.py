@@ -94,3 +94,46 @@ def test_every_route_returns_the_reference_bits(case):
         dhq.dhq_destroy(h)
         for x in imported:
             dhq.dhq_destroy(x)
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C5"])
+def test_forward_can_be_captured_in_a_cuda_graph_and_replayed(name):
+    # A serving loop captures the launch once and replays it on new coordinates in the same buffers.
+    # dhq_forward on a calibrated handle enqueues only the fused kernel (no allocation, no synchronisation),
+    # so stream capture takes it; the replays must give the bits of plain calls.
+    w = dhq_inputs.WORKLOADS[name]
+    weights, biases = w.network()
+    h = dhq.dhq_prepare(w.dims, [to_dev(x) for x in weights], [to_dev(x) for x in biases], w.omega0,
+                        w.w_bits, w.a_bits, w.w_gran, w.a_gran)
+    try:
+        grid = w.coords()
+        n = min(20000, grid.shape[0] // 3)
+        dhq.dhq_calibrate(h, to_dev(grid[::7]))
+        batches = [to_dev(grid[i * n:(i + 1) * n]) for i in range(3)]
+        want = []
+        for b in batches:
+            o = torch.empty((n, w.dims[-1]), device="cuda")
+            dhq.dhq_forward(h, b, o)
+            want.append(o)
+        torch.cuda.synchronize()
+        buf_in = batches[0].clone()
+        buf_out = torch.full((n, w.dims[-1]), float("nan"), device="cuda")
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            dhq.dhq_forward(h, buf_in, buf_out, stream=side)          # warm-up on the capture stream
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                dhq.dhq_forward(h, buf_in, buf_out, stream=torch.cuda.current_stream())
+        launches = dhq.dhq_launch_count(h)
+        for b, o in zip(batches, want):
+            buf_in.copy_(b)
+            buf_out.fill_(float("nan"))
+            graph.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(buf_out.view(torch.int32), o.view(torch.int32))
+        assert dhq.dhq_launch_count(h) == launches                    # replays go through no library call
+        assert dhq.dhq_last_status(h) == 0
+    finally:
+        dhq.dhq_destroy(h)
