@@ -41,12 +41,12 @@ import dhq_inputs  # noqa: E402
 # amount per coordinate, so it is scaled to the timed launch by the coordinate count.  An entry is
 # removed (traffic: null) when the kernel changes after its capture.
 NCU_DRAM_BYTES = {
-    ("C1", "input"): (100608, 4096),
-    ("C2", "input"): (784640, 65536),
-    ("C3", "input"): (2508544, 262144),
-    ("C4-W4A4", "input"): (2859776, 303104),
-    ("C4-W6A6", "input"): (2841344, 303104),
-    ("C5", "input"): (3344640, 303104),
+    ("C1", "input"): (99328, 4096),
+    ("C2", "input"): (782080, 65536),
+    ("C3", "input"): (2504704, 262144),
+    ("C4-W4A4", "input"): (2875648, 303104),
+    ("C4-W6A6", "input"): (2835968, 303104),
+    ("C5", "input"): (3344896, 303104),
 }
 METRIC = "coords/sec, fused W8A8 DHQ INR forward"
 UNIT = "coords/s"

@@ -124,7 +124,7 @@ struct BlobHeader {
     float phase_bound[kMaxLayers];
     uint64_t payload_bytes, payload_fnv1a;
 };
-constexpr uint32_t kBlobVersion = 3;
+constexpr uint32_t kBlobVersion = 4;
 const char kBlobMagic[8] = {'D', 'H', 'Q', 'B', '2', '0', '0', 0};
 
 uint64_t fnv1a(const uint8_t *p, size_t n)
@@ -393,14 +393,17 @@ static dhq_status_t prepare_impl(const dhq_config_t *cfg, const float *const *W,
         bool both_fused = both && cfg->w_gran == DHQ_GRAN_TENSOR && !h->float_mode;
         for (int l = 1; l <= L && both_fused; ++l)
             if (sums[l - 1] * (unsigned long long)((1 << (cfg->a_bits - 1)) - 1) >= (1ull << 31)) both_fused = false;
+        const bool a_per_token = cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN;
         for (int l = 1; l <= L; ++l) {
             LayerDev &d = h->layer[l - 1];
             d.phase_bound = bounds[l - 1];
             if (l == L) d.epi_mode = EPI_LINEAR;
             else if (l == 1) {}
             // (two-sided: the quantization error of all M rows meets in every output; no tight phase bound)
-            else d.epi_mode = (bounds[l - 1] <= (cfg->a_gran == DHQ_GRAN_CHANNEL_OR_TOKEN ? kFastPhaseLimitPerToken : kFastPhaseLimit) &&
-                               !gabor && !both) ? EPI_SINE_FAST : EPI_SINE_WIDE;
+            else if (bounds[l - 1] <= (a_per_token ? kFastPhaseLimitPerToken : kFastPhaseLimit) && !gabor && !both) d.epi_mode = EPI_SINE_FAST;
+            // no bound below the limit: the values that are below it still take the short route (the kernels
+            // with a per-token scale and the fused two-sided ones carry that variant)
+            else d.epi_mode = (!gabor && !h->float_mode && ((a_per_token && !both) || both_fused)) ? EPI_SINE_MIXED : EPI_SINE_WIDE;
         }
         h->calibrated = per_token;
         // layer by layer: the fp32 datapaths, the two-sided transform with per-channel weight scales, and the
@@ -734,7 +737,7 @@ dhq_status_t dhq_import(const void *host_buf, int64_t bytes, void *stream, dhq_h
         layer_arrays(d, t);
         for (const ArrayRef &a : t) payload += a.bytes;
         const int e = hd.epi_mode[l - 1];
-        if (e < EPI_LINEAR || e > EPI_BOTH) { delete h; return DHQ_ERR_INVALID_ARG; }
+        if (e < EPI_LINEAR || e > EPI_SINE_MIXED) { delete h; return DHQ_ERR_INVALID_ARG; }
         d.epi_mode = e;
         d.phase_bound = hd.phase_bound[l - 1];
     }

@@ -103,6 +103,58 @@ static fused_dump_fn pick_dump_kernel(int W, bool per_token, bool rot)
     return nullptr;
 }
 
+static fused_fn pick_mixed_kernel(int W, bool rot, bool ahead)
+{
+    switch (W) {
+    case 64: return fused_pick_mixed_64(rot, ahead);
+    case 128: return fused_pick_mixed_128(rot, ahead);
+    case 256: return fused_pick_mixed_256(rot, ahead);
+    case 512: return fused_pick_mixed_512(rot, ahead);
+    }
+    return nullptr;
+}
+
+static fused_dump_fn pick_mixed_dump_kernel(int W, bool rot)
+{
+    switch (W) {
+    case 64: return fused_pick_mixed_dump_64(rot);
+    case 128: return fused_pick_mixed_dump_128(rot);
+    case 256: return fused_pick_mixed_dump_256(rot);
+    case 512: return fused_pick_mixed_dump_512(rot);
+    }
+    return nullptr;
+}
+
+// Per-token scales, one-sided or no rotation, sine, and a hidden layer under EPI_SINE_MIXED: the handle
+// runs the instantiations that carry that variant.
+static bool runs_mixed(const dhq_handle_s *h)
+{
+    if (h->cfg.a_gran != DHQ_GRAN_CHANNEL_OR_TOKEN || h->cfg.rotation == DHQ_ROT_BOTH || h->gabor_s0 > 0.0) return false;
+    for (int l = 0; l < h->L; ++l)
+        if (h->layer[l].epi_mode == EPI_SINE_MIXED) return true;
+    return false;
+}
+
+// The kernel a handle's forward launches (spread, ahead: see pick_kernel; the other families have one mapping).
+static fused_fn pick_for(const dhq_handle_s *h, bool per_token, bool spread, bool ahead)
+{
+    const bool both = h->cfg.rotation == DHQ_ROT_BOTH, rot = h->cfg.rotation == DHQ_ROT_INPUT;
+    if (h->gabor_s0 > 0.0) return both ? pick_gabor_both_kernel(h->w, per_token) : pick_gabor_kernel(h->w, per_token, rot);
+    if (both) return pick_both_kernel(h->w, per_token);
+    if (runs_mixed(h)) return pick_mixed_kernel(h->w, rot, ahead);
+    return pick_kernel(h->w, per_token, rot, spread, ahead);
+}
+
+// Its observing instantiation.
+static fused_dump_fn pick_dump_for(const dhq_handle_s *h, bool per_token)
+{
+    const bool both = h->cfg.rotation == DHQ_ROT_BOTH, rot = h->cfg.rotation == DHQ_ROT_INPUT;
+    if (h->gabor_s0 > 0.0) return both ? pick_gabor_both_dump_kernel(h->w, per_token) : pick_gabor_dump_kernel(h->w, per_token, rot);
+    if (both) return pick_both_dump_kernel(h->w, per_token);
+    if (runs_mixed(h)) return pick_mixed_dump_kernel(h->w, rot);
+    return pick_dump_kernel(h->w, per_token, rot);
+}
+
 dhq_status_t fused_create(dhq_handle_s *h)
 {
     FusedState *fs = new (std::nothrow) FusedState();
@@ -130,14 +182,12 @@ dhq_status_t fused_create(dhq_handle_s *h)
         f.epi_mode = d.epi_mode;
         f.c_off = words;
         if (l < h->L - 1) {
-            int areas = (l == 0) ? (d.epi_mode == EPI_SINE_FIXED ? 3 : (both ? 5 : 4)) : (d.epi_mode == EPI_SINE_WIDE ? 3 : 2);
+            int areas = (l == 0) ? (d.epi_mode == EPI_SINE_FIXED ? 3 : (both ? 5 : 4)) : ((d.epi_mode == EPI_SINE_WIDE || d.epi_mode == EPI_SINE_MIXED) ? 3 : 2);
             words += areas * h->w;
         }
     }
     p.const_words = words;
-    fused_fn fn = gabor ? (both ? pick_gabor_both_kernel(h->w, p.per_token) : pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
-                  : both ? pick_both_kernel(h->w, p.per_token)
-                         : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, false, false);
+    fused_fn fn = pick_for(h, p.per_token, false, false);
     if (!fn) return DHQ_ERR_UNSUPPORTED;
     int dev = 0, max_optin = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -160,9 +210,7 @@ dhq_status_t fused_create(dhq_handle_s *h)
     if (bytes < (size_t)kMinSmem) bytes = kMinSmem;
     fs->smem_bytes = bytes;
     for (int v = 0; v < 4; ++v) { // every variant of this handle's kernel
-        fused_fn f = gabor ? (both ? pick_gabor_both_kernel(h->w, p.per_token) : pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
-                     : both ? pick_both_kernel(h->w, p.per_token)
-                          : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, (v & 1) != 0, (v & 2) != 0);
+        fused_fn f = pick_for(h, p.per_token, (v & 1) != 0, (v & 2) != 0);
         if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
@@ -171,9 +219,7 @@ dhq_status_t fused_create(dhq_handle_s *h)
         if (!fc || cudaFuncSetAttribute(fc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return DHQ_ERR_CUDA;
     }
-    fused_dump_fn fd = gabor ? (both ? pick_gabor_both_dump_kernel(h->w, p.per_token) : pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
-                       : both ? pick_both_dump_kernel(h->w, p.per_token)
-                              : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    fused_dump_fn fd = pick_dump_for(h, p.per_token);
     if (!fd || cudaFuncSetAttribute(fd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
         return DHQ_ERR_CUDA;
     return DHQ_OK;
@@ -216,9 +262,8 @@ dhq_status_t fused_forward(dhq_handle_s *h, const float *coords, int64_t n, floa
     const int slots = (h->w == 512) ? 1 : 2;
     const bool both = h->cfg.rotation == DHQ_ROT_BOTH;
     const bool gabor = h->gabor_s0 > 0.0;
-    const bool spread = !both && !gabor && slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
-    fused_fn fn = gabor ? (both ? pick_gabor_both_kernel(h->w, p.per_token) : pick_gabor_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
-                  : both ? pick_both_kernel(h->w, p.per_token) : pick_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT, spread, !on_host);
+    const bool spread = !both && !gabor && !runs_mixed(h) && slots > 1 && p.n_tiles < (long long)fs->sm_count * slots;
+    fused_fn fn = pick_for(h, p.per_token, spread, !on_host);
     const long long ctas = spread ? p.n_tiles : (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);
@@ -278,9 +323,7 @@ dhq_status_t fused_forward_dump(dhq_handle_s *h, const float *coords, int64_t n,
     fill_call(h, p, coords, n, out);
     p.d = d;
     const int slots = (h->w == 512) ? 1 : 2;
-    fused_dump_fn fn = h->gabor_s0 > 0.0 ? (h->cfg.rotation == DHQ_ROT_BOTH ? pick_gabor_both_dump_kernel(h->w, p.per_token) : pick_gabor_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT))
-                       : h->cfg.rotation == DHQ_ROT_BOTH ? pick_both_dump_kernel(h->w, p.per_token)
-                                                         : pick_dump_kernel(h->w, p.per_token, h->cfg.rotation == DHQ_ROT_INPUT);
+    fused_dump_fn fn = pick_dump_for(h, p.per_token);
     const long long ctas = (p.n_tiles + slots - 1) / slots;
     int grid = (int)(ctas < fs->sm_count ? ctas : fs->sm_count);
     fn<<<grid, h->w == 512 ? kThreads + 32 : kThreads, fs->smem_bytes, st>>>(p);

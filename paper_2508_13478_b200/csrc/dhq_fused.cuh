@@ -419,10 +419,13 @@ template <int W> __device__ __forceinline__ void dump_y4(float *yrow, int col, f
 
 // Hidden layer: dequantize + bias + sine of the CH columns starting at column m0.  Constants come
 // from shared memory in column order: area A = cA, B = cB, C = cA_lo, each W words.
-template <int W, int CH, bool PER_TOKEN, bool ROT, int MODE, bool DUMP = false, bool GABOR = false>
+// TRACK (with EPI_SINE_FAST): *xmax receives the largest |phase| the thread met, for the caller's decision
+// whether the chunk has to be redone under EPI_SINE_MIXED.  LIMIT: the limit of EPI_SINE_MIXED.
+template <int W, int CH, bool PER_TOKEN, bool ROT, int MODE, bool DUMP = false, bool GABOR = false, bool TRACK = false>
 __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, uint32_t (&v)[CH], float *dump_y = nullptr,
-                                             float gabor_c = 0.f)
+                                             float gabor_c = 0.f, [[maybe_unused]] float *xmax = nullptr, [[maybe_unused]] float limit = 0.f)
 {
+    [[maybe_unused]] float xm = 0.f;
     chunk_pipeline<CH, ROT>(v, [&](int j, f32x2 *out) {
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
@@ -434,19 +437,28 @@ __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, 
                 float x0, x1, x2, x3;
                 unpack2(fma2(pack2((float)(int)v[i], (float)(int)v[i + 1]), pack2(a.x, a.y), pack2(b.x, b.y)), x0, x1);
                 unpack2(fma2(pack2((float)(int)v[i + 2], (float)(int)v[i + 3]), pack2(a.z, a.w), pack2(b.z, b.w)), x2, x3);
+                if constexpr (TRACK) xm = fmaxf(xm, fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3))));
                 out[2 * q] = pack2(sin_approx(x0), sin_approx(x1));
                 out[2 * q + 1] = pack2(sin_approx(x2), sin_approx(x3));
             } else {
                 float4 lo = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (MODE == EPI_SINE_WIDE) lo = lds128(cbase + (2 * W + m0 + i) * 4);
+                if (MODE == EPI_SINE_WIDE || MODE == EPI_SINE_MIXED) lo = lds128(cbase + (2 * W + m0 + i) * 4);
                 const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w}, lv[4] = {lo.x, lo.y, lo.z, lo.w};
                 float y[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     float c_hi = av[e], c_lo = lv[e];
                     if (PER_TOKEN) token_const(av[e], lv[e], s_x, c_hi, c_lo);
-                    y[e] = GABOR ? gabor_epilogue((float)(int)v[i + e], c_hi, c_lo, bv[e], gabor_c)
-                                 : epilogue(MODE, (float)(int)v[i + e], c_hi, c_lo, bv[e]);
+                    if constexpr (TRACK) { // EPI_SINE_FAST, keeping the phase
+                        const float x = __fmaf_rn((float)(int)v[i + e], c_hi, bv[e]);
+                        xm = fmaxf(xm, fabsf(x));
+                        y[e] = sin_approx(x);
+                    } else if constexpr (MODE == EPI_SINE_MIXED) {
+                        y[e] = epilogue_mixed((float)(int)v[i + e], c_hi, c_lo, bv[e], limit);
+                    } else {
+                        y[e] = GABOR ? gabor_epilogue((float)(int)v[i + e], c_hi, c_lo, bv[e], gabor_c)
+                                     : epilogue(MODE, (float)(int)v[i + e], c_hi, c_lo, bv[e]);
+                    }
                 }
                 out[2 * q] = pack2(y[0], y[1]);
                 out[2 * q + 1] = pack2(y[2], y[3]);
@@ -454,6 +466,7 @@ __device__ __forceinline__ void hidden_chunk(uint32_t cbase, int m0, float s_x, 
             if constexpr (DUMP) dump_y4<W>(dump_y, m0 + i, out[2 * q], out[2 * q + 1]);
         }
     });
+    if constexpr (TRACK) *xmax = xm;
 }
 
 // Layer 1 for the CH columns starting at column m0.  Fixed-point mode: areas A = P, B = B, C = Q.
@@ -738,7 +751,7 @@ template <int W> __device__ __forceinline__ bool int_butterfly_across(SlotCtx &c
     return true;
 }
 
-template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP, bool BOTH, bool CALIB, bool GABOR>
+template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP, bool BOTH, bool CALIB, bool GABOR, bool MIXED>
 __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32_t smem_base, int warp, int lane,
                               uint32_t tmem_base, volatile int *abort_flag)
 {
@@ -940,8 +953,29 @@ __device__ void epilogue_role(const ParamsOf<DUMP> &p, const SmemMap &sm, uint32
                     dY = (valid && p.d.Y[l - 1]) ? p.d.Y[l - 1] + tok * W : nullptr;
                     if constexpr (!BOTH) dump_acc_chunk<W, CH>((valid && p.d.acc[l - 1]) ? p.d.acc[l - 1] + tok * W : nullptr, ch * CH, v);
                 }
-                if (fast) hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_FAST, DUMP>(cbase, ch * CH, s_x, v, dY);
-                else hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_WIDE, DUMP, GABOR>(cbase, ch * CH, s_x, v, dY, p.gabor_c);
+                if (fast) {
+                    hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_FAST, DUMP>(cbase, ch * CH, s_x, v, dY);
+                } else {
+                    [[maybe_unused]] bool done = false;
+                    if constexpr ((MIXED || BOTH) && !GABOR) {
+                        if (ly.epi_mode == EPI_SINE_MIXED) {
+                            // No bound says that the short route is accurate enough for this layer, but the phases
+                            // that are actually met mostly are: take it, keep the largest |phase|, and redo the
+                            // chunk value by value (accumulators are still in tensor memory) only if a warp met one
+                            // beyond the limit.  The per-value rule gives the same bits either way.
+                            constexpr float kLimit = BOTH ? kMixedPhaseLimitBoth : PER_TOKEN ? kFastPhaseLimitPerToken : kFastPhaseLimit;
+                            float xm = 0.f;
+                            hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_FAST, DUMP, false, true>(cbase, ch * CH, s_x, v, dY, 0.f, &xm);
+                            if (!__all_sync(0xffffffffu, xm <= kLimit)) {
+                                tmem_ld<CH>(c.taddr + ch * CH, v);
+                                ptx::tmem_wait_ld();
+                                hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_MIXED, DUMP>(cbase, ch * CH, s_x, v, dY, 0.f, nullptr, kLimit);
+                            }
+                            done = true;
+                        }
+                    }
+                    if (!done) hidden_chunk<W, CH, PER_TOKEN, ROT, EPI_SINE_WIDE, DUMP, GABOR>(cbase, ch * CH, s_x, v, dY, p.gabor_c);
+                }
                 tmem_st<CH>(c.taddr + ch * CH, v);
             }
             if constexpr (DUMP) dC = (valid && p.d.codes[l]) ? p.d.codes[l] + tok * W : nullptr;
@@ -1199,7 +1233,7 @@ __device__ void xy_role(const FusedParams &p, const SmemMap &sm, uint32_t smem_b
 }
 
 template <int W, bool PER_TOKEN, bool ROT, bool SPREAD, bool AHEAD, bool DUMP = false, bool BOTH = false, bool CALIB = false,
-          bool GABOR = false>
+          bool GABOR = false, bool MIXED = false>
 __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_constant__ ParamsOf<DUMP> p)
 {
     using C = Cfg<W>;
@@ -1252,7 +1286,7 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
             const uint32_t *srcA = fixed ? ly.fxP : reinterpret_cast<const uint32_t *>(ly.cA);
             const uint32_t *srcB = fixed ? ly.fxB : reinterpret_cast<const uint32_t *>(ly.cB);
             const uint32_t *srcC = fixed ? ly.fxQ : reinterpret_cast<const uint32_t *>(ly.cA_lo);
-            const int areas = (l == 0) ? (fixed ? 3 : (BOTH ? 5 : 4)) : (ly.epi_mode == EPI_SINE_WIDE ? 3 : 2);
+            const int areas = (l == 0) ? (fixed ? 3 : (BOTH ? 5 : 4)) : ((ly.epi_mode == EPI_SINE_WIDE || ly.epi_mode == EPI_SINE_MIXED) ? 3 : 2);
             for (int i = threadIdx.x; i < W; i += C::THREADS) { // i: tensor-memory column, m: its feature
                 const int m = fused_feature(i, W);
                 d[i] = __ldg(srcA + m);
@@ -1272,7 +1306,7 @@ __global__ void __launch_bounds__(Cfg<W>::THREADS, 1) fused_kernel(const __grid_
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp < kEpiWarps) {
-        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP, BOTH, CALIB, GABOR>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
+        epilogue_role<W, PER_TOKEN, ROT, SPREAD, AHEAD, DUMP, BOTH, CALIB, GABOR, MIXED>(p, sm, smem_base, warp, lane, tmem_base, abort_flag);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_role<W, SPREAD, CALIB>(p, sm, smem_base, tmem_base, abort_flag);
     } else if (warp == kLoadWarp) {
@@ -1328,6 +1362,20 @@ template <int W, bool AHEAD_OK> fused_dump_fn pick_dump_width(bool per_token, bo
     if (rot) return per_token ? fused_kernel<W, true, true, false, AHEAD_OK, true> : fused_kernel<W, false, true, false, AHEAD_OK, true>;
     return per_token ? fused_kernel<W, true, false, false, AHEAD_OK, true> : fused_kernel<W, false, false, false, AHEAD_OK, true>;
 }
+// Per-token scales with a layer under EPI_SINE_MIXED: the instantiation that carries the tracked short
+// route and its redo (kept out of the others, whose code it would only make larger).  Not spread.
+template <int W, bool AHEAD_OK> fused_fn pick_mixed_width(bool rot, bool ahead)
+{
+    if (AHEAD_OK && ahead) return rot ? fused_kernel<W, true, true, false, AHEAD_OK, false, false, false, false, true>
+                                      : fused_kernel<W, true, false, false, AHEAD_OK, false, false, false, false, true>;
+    return rot ? fused_kernel<W, true, true, false, false, false, false, false, false, true>
+               : fused_kernel<W, true, false, false, false, false, false, false, false, true>;
+}
+template <int W, bool AHEAD_OK> fused_dump_fn pick_mixed_dump_width(bool rot)
+{
+    return rot ? fused_kernel<W, true, true, false, AHEAD_OK, true, false, false, false, true>
+               : fused_kernel<W, true, false, false, AHEAD_OK, true, false, false, false, true>;
+}
 // The two-sided transform's kernels: not spread, coordinates not fetched ahead.
 template <int W> fused_fn pick_both_width(bool per_token)
 {
@@ -1382,6 +1430,14 @@ fused_fn fused_pick_gabor_64(bool per_token, bool rot);
 fused_fn fused_pick_gabor_128(bool per_token, bool rot);
 fused_fn fused_pick_gabor_256(bool per_token, bool rot);
 fused_fn fused_pick_gabor_512(bool per_token, bool rot);
+fused_fn fused_pick_mixed_64(bool rot, bool ahead);
+fused_fn fused_pick_mixed_128(bool rot, bool ahead);
+fused_fn fused_pick_mixed_256(bool rot, bool ahead);
+fused_fn fused_pick_mixed_512(bool rot, bool ahead);
+fused_dump_fn fused_pick_mixed_dump_64(bool rot);
+fused_dump_fn fused_pick_mixed_dump_128(bool rot);
+fused_dump_fn fused_pick_mixed_dump_256(bool rot);
+fused_dump_fn fused_pick_mixed_dump_512(bool rot);
 fused_fn fused_pick_gabor_both_64(bool per_token);
 fused_fn fused_pick_gabor_both_128(bool per_token);
 fused_fn fused_pick_gabor_both_256(bool per_token);

@@ -9,6 +9,8 @@ fused_dump_fn fused_pick_dump_256(bool per_token, bool rot) { return pick_dump_w
 fused_fn fused_pick_both_256(bool per_token) { return pick_both_width<256>(per_token); }
 fused_dump_fn fused_pick_both_dump_256(bool per_token) { return pick_both_dump_width<256>(per_token); }
 fused_fn fused_pick_calib_256(bool rot, bool gabor, bool both) { return pick_calib_width<256>(rot, gabor, both); }
+fused_fn fused_pick_mixed_256(bool rot, bool ahead) { return pick_mixed_width<256, true>(rot, ahead); }
+fused_dump_fn fused_pick_mixed_dump_256(bool rot) { return pick_mixed_dump_width<256, true>(rot); }
 fused_fn fused_pick_gabor_256(bool per_token, bool rot) { return pick_gabor_width<256>(per_token, rot); }
 fused_dump_fn fused_pick_gabor_dump_256(bool per_token, bool rot) { return pick_gabor_dump_width<256>(per_token, rot); }
 fused_fn fused_pick_gabor_both_256(bool per_token) { return pick_gabor_both_width<256>(per_token); }

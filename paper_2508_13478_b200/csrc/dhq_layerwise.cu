@@ -115,6 +115,8 @@ __global__ void __launch_bounds__(LW_THREADS) layer_kernel(LayerArgs a)
                 y = sine_fixed((int)cs[t * K + 0], (int)cs[t * K + 1], a.fxP[m], a.fxQ[m], a.fxB[m]);
             else if (a.gabor_s0 > 0.0 && a.sine)
                 y = gabor_epilogue((float)acc[t], c_hi, c_lo, cB, (float)(a.gabor_s0 / a.omega0));
+            else if (a.epi_mode == EPI_SINE_MIXED)
+                y = epilogue_mixed((float)acc[t], c_hi, c_lo, cB, a.per_token ? kFastPhaseLimitPerToken : kFastPhaseLimit);
             else
                 y = epilogue(a.epi_mode, (float)acc[t], c_hi, c_lo, cB);
             if (a.dacc) a.dacc[tok * M + m] = acc[t];

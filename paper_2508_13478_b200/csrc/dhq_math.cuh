@@ -15,7 +15,9 @@ enum EpiMode : int {
                        // unsaturated inputs, quantization error of weights and activations included): sin.approx(fma(acc, c, B))
     EPI_SINE_WIDE = 2, // large phases: compensated phase and explicit 2*pi reduction
     EPI_SINE_FIXED = 3, // first layer with a per-tensor activation scale: phase in 32-bit fixed point
-    EPI_BOTH = 4       // two-sided transform: the layer kernel undoes the output-side rotation in fp64
+    EPI_BOTH = 4,      // two-sided transform: the layer kernel undoes the output-side rotation in fp64
+    EPI_SINE_MIXED = 5 // hidden layer without a bound below the limit: decided per value, x = fma(acc, c, B);
+                       // |x| <= limit -> sin.approx(x), else the compensated phase and explicit reduction
 };
 
 // Largest |omega0 z| for which EPI_SINE_FAST keeps the result within 1e-5 of an exact sine.  Worst
@@ -29,6 +31,10 @@ enum EpiMode : int {
 // fma result still has half the ulp: 0.95e-6 + 3.8e-6 + 1e-7 + 4.4e-6 = 9.3e-6.
 constexpr float kFastPhaseLimit = 36.0f;
 constexpr float kFastPhaseLimitPerToken = 32.0f;
+// Two-sided transform inside the fused kernel: acc' = H_M acc may pass 2^24, so its conversion to
+// fp32 adds a relative 2^-24 to the phase; with the limit at 24 rad the sum is 0.95e-6 (fma) + 2.9e-6
+// (constant, twice for a per-token scale) + 1.4e-6 (conversion) + 4.4e-6 (approximation) = 9.7e-6.
+constexpr float kMixedPhaseLimitBoth = 24.0f;
 
 __device__ __forceinline__ float qmax_of(int bits) { return (float)((1 << (bits - 1)) - 1); }
 
@@ -84,6 +90,16 @@ __device__ __forceinline__ float epilogue(int mode, float accf, float c_hi, floa
     if (mode == EPI_SINE_FAST) return sin_approx(__fmaf_rn(accf, c_hi, cb));
     if (mode == EPI_SINE_WIDE) return sin_wide(__fmaf_rn(accf, c_lo, __fmaf_rn(accf, c_hi, cb)));
     return __fmaf_rn(accf, c_hi, cb);
+}
+
+// EPI_SINE_MIXED: the rule is per value and depends on nothing but (acc, constants), so every kernel
+// that applies it gives the same bits.  The error terms listed at kFastPhaseLimit all grow with the
+// phase that is actually computed, so a value below the limit is as accurate as under EPI_SINE_FAST.
+__device__ __forceinline__ float epilogue_mixed(float accf, float c_hi, float c_lo, float cb, float limit)
+{
+    const float x = __fmaf_rn(accf, c_hi, cb);
+    if (fabsf(x) <= limit) return sin_approx(x);
+    return sin_wide(__fmaf_rn(accf, c_lo, x));
 }
 
 // Wavelet activation (reading of the paper's WIRE experiments, Section IV): the real Gabor wavelet

@@ -241,6 +241,51 @@ def test_free_running_chains_differ_only_through_code_flips_at_rounding_ties():
         dhq.dhq_destroy(h)
 
 
+@pytest.mark.parametrize("width,scale", [(64, 10.0), (256, 10.0), (512, 10.0), (128, 16.0), (256, 25.0)])
+def test_layers_without_a_phase_bound_decide_per_value(width, scale):
+    # Per-token scales and a hidden layer whose phase bound is beyond the short sine's limit (32 rad): the
+    # rule is per value - below the limit sin.approx of the plain fma phase, above it the compensated phase
+    # with explicit reduction - and the fused kernel, which takes the short route for a whole chunk and
+    # redoes the chunk when a warp met a larger phase, must give the bits of the layer-by-layer kernel,
+    # which applies the rule value by value.  The weights are scaled so that both sides of the limit occur
+    # (scale 10: a fraction of a percent of the phases, in a third of the tokens; 16: a few percent, in nearly
+    # every token; 25: a fifth of them, phases to 130 rad).
+    # (Beyond 256 rad the fp32 phase itself carries half an ulp of 1.5e-5 or more: outside the 1e-5 claim.)
+    dims = (2, width, width, width, width, 3)
+    weights, biases = dhq_inputs.Workload("mixed", dims, 30.0, 2100 + width, 8, 8, 1, 1, (8, 8)).network()
+    weights[1] = (weights[1] * scale).astype(np.float32)
+    weights[2] = (weights[2] * scale).astype(np.float32)
+    n = 148 * (1 if width == 512 else 2) * 128 + 55
+    coords = dhq_inputs.grid_coords(241, 163)[:n]
+    h, net = prepare_pair(dims, weights, biases, 30.0, 8, 8, 1, 1)
+    try:
+        check_weights(h, net)
+        cd = to_dev(coords)
+        out_obs, bufs = run_debug(h, net, cd, fused=True)
+        check_layers_against_oracle(h, net, coords, out_obs, bufs)
+        for l in (2, 3):     # the phases that these layers really met, from the kernel's own accumulators and scales
+            lay = net.layers[l - 1]
+            acc = bufs["acc"][l - 1].cpu().numpy().astype(np.float64)
+            s_x = bufs["s_x"][l - 1].cpu().numpy().astype(np.float64)
+            phase = 30.0 * (acc * lay.s_w.astype(np.float64)[None, :] * s_x[:, None] + lay.b_pad.astype(np.float64)[None, :])
+            above = float((np.abs(phase) > 32.0).mean())
+            rows_clean = float((np.abs(phase).max(axis=1) <= 32.0).mean())
+            print(f"width {width} scale {scale} layer {l}: {above:.2%} of the phases above the limit, {rows_clean:.1%} of the tokens all below")
+            assert above > 1e-4
+            if scale <= 16:
+                assert above < 0.2
+        out_lw, bufs_lw = run_debug(h, net, cd)                  # layer by layer: the rule value by value
+        assert torch.equal(out_lw.view(torch.int32), out_obs.view(torch.int32))
+        for l in range(len(dims) - 1):
+            assert torch.equal(bufs_lw["Y"][l].view(torch.int32), bufs["Y"][l].view(torch.int32)), f"layer {l + 1} outputs"
+        out = torch.empty_like(out_obs)
+        dhq.dhq_forward(h, cd, out)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int32), out_obs.view(torch.int32))
+    finally:
+        dhq.dhq_destroy(h)
+
+
 @pytest.mark.parametrize("w_bits,a_bits,d_out,omega0,width,gran", [
     (2, 2, 3, 30.0, 256, 0), (2, 2, 1, 30.0, 128, 1), (3, 5, 2, 30.0, 64, 1), (4, 8, 4, 30.0, 256, 1), (8, 4, 3, 30.0, 512, 0),
     (7, 7, 4, 30.0, 512, 1), (8, 8, 2, -30.0, 256, 0), (8, 8, 3, 1.0, 128, 0), (8, 8, 1, 75.0, 256, 1), (8, 8, 3, 75.0, 512, 0),
